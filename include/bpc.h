@@ -1,0 +1,150 @@
+/*
+ * bpc.h - C-ABI of the BinaryPC decode-time sparse-attention library (single GPU, sm_100a).
+ *
+ * The library implements the per-token hot path of "Training-Free Hashing-Based Attention via
+ * Binary Principal Components": fit the per-head hash projection (Algorithm 1), encode cached keys
+ * (Algorithm 2), append a code on every cache write, and per decode step hash the query, score it
+ * against every packed key code (Algorithm 3), keep the top-k keys per KV head and run softmax
+ * attention over those rows only (Section 3.2, "Retrieval Phase").
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer owned by the caller unless its name starts with host_.
+ *     The library allocates device memory only inside bpc_create (state of the context) and frees
+ *     it in bpc_destroy.  No entry point copies, resizes or keeps caller buffers beyond the call.
+ *   - Every compute call is asynchronous on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     legacy default stream) and returns a bpc_status; nothing aborts, traps or prints.
+ *   - Layouts (row-major, contiguous):
+ *       k_cache, v_cache : [batch][n_kv_heads][n_max][head_dim]   kv_dtype, base 16-byte aligned
+ *       codes            : [batch][n_kv_heads][n_max][code_bits/64] uint64
+ *                          bit j of a key (Algorithm 2 iteration j+1) is word j/64, bit j%64,
+ *                          least significant first; 1 means the component is +1 (decision value >= 0)
+ *       q                : [batch][n_q_heads][head_dim]            kv_dtype
+ *       out              : [batch][n_q_heads][head_dim]            float
+ *       k_new, v_new     : [batch][n_kv_heads][head_dim]           kv_dtype
+ *       projection P     : [hash_sets][code_bits][head_dim]        float
+ *     Query head hq belongs to KV head hq / (n_q_heads / n_kv_heads).  A "unit" is one
+ *     (sequence, KV head) pair, unit = sequence * n_kv_heads + kv_head.
+ *   - Limits: head_dim == 128; code_bits in {64,128,256}; n_q_heads a multiple of n_kv_heads with
+ *     at most 8 query heads per KV head; n_max <= bpc_max_context(cfg).
+ */
+#ifndef BPC_H_
+#define BPC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  BPC_OK = 0,
+  BPC_ERR_INVALID_ARG = 1,   /* null / misaligned pointer, bad size */
+  BPC_ERR_UNSUPPORTED = 2,   /* shape or mode outside the limits above */
+  BPC_ERR_CAPACITY = 3,      /* a sequence would exceed n_max; nothing was written */
+  BPC_ERR_NOT_FITTED = 4,    /* a call needs the projection before bpc_fit / bpc_set_projection */
+  BPC_ERR_CUDA = 5,          /* a CUDA runtime call failed (see bpc_last_cuda_error) */
+  BPC_ERR_DEVICE = 6         /* a kernel reported an internal error through the device error word */
+} bpc_status;
+
+typedef enum { BPC_BF16 = 0, BPC_F32 = 1 } bpc_dtype;
+
+/* Algorithm 3 with one magnitude plane (all magnitudes 1: Hamming similarity) or the paper's
+ * sign + seven magnitude planes. */
+typedef enum { BPC_SCORE_HAMMING = 0, BPC_SCORE_WEIGHTED7 = 1 } bpc_score_mode;
+
+typedef struct {
+  int32_t batch;
+  int32_t n_q_heads;
+  int32_t n_kv_heads;
+  int32_t head_dim;             /* 128 */
+  int32_t code_bits;            /* 64 | 128 | 256 */
+  int32_t n_max;                /* rows per unit in the caches and the code array */
+  int32_t kv_dtype;             /* bpc_dtype */
+  int32_t score_mode;           /* bpc_score_mode */
+  float   sm_scale;             /* softmax scale; 0 selects 1/sqrt(head_dim) */
+  int32_t hash_sets;            /* batch*n_kv_heads (one projection per unit) or n_kv_heads (shared per KV head) */
+  int32_t residual_correction;  /* 1: Algorithm 2 (default). 0: plain sign(k P^T), for comparison only */
+} bpc_config;
+
+typedef struct bpc_ctx bpc_ctx;
+
+/* Context life cycle.  bpc_create validates cfg, allocates the projection, Gram matrix, per-unit
+ * lengths, a selected-index scratch list and the device error word on the current device. */
+bpc_status bpc_create(const bpc_config* host_cfg, bpc_ctx** host_out);
+bpc_status bpc_destroy(bpc_ctx* ctx);
+
+/* Sizes the caller needs: bytes of the code array, bytes of the workspace bpc_fit needs, the largest
+ * n_max this build supports for cfg (scores of one unit are kept in the shared memory of one thread
+ * block cluster), and the most keys a decode step can select per unit (= n_max). */
+size_t  bpc_codes_bytes(const bpc_config* host_cfg);
+size_t  bpc_fit_workspace_bytes(const bpc_config* host_cfg);
+/* Byte offset inside the fit workspace at which bpc_fit leaves the codes H that Algorithm 1 itself
+ * assigns to the fitted keys ([units][n_max][code_bits/64] uint64, same bit layout as `codes`).  They are a
+ * diagnostic: the cache codes always come from Algorithm 2 (bpc_encode_keys). */
+size_t  bpc_fit_codes_offset(const bpc_config* host_cfg);
+int64_t bpc_max_context(const bpc_config* host_cfg);
+
+/* Current number of cached keys of every sequence (host array [batch]).  Setting it uploads the
+ * lengths asynchronously; the context keeps a host shadow that bpc_append advances, so capacity
+ * errors are raised before any launch. */
+bpc_status bpc_set_seq_lens(bpc_ctx* ctx, const int32_t* host_lens, void* stream);
+bpc_status bpc_get_seq_lens(bpc_ctx* ctx, int32_t* host_lens_out);
+
+/* Algorithm 1 (Section 3.2, "Binary Principal Components Finding"): for every unit, run code_bits
+ * greedy iterations on its first seq_len keys of k_cache.  v_star [hash_sets][code_bits][head_dim]
+ * float are the Gaussian directions the algorithm samples (supplied by the caller so that a run is
+ * reproducible).  workspace must hold bpc_fit_workspace_bytes(cfg).  Requires hash_sets ==
+ * batch*n_kv_heads.  Leaves P, P rounded to the cache precision (the hash function proper) and
+ * its Gram matrix in the context. */
+bpc_status bpc_fit(bpc_ctx* ctx, const void* k_cache, const float* v_star,
+                   void* workspace, size_t workspace_bytes, void* stream);
+
+/* Offline-calibrated projection (Section 3.2, "Offline Projection Calibration"): install a caller
+ * supplied P [hash_sets][code_bits][head_dim] float instead of fitting. */
+bpc_status bpc_set_projection(bpc_ctx* ctx, const float* P, void* stream);
+
+/* Copy out the projection (float), its cache-precision rounding as float values, and the Gram
+ * matrix [hash_sets][code_bits][code_bits] float.  Any pointer may be NULL. */
+bpc_status bpc_get_projection(bpc_ctx* ctx, float* P_out, float* P_hash_out, float* gram_out, void* stream);
+
+/* Algorithm 2 for the first seq_len keys of every unit: codes[unit][0..seq_len). */
+bpc_status bpc_encode_keys(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, void* stream);
+
+/* Cache write of one new (k, v) row per unit at position seq_len, Algorithm 2 on the new key, its
+ * code stored beside the others, seq_len += 1 (on the device and in the host shadow).
+ * Returns BPC_ERR_CAPACITY, with nothing written, if any sequence is already at n_max. */
+bpc_status bpc_append(bpc_ctx* ctx, const void* k_new, const void* v_new,
+                      void* k_cache, void* v_cache, uint64_t* codes, void* stream);
+
+/* One decode step (Section 3.2 "Retrieval Phase", Algorithm 3, Appendix "CUDA Optimizations"):
+ * hash the queries of each KV head, score every cached key of the unit, keep the k keys with the
+ * highest score (ties to the lowest index) and write softmax(sm_scale q K_S^T) V_S for every query
+ * head.  k = budget_count if > 0 else ceil(seq_len * budget_ppm / 1e6), never more than seq_len;
+ * it is computed on the device from the device-side lengths.  sel_idx, if not NULL, receives the
+ * selected indices of each unit in ascending order, [units][n_max] int32 (first k entries). */
+bpc_status bpc_decode_attn(bpc_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
+                           const uint64_t* codes, int32_t budget_ppm, int32_t budget_count,
+                           float* out, int32_t* sel_idx, void* stream);
+
+/* Parity aids.  When set (non-NULL), the next bpc_decode_attn calls also write the integer hash
+ * score of every cached key (scores [units][n_max] int32) and the collapsed integer query weights
+ * A = sum over the group's heads of sign*magnitude (qweights [units][code_bits] int32). */
+bpc_status bpc_debug_set_buffers(bpc_ctx* ctx, int32_t* scores, int32_t* qweights);
+
+/* Launch geometry of the decode kernel: thread blocks per cluster (0 = choose automatically).
+ * Returns BPC_ERR_UNSUPPORTED if n_max does not fit that many blocks. */
+bpc_status bpc_set_cluster_size(bpc_ctx* ctx, int32_t cluster_size);
+int32_t    bpc_get_cluster_size(bpc_ctx* ctx);
+
+/* Diagnostics: device error word (synchronises the stream), last CUDA error code seen by the
+ * context, number of kernels this context has launched so far. */
+bpc_status bpc_last_device_error(bpc_ctx* ctx, int32_t* host_out, void* stream);
+int32_t    bpc_last_cuda_error(bpc_ctx* ctx);
+int64_t    bpc_launch_count(bpc_ctx* ctx);
+const char* bpc_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BPC_H_ */

@@ -1,0 +1,306 @@
+// C-ABI entry points: argument validation, context life cycle, stream plumbing.
+#include <new>
+#include <string.h>
+#include "common.cuh"
+
+cudaError_t bpc_launch_decode_bf16(bpc_ctx*, const DecodeParams&, cudaStream_t);
+cudaError_t bpc_launch_decode_f32(bpc_ctx*, const DecodeParams&, cudaStream_t);
+cudaError_t bpc_decode_limits_bf16(const bpc_ctx*, int, int*, int*, size_t*);
+cudaError_t bpc_decode_limits_f32(const bpc_ctx*, int, int*, int*, size_t*);
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bpc_status check_cfg(const bpc_config* c) {
+  if (c == nullptr) return BPC_ERR_INVALID_ARG;
+  if (c->batch < 1 || c->n_kv_heads < 1 || c->n_q_heads < 1 || c->n_max < 1) return BPC_ERR_INVALID_ARG;
+  if (c->head_dim != BPC_D) return BPC_ERR_UNSUPPORTED;
+  if (c->code_bits != 64 && c->code_bits != 128 && c->code_bits != 256) return BPC_ERR_UNSUPPORTED;
+  if (c->n_q_heads % c->n_kv_heads != 0) return BPC_ERR_INVALID_ARG;
+  if (c->n_q_heads / c->n_kv_heads > BPC_MAX_GROUP) return BPC_ERR_UNSUPPORTED;
+  if (c->kv_dtype != BPC_BF16 && c->kv_dtype != BPC_F32) return BPC_ERR_UNSUPPORTED;
+  if (c->score_mode != BPC_SCORE_HAMMING && c->score_mode != BPC_SCORE_WEIGHTED7) return BPC_ERR_INVALID_ARG;
+  if (c->score_mode == BPC_SCORE_WEIGHTED7) return BPC_ERR_UNSUPPORTED;   // not built yet
+  const long long units = (long long)c->batch * c->n_kv_heads;
+  if (c->hash_sets != units && c->hash_sets != c->n_kv_heads) return BPC_ERR_INVALID_ARG;
+  if (c->residual_correction != 0 && c->residual_correction != 1) return BPC_ERR_INVALID_ARG;
+  if (!(c->sm_scale >= 0.f)) return BPC_ERR_INVALID_ARG;
+  if (c->n_max % 2 != 0) return BPC_ERR_INVALID_ARG;   // keeps every unit's code rows 16-byte aligned at 64 bits
+  return BPC_OK;
+}
+
+bpc_status cuda_fail(bpc_ctx* ctx, cudaError_t e) {
+  if (ctx) ctx->last_cuda_error = (int32_t)e;
+  (void)cudaGetLastError();
+  return BPC_ERR_CUDA;
+}
+
+cudaError_t decode_limits(const bpc_ctx* ctx, int cs, int* max_cluster, int* chunk_cap, size_t* smem) {
+  return ctx->cfg.kv_dtype == BPC_BF16 ? bpc_decode_limits_bf16(ctx, cs, max_cluster, chunk_cap, smem)
+                                       : bpc_decode_limits_f32(ctx, cs, max_cluster, chunk_cap, smem);
+}
+
+int hamming_bins(const bpc_ctx* ctx) {
+  const int G = ctx->group;
+  const int cs = (G % 2 == 0) ? 1 : 0;
+  return ((G * ctx->cfg.code_bits) >> cs) + 1;
+}
+
+int chunk_for(int n_max, int cs) { return (((n_max + cs - 1) / cs) + 63) & ~63; }
+
+// Smallest power-of-two cluster whose blocks can hold n_max scores; then grow it while the whole grid
+// still fits one wave of the device.
+int choose_cluster(const bpc_ctx* ctx, int chunk_cap, int max_cluster) {
+  int cs = 1;
+  while (cs <= max_cluster && chunk_for(ctx->cfg.n_max, cs) > chunk_cap) cs *= 2;
+  if (cs > max_cluster) return 0;
+  while (cs * 2 <= max_cluster && (long long)ctx->units * cs * 2 <= ctx->sm_count &&
+         chunk_for(ctx->cfg.n_max, cs * 2) >= 1024)
+    cs *= 2;
+  return cs;
+}
+
+}  // namespace
+
+extern "C" {
+#pragma GCC visibility push(default)
+
+const char* bpc_version(void) { return "bpc 0.1 (sm_100a)"; }
+
+size_t bpc_codes_bytes(const bpc_config* c) {
+  if (check_cfg(c) != BPC_OK) return 0;
+  return (size_t)c->batch * c->n_kv_heads * (size_t)c->n_max * (c->code_bits / 8);
+}
+
+size_t bpc_fit_workspace_bytes(const bpc_config* c) {
+  if (check_cfg(c) != BPC_OK) return 0;
+  return bpc_fit_workspace_bytes_impl(c);
+}
+
+size_t bpc_fit_codes_offset(const bpc_config* c) {
+  if (check_cfg(c) != BPC_OK) return 0;
+  return bpc_fit_codes_offset_impl(c);
+}
+
+int64_t bpc_max_context(const bpc_config* c) {
+  if (check_cfg(c) != BPC_OK) return 0;
+  bpc_ctx tmp;
+  memset(&tmp, 0, sizeof(tmp));
+  tmp.cfg = *c;
+  tmp.group = c->n_q_heads / c->n_kv_heads;
+  if (cudaGetDevice(&tmp.device) != cudaSuccess) return 0;
+  int max_cluster = 1, cap = 0;
+  if (decode_limits(&tmp, 0, &max_cluster, &cap, nullptr) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+  return (int64_t)max_cluster * cap;
+}
+
+bpc_status bpc_create(const bpc_config* cfg, bpc_ctx** out) {
+  if (out == nullptr) return BPC_ERR_INVALID_ARG;
+  *out = nullptr;
+  bpc_status s = check_cfg(cfg);
+  if (s != BPC_OK) return s;
+  bpc_ctx* ctx = new (std::nothrow) bpc_ctx;
+  if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
+  memset(ctx, 0, sizeof(*ctx));
+  ctx->cfg = *cfg;
+  if (ctx->cfg.sm_scale == 0.f) ctx->cfg.sm_scale = 0.08838834764831845f;   // 1/sqrt(128)
+  ctx->units = cfg->batch * cfg->n_kv_heads;
+  ctx->group = cfg->n_q_heads / cfg->n_kv_heads;
+  cudaError_t e = cudaGetDevice(&ctx->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device);
+  const size_t b = cfg->code_bits, hs = cfg->hash_sets;
+  const size_t esz = cfg->kv_dtype == BPC_BF16 ? 2 : 4;
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->P, hs * b * BPC_D * 4);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->P_h, hs * b * BPC_D * esz);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->P_hf, hs * b * BPC_D * 4);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->gram, hs * b * b * 4);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->unit_lens, (size_t)ctx->units * 4);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->sel_scratch, (size_t)ctx->units * cfg->n_max * 4);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->dev_err, 4);
+  if (e == cudaSuccess) e = cudaMemset(ctx->dev_err, 0, 4);
+  if (e == cudaSuccess) e = cudaMemset(ctx->unit_lens, 0, (size_t)ctx->units * 4);
+  ctx->host_lens = new (std::nothrow) int32_t[cfg->batch];
+  if (ctx->host_lens) memset(ctx->host_lens, 0, sizeof(int32_t) * cfg->batch);
+  if (e != cudaSuccess || ctx->host_lens == nullptr) {
+    bpc_destroy(ctx);
+    (void)cudaGetLastError();
+    return BPC_ERR_CUDA;
+  }
+  int cap = 0;
+  e = decode_limits(ctx, 0, &ctx->max_cluster, &cap, nullptr);
+  if (e != cudaSuccess) { bpc_destroy(ctx); (void)cudaGetLastError(); return BPC_ERR_CUDA; }
+  ctx->chunk_cap_limit = cap;
+  ctx->cluster_size = choose_cluster(ctx, cap, ctx->max_cluster);
+  if (ctx->cluster_size == 0) { bpc_destroy(ctx); return BPC_ERR_UNSUPPORTED; }
+  if (hamming_bins(ctx) > 2048) { bpc_destroy(ctx); return BPC_ERR_UNSUPPORTED; }
+  *out = ctx;
+  return BPC_OK;
+}
+
+bpc_status bpc_destroy(bpc_ctx* ctx) {
+  if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
+  cudaFree(ctx->P); cudaFree(ctx->P_h); cudaFree(ctx->P_hf); cudaFree(ctx->gram);
+  cudaFree(ctx->unit_lens); cudaFree(ctx->sel_scratch); cudaFree(ctx->dev_err);
+  delete[] ctx->host_lens;
+  delete ctx;
+  (void)cudaGetLastError();
+  return BPC_OK;
+}
+
+bpc_status bpc_set_cluster_size(bpc_ctx* ctx, int32_t cs) {
+  if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
+  const int cap = ctx->chunk_cap_limit, mc = ctx->max_cluster;
+  if (cs == 0) cs = choose_cluster(ctx, cap, mc);
+  if (cs < 1 || cs > mc || (cs & (cs - 1)) != 0) return BPC_ERR_UNSUPPORTED;
+  if (chunk_for(ctx->cfg.n_max, cs) > cap) return BPC_ERR_UNSUPPORTED;
+  ctx->cluster_size = cs;
+  return BPC_OK;
+}
+
+int32_t bpc_get_cluster_size(bpc_ctx* ctx) { return ctx ? ctx->cluster_size : 0; }
+
+bpc_status bpc_set_seq_lens(bpc_ctx* ctx, const int32_t* host_lens, void* stream) {
+  if (ctx == nullptr || host_lens == nullptr) return BPC_ERR_INVALID_ARG;
+  const bpc_config& c = ctx->cfg;
+  for (int i = 0; i < c.batch; ++i)
+    if (host_lens[i] < 0 || host_lens[i] > c.n_max) return BPC_ERR_CAPACITY;
+  // expand to per-unit lengths through a small pageable staging array: the copy is synchronous with
+  // respect to the host buffer, so the temporary can be released on return
+  int32_t* tmp = new (std::nothrow) int32_t[ctx->units];
+  if (tmp == nullptr) return BPC_ERR_INVALID_ARG;
+  for (int i = 0; i < c.batch; ++i) {
+    ctx->host_lens[i] = host_lens[i];
+    for (int h = 0; h < c.n_kv_heads; ++h) tmp[i * c.n_kv_heads + h] = host_lens[i];
+  }
+  cudaError_t e = cudaMemcpyAsync(ctx->unit_lens, tmp, (size_t)ctx->units * 4, cudaMemcpyHostToDevice, (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+  delete[] tmp;
+  return e == cudaSuccess ? BPC_OK : cuda_fail(ctx, e);
+}
+
+bpc_status bpc_get_seq_lens(bpc_ctx* ctx, int32_t* host_out) {
+  if (ctx == nullptr || host_out == nullptr) return BPC_ERR_INVALID_ARG;
+  for (int i = 0; i < ctx->cfg.batch; ++i) host_out[i] = ctx->host_lens[i];
+  return BPC_OK;
+}
+
+bpc_status bpc_set_projection(bpc_ctx* ctx, const float* P, void* stream) {
+  if (ctx == nullptr || P == nullptr) return BPC_ERR_INVALID_ARG;
+  const bpc_config& c = ctx->cfg;
+  cudaError_t e = cudaMemcpyAsync(ctx->P, P, (size_t)c.hash_sets * c.code_bits * BPC_D * 4, cudaMemcpyDeviceToDevice,
+                                  (cudaStream_t)stream);
+  if (e == cudaSuccess) e = bpc_launch_finalize_projection(ctx, (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  ctx->fitted = true;
+  return BPC_OK;
+}
+
+bpc_status bpc_get_projection(bpc_ctx* ctx, float* P_out, float* Ph_out, float* gram_out, void* stream) {
+  if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
+  if (!ctx->fitted) return BPC_ERR_NOT_FITTED;
+  const bpc_config& c = ctx->cfg;
+  const size_t pb = (size_t)c.hash_sets * c.code_bits * BPC_D * 4;
+  cudaError_t e = cudaSuccess;
+  if (P_out) e = cudaMemcpyAsync(P_out, ctx->P, pb, cudaMemcpyDeviceToDevice, (cudaStream_t)stream);
+  if (e == cudaSuccess && Ph_out) e = cudaMemcpyAsync(Ph_out, ctx->P_hf, pb, cudaMemcpyDeviceToDevice, (cudaStream_t)stream);
+  if (e == cudaSuccess && gram_out)
+    e = cudaMemcpyAsync(gram_out, ctx->gram, (size_t)c.hash_sets * c.code_bits * c.code_bits * 4, cudaMemcpyDeviceToDevice,
+                        (cudaStream_t)stream);
+  return e == cudaSuccess ? BPC_OK : cuda_fail(ctx, e);
+}
+
+bpc_status bpc_fit(bpc_ctx* ctx, const void* k_cache, const float* v_star, void* workspace, size_t workspace_bytes,
+                   void* stream) {
+  if (ctx == nullptr || k_cache == nullptr || v_star == nullptr || workspace == nullptr) return BPC_ERR_INVALID_ARG;
+  if (!aligned16(k_cache) || !aligned16(v_star) || !aligned16(workspace)) return BPC_ERR_INVALID_ARG;
+  if (ctx->cfg.hash_sets != ctx->units) return BPC_ERR_UNSUPPORTED;
+  if (workspace_bytes < bpc_fit_workspace_bytes_impl(&ctx->cfg)) return BPC_ERR_INVALID_ARG;
+  int launches = 0;
+  cudaError_t e = bpc_launch_fit(ctx, k_cache, v_star, workspace, (cudaStream_t)stream, &launches);
+  ctx->launches += launches;
+  if (e == cudaSuccess) e = bpc_launch_finalize_projection(ctx, (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  ctx->fitted = true;
+  return BPC_OK;
+}
+
+bpc_status bpc_encode_keys(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, void* stream) {
+  if (ctx == nullptr || k_cache == nullptr || codes == nullptr) return BPC_ERR_INVALID_ARG;
+  if (!aligned16(k_cache) || !aligned16(codes)) return BPC_ERR_INVALID_ARG;
+  if (!ctx->fitted) return BPC_ERR_NOT_FITTED;
+  cudaError_t e = bpc_launch_encode_tc(ctx, k_cache, codes, (cudaStream_t)stream);
+  if (e == cudaErrorNotSupported) {
+    (void)cudaGetLastError();
+    e = bpc_launch_encode_simple(ctx, k_cache, codes, (cudaStream_t)stream);
+  }
+  return e == cudaSuccess ? BPC_OK : cuda_fail(ctx, e);
+}
+
+bpc_status bpc_append(bpc_ctx* ctx, const void* k_new, const void* v_new, void* k_cache, void* v_cache, uint64_t* codes,
+                      void* stream) {
+  if (ctx == nullptr || k_new == nullptr || v_new == nullptr || k_cache == nullptr || v_cache == nullptr || codes == nullptr)
+    return BPC_ERR_INVALID_ARG;
+  if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(codes))
+    return BPC_ERR_INVALID_ARG;
+  if (!ctx->fitted) return BPC_ERR_NOT_FITTED;
+  for (int i = 0; i < ctx->cfg.batch; ++i)
+    if (ctx->host_lens[i] >= ctx->cfg.n_max) return BPC_ERR_CAPACITY;
+  cudaError_t e = bpc_launch_append(ctx, k_new, v_new, k_cache, v_cache, codes, (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  for (int i = 0; i < ctx->cfg.batch; ++i) ctx->host_lens[i] += 1;
+  return BPC_OK;
+}
+
+bpc_status bpc_decode_attn(bpc_ctx* ctx, const void* q, const void* k_cache, const void* v_cache, const uint64_t* codes,
+                           int32_t budget_ppm, int32_t budget_count, float* out, int32_t* sel_idx, void* stream) {
+  if (ctx == nullptr || q == nullptr || k_cache == nullptr || v_cache == nullptr || codes == nullptr || out == nullptr)
+    return BPC_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(codes) || !aligned16(out))
+    return BPC_ERR_INVALID_ARG;
+  if (sel_idx != nullptr && !aligned16(sel_idx)) return BPC_ERR_INVALID_ARG;
+  if (budget_ppm < 0 || budget_ppm > 1000000 || budget_count < 0) return BPC_ERR_INVALID_ARG;
+  if (budget_ppm == 0 && budget_count == 0) return BPC_ERR_INVALID_ARG;
+  if (!ctx->fitted) return BPC_ERR_NOT_FITTED;
+  const bpc_config& c = ctx->cfg;
+  const int cap = ctx->chunk_cap_limit;
+  cudaError_t e;
+  DecodeParams p;
+  memset(&p, 0, sizeof(p));
+  p.q = q; p.k_cache = k_cache; p.v_cache = v_cache; p.codes = codes; p.P_h = ctx->P_h;
+  p.unit_lens = ctx->unit_lens; p.out = out;
+  p.sel = sel_idx != nullptr ? sel_idx : ctx->sel_scratch;
+  p.dbg_scores = ctx->dbg_scores; p.dbg_qweights = ctx->dbg_qweights; p.err = ctx->dev_err;
+  p.n_kv_heads = c.n_kv_heads; p.group = ctx->group; p.n_max = c.n_max;
+  p.shared_sets = c.hash_sets != ctx->units;
+  p.budget_ppm = budget_ppm; p.budget_count = budget_count; p.sm_scale = c.sm_scale;
+  const int chunk = chunk_for(c.n_max, ctx->cluster_size);
+  if (chunk > cap) return BPC_ERR_UNSUPPORTED;
+  p.chunk_cap = chunk;                                    // shared memory is sized for the largest possible unit
+  p.nbins = hamming_bins(ctx);
+  e = c.kv_dtype == BPC_BF16 ? bpc_launch_decode_bf16(ctx, p, (cudaStream_t)stream)
+                             : bpc_launch_decode_f32(ctx, p, (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  ctx->launches += 1;
+  return BPC_OK;
+}
+
+bpc_status bpc_debug_set_buffers(bpc_ctx* ctx, int32_t* scores, int32_t* qweights) {
+  if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
+  ctx->dbg_scores = scores;
+  ctx->dbg_qweights = qweights;
+  return BPC_OK;
+}
+
+bpc_status bpc_last_device_error(bpc_ctx* ctx, int32_t* host_out, void* stream) {
+  if (ctx == nullptr || host_out == nullptr) return BPC_ERR_INVALID_ARG;
+  cudaError_t e = cudaMemcpyAsync(host_out, ctx->dev_err, 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+  return e == cudaSuccess ? BPC_OK : cuda_fail(ctx, e);
+}
+
+int32_t bpc_last_cuda_error(bpc_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+int64_t bpc_launch_count(bpc_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+#pragma GCC visibility pop
+}  // extern "C"

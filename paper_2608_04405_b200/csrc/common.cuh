@@ -1,0 +1,110 @@
+// Shared declarations of the BinaryPC CUDA library (device helpers, context, launch parameters).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "../../include/bpc.h"
+
+#define BPC_D 128            // head_dim (the paper's models all use 128)
+#define BPC_MAX_GROUP 8
+#define BPC_MAX_CLUSTER 16
+
+// Device error word bits.
+#define BPC_DEVERR_CHUNK_CAP   1   // a unit does not fit the cluster's score storage
+#define BPC_DEVERR_APPEND_CAP  2   // append at n_max
+#define BPC_DEVERR_TIMEOUT     4   // a bounded wait gave up
+
+struct bpc_ctx {
+  bpc_config cfg;
+  int device;
+  int units;                // batch * n_kv_heads
+  int group;                // query heads per KV head
+  int cluster_size;         // decode: thread blocks per cluster
+  int max_cluster;          // largest cluster size the device schedules for the decode kernel
+  int sm_count;
+  bool fitted;
+  float* P;                 // [hash_sets][b][D] float
+  void*  P_h;               // [hash_sets][b][D] cache dtype (the hash function)
+  float* P_hf;              // P_h as float values
+  float* gram;              // [hash_sets][b][b] float, P_h P_h^T
+  int32_t* unit_lens;       // [units] device
+  int32_t* host_lens;       // [batch] host shadow
+  int32_t* sel_scratch;     // [units][n_max] int32
+  int32_t* dev_err;         // device error word
+  int32_t* dbg_scores;      // caller buffers (may be null)
+  int32_t* dbg_qweights;
+  int32_t last_cuda_error;
+  int64_t launches;
+  int chunk_cap_limit;      // keys one decode block can hold with all opt-in shared memory
+  size_t decode_smem_set;   // non-zero once the decode kernel's function attributes have been set
+};
+
+struct DecodeParams {
+  const void* q;
+  const void* k_cache;
+  const void* v_cache;
+  const uint64_t* codes;
+  const void* P_h;
+  const int32_t* unit_lens;
+  float* out;
+  int32_t* sel;              // [units][n_max]
+  int32_t* dbg_scores;
+  int32_t* dbg_qweights;
+  int32_t* err;
+  int n_kv_heads;
+  int group;
+  int n_max;
+  int shared_sets;           // 1: projection shared per KV head, 0: one per unit
+  int budget_ppm;
+  int budget_count;
+  float sm_scale;
+  int chunk_cap;             // keys whose scores one thread block can hold
+  int nbins;                 // histogram bins (largest score key + 1)
+};
+
+// ---- launchers implemented in the per-dtype translation units
+
+// ---- prefill-side launchers (prefill.cu)
+cudaError_t bpc_launch_finalize_projection(bpc_ctx* ctx, cudaStream_t stream);
+cudaError_t bpc_launch_encode_simple(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStream_t stream);
+cudaError_t bpc_launch_append(bpc_ctx* ctx, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                              uint64_t* codes, cudaStream_t stream);
+cudaError_t bpc_launch_fit(bpc_ctx* ctx, const void* k_cache, const float* v_star, void* workspace,
+                           cudaStream_t stream, int* launches);
+size_t bpc_fit_workspace_bytes_impl(const bpc_config* cfg);
+size_t bpc_fit_codes_offset_impl(const bpc_config* cfg);
+
+// ---- tensor-core encode (encode_tc.cu); returns cudaErrorNotSupported when the shape is not covered
+cudaError_t bpc_launch_encode_tc(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStream_t stream);
+
+// --------------------------------------------------------------------------- device helpers
+#ifdef __CUDACC__
+__device__ __forceinline__ float bf16_lo(uint32_t x) { return __uint_as_float(x << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
+
+// 16-byte streaming load that does not allocate in L1 (data read once per step).
+__device__ __forceinline__ uint4 ld_stream_v4(const void* p) {
+  uint4 r;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+  return r;
+}
+__device__ __forceinline__ uint2 ld_stream_v2(const void* p) {
+  uint2 r;
+  asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p));
+  return r;
+}
+
+template <typename T> struct KvTraits;
+template <> struct KvTraits<__nv_bfloat16> {
+  typedef float acc_t;                 // bf16 products are exact in fp32
+  static constexpr int kBytes = 2;
+};
+template <> struct KvTraits<float> {
+  typedef double acc_t;                // fp32 caches: logits and averages in fp64 (1e-5 output tolerance)
+  static constexpr int kBytes = 4;
+};
+
+__device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ float to_float(float v) { return v; }
+#endif

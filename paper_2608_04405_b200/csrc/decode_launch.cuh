@@ -1,0 +1,111 @@
+// Host-side dispatch of the fused decode kernel for one cache dtype (included by decode_bf16.cu / decode_f32.cu).
+#pragma once
+#include "decode_kernel.cuh"
+
+namespace bpcdev {
+
+// The shared-memory ceiling is always raised to the device's opt-in maximum, so contexts with different
+// n_max can share one kernel instance.
+template <typename KV, int GP, int W32, int MODE>
+static cudaError_t configure_kernel(int device) {
+  auto kern = bpc_decode_kernel<KV, GP, W32, MODE>;
+  int optin = 0;
+  cudaError_t e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, optin);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+}
+
+template <typename KV, int GP, int W32, int MODE>
+static cudaError_t launch_one(bpc_ctx* ctx, const DecodeParams& p, cudaStream_t stream) {
+  typedef DecodeSmem<KV, GP, W32> L;
+  const size_t smem = L::total(p.chunk_cap);
+  cudaError_t e = cudaSuccess;
+  if (ctx->decode_smem_set == 0) {                          // function attributes are sticky: set them once
+    e = configure_kernel<KV, GP, W32, MODE>(ctx->device);
+    if (e != cudaSuccess) return e;
+    ctx->decode_smem_set = 1;
+  }
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3((unsigned)(ctx->units * ctx->cluster_size), 1, 1);
+  lc.blockDim = dim3(L::NT, 1, 1);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = (unsigned)ctx->cluster_size;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = 1;
+  lc.attrs = at;
+  lc.numAttrs = 1;
+  return cudaLaunchKernelEx(&lc, bpc_decode_kernel<KV, GP, W32, MODE>, p);
+}
+
+// Largest cluster size (power of two) the device can schedule with `smem` bytes per block, and the
+// shared-memory budget of one block.
+template <typename KV, int GP, int W32, int MODE>
+static cudaError_t limits_one(const bpc_ctx* ctx, int cluster_size, int* max_cluster, int* chunk_cap, size_t* smem_bytes) {
+  typedef DecodeSmem<KV, GP, W32> L;
+  int dev = ctx->device, optin = 0;
+  cudaError_t e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  if (e != cudaSuccess) return e;
+  // score capacity of one block: what is left of the opt-in shared memory after the fixed regions
+  const size_t fixed = L::off_scores;
+  size_t avail = (size_t)optin > fixed + 1024 ? (size_t)optin - fixed - 1024 : 0;
+  int cap = (int)((avail / (kSegSlots * 2)) * kSegKeys);
+  cap &= ~63;
+  if (chunk_cap) *chunk_cap = cap;
+  if (smem_bytes) *smem_bytes = (size_t)optin;
+  if (max_cluster) {
+    int best = 1;
+    for (int cs = 2; cs <= BPC_MAX_CLUSTER; cs *= 2) {
+      const size_t smem = L::total(cap);
+      e = configure_kernel<KV, GP, W32, MODE>(dev);
+      if (e != cudaSuccess) return e;
+      cudaLaunchConfig_t lc = {};
+      lc.gridDim = dim3((unsigned)cs, 1, 1);
+      lc.blockDim = dim3(L::NT, 1, 1);
+      lc.dynamicSmemBytes = smem;
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = (unsigned)cs; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+      lc.attrs = at; lc.numAttrs = 1;
+      int nclusters = 0;
+      cudaError_t q = cudaOccupancyMaxActiveClusters(&nclusters, bpc_decode_kernel<KV, GP, W32, MODE>, &lc);
+      if (q != cudaSuccess) { (void)cudaGetLastError(); break; }
+      if (nclusters < 1) break;
+      best = cs;
+    }
+    *max_cluster = best;
+  }
+  (void)cluster_size;
+  return cudaSuccess;
+}
+
+#define BPC_DISPATCH_W(KV, GP, MODE, FN, ...)                                        \
+  switch (ctx->cfg.code_bits) {                                                      \
+    case 64:  return FN<KV, GP, 2, MODE>(__VA_ARGS__);                               \
+    case 128: return FN<KV, GP, 4, MODE>(__VA_ARGS__);                               \
+    case 256: return FN<KV, GP, 8, MODE>(__VA_ARGS__);                               \
+    default:  return cudaErrorInvalidValue;                                          \
+  }
+
+#define BPC_DISPATCH_G(KV, MODE, FN, ...)                                            \
+  if (ctx->group == 1)      { BPC_DISPATCH_W(KV, 1, MODE, FN, __VA_ARGS__) }         \
+  else if (ctx->group == 2) { BPC_DISPATCH_W(KV, 2, MODE, FN, __VA_ARGS__) }         \
+  else if (ctx->group <= 4) { BPC_DISPATCH_W(KV, 4, MODE, FN, __VA_ARGS__) }         \
+  else                      { BPC_DISPATCH_W(KV, 8, MODE, FN, __VA_ARGS__) }
+
+template <typename KV>
+static cudaError_t launch_dtype(bpc_ctx* ctx, const DecodeParams& p, cudaStream_t stream) {
+  if (ctx->cfg.score_mode != BPC_SCORE_HAMMING) return cudaErrorNotSupported;
+  BPC_DISPATCH_G(KV, 0, launch_one, ctx, p, stream)
+}
+template <typename KV>
+static cudaError_t limits_dtype(const bpc_ctx* ctx, int cluster_size, int* max_cluster, int* chunk_cap, size_t* smem) {
+  if (ctx->cfg.score_mode != BPC_SCORE_HAMMING) return cudaErrorNotSupported;
+  BPC_DISPATCH_G(KV, 0, limits_one, ctx, cluster_size, max_cluster, chunk_cap, smem)
+}
+
+}  // namespace bpcdev

@@ -1,0 +1,381 @@
+// Prefill-side and cache-write kernels: projection finalisation, Algorithm 1 (fit), Algorithm 2 on CUDA
+// cores (fp32 caches and shapes the tensor-core encode does not cover), and the per-step append.
+#include "common.cuh"
+
+namespace {
+
+// --------------------------------------------------------------------------- projection finalisation
+// P (float) -> P_h in the cache dtype (the hash function is defined on these rounded values),
+// the same values as float, and the Gram matrix G = P_h P_h^T used by the Gram form of Algorithm 2:
+// t_i = k.P_i - sum_{j<i} u_j G_ji is the decision value r.P_i of the residual form.
+template <typename KV>
+__global__ void round_projection_kernel(const float* __restrict__ P, KV* __restrict__ Ph, float* __restrict__ Phf, size_t n) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) {
+    KV v = (KV)P[i];
+    Ph[i] = v;
+    Phf[i] = to_float(v);
+  }
+}
+template <> __global__ void round_projection_kernel<__nv_bfloat16>(const float* __restrict__ P, __nv_bfloat16* __restrict__ Ph,
+                                                                   float* __restrict__ Phf, size_t n) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) {
+    __nv_bfloat16 v = __float2bfloat16_rn(P[i]);
+    Ph[i] = v;
+    Phf[i] = __bfloat162float(v);
+  }
+}
+
+__global__ void gram_kernel(const float* __restrict__ Phf, float* __restrict__ gram, int b) {
+  // grid (b, hash_sets); thread j computes G[i][j] with fp64 accumulation
+  const int i = blockIdx.x, s = blockIdx.y;
+  const float* base = Phf + (size_t)s * b * BPC_D;
+  __shared__ float ri[BPC_D];
+  for (int c = threadIdx.x; c < BPC_D; c += blockDim.x) ri[c] = base[(size_t)i * BPC_D + c];
+  __syncthreads();
+  for (int j = threadIdx.x; j < b; j += blockDim.x) {
+    const float* rj = base + (size_t)j * BPC_D;
+    double acc = 0.0;
+    for (int c = 0; c < BPC_D; ++c) acc = fma((double)ri[c], (double)rj[c], acc);
+    gram[((size_t)s * b + i) * b + j] = (float)acc;
+  }
+}
+
+// --------------------------------------------------------------------------- Algorithm 2 on CUDA cores
+// One thread per key.  Decision values t = k P_h^T are accumulated in fp64 and kept as fp32 in shared
+// memory ([bit][thread]); the greedy sweep u_i = sign(t_i), t_j -= u_i G_ij (j > i) then runs per thread.
+constexpr int kEncThreads = 128;
+
+template <typename KV>
+__global__ void __launch_bounds__(kEncThreads)
+encode_simple_kernel(const KV* __restrict__ k_cache, const float* __restrict__ Phf, const float* __restrict__ gram,
+                     const int32_t* __restrict__ unit_lens, uint64_t* __restrict__ codes, int n_kv_heads, int n_max,
+                     int b, int shared_sets, int residual_correction) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  float* ps = reinterpret_cast<float*>(smem);                       // [128 rows of P][128]
+  float* ts = ps + 128 * BPC_D;                                      // [b][kEncThreads]
+  const int unit = blockIdx.y;
+  const int n = min(unit_lens[unit], n_max);
+  const int key = blockIdx.x * kEncThreads + threadIdx.x;
+  if (blockIdx.x * kEncThreads >= n) return;                         // whole block beyond the unit: uniform
+  const int set = shared_sets ? unit % n_kv_heads : unit;
+  const float* Pset = Phf + (size_t)set * b * BPC_D;
+  const float* Gset = gram + (size_t)set * b * b;
+  const bool live = key < n;
+  float kr[BPC_D];
+  {
+    const KV* row = k_cache + ((size_t)unit * n_max + (live ? key : 0)) * BPC_D;
+#pragma unroll
+    for (int c = 0; c < BPC_D; ++c) kr[c] = to_float(row[c]);
+  }
+  for (int jb = 0; jb < b; jb += 128) {
+    const int rows = min(128, b - jb);
+    __syncthreads();
+    for (int i = threadIdx.x; i < rows * BPC_D; i += kEncThreads) ps[i] = Pset[(size_t)jb * BPC_D + i];
+    __syncthreads();
+    for (int j = 0; j < rows; ++j) {
+      const float4* pr = reinterpret_cast<const float4*>(ps + j * BPC_D);
+      double a0 = 0, a1 = 0, a2 = 0, a3 = 0;
+#pragma unroll
+      for (int c4 = 0; c4 < BPC_D / 4; ++c4) {
+        const float4 pv = pr[c4];
+        a0 = fma((double)kr[4 * c4], (double)pv.x, a0);
+        a1 = fma((double)kr[4 * c4 + 1], (double)pv.y, a1);
+        a2 = fma((double)kr[4 * c4 + 2], (double)pv.z, a2);
+        a3 = fma((double)kr[4 * c4 + 3], (double)pv.w, a3);
+      }
+      ts[(size_t)(jb + j) * kEncThreads + threadIdx.x] = (float)((a0 + a1) + (a2 + a3));
+    }
+  }
+  uint32_t* dst = reinterpret_cast<uint32_t*>(codes + ((size_t)unit * n_max + (live ? key : 0)) * (b / 64));
+  uint32_t word = 0;
+  for (int i = 0; i < b; ++i) {
+    const float ti = ts[(size_t)i * kEncThreads + threadIdx.x];
+    const bool pos = ti >= 0.f;
+    word |= (pos ? 1u : 0u) << (i & 31);
+    if ((i & 31) == 31) {
+      if (live) dst[i >> 5] = word;
+      word = 0;
+    }
+    if (residual_correction) {
+      const float u = pos ? 1.f : -1.f;
+      const float* gi = Gset + (size_t)i * b;
+      for (int j = i + 1; j < b; ++j) ts[(size_t)j * kEncThreads + threadIdx.x] -= u * __ldg(gi + j);
+    }
+  }
+}
+
+// --------------------------------------------------------------------------- append (cache write + Algorithm 2 on one key)
+// One block per unit.  The decision values come from a warp-cooperative fp32 mat-vec; the greedy sweep is
+// split in 32-bit column blocks: warp B owns columns 32B..32B+31, sweeps its diagonal block with register
+// shuffles, publishes its 32 signs, and the later warps apply that rank-32 update.
+constexpr int kAppThreads = 256;
+
+template <typename KV>
+__global__ void __launch_bounds__(kAppThreads)
+append_kernel(const KV* __restrict__ k_new, const KV* __restrict__ v_new, KV* __restrict__ k_cache, KV* __restrict__ v_cache,
+              uint64_t* __restrict__ codes, const KV* __restrict__ Ph, const float* __restrict__ gram,
+              int32_t* __restrict__ unit_lens, int32_t* __restrict__ err, int n_kv_heads, int n_max, int b,
+              int shared_sets, int residual_correction) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  float* gs = reinterpret_cast<float*>(smem);                        // [b][b] when b <= 128
+  __shared__ float t_s[256];
+  __shared__ float k_s[BPC_D];
+  __shared__ uint32_t ubits_s[8];
+  const int unit = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n = unit_lens[unit];
+  if (n >= n_max || n < 0) {
+    if (tid == 0) atomicOr(err, BPC_DEVERR_APPEND_CAP);
+    return;
+  }
+  const int set = shared_sets ? unit % n_kv_heads : unit;
+  const float* Gset = gram + (size_t)set * b * b;
+  const bool g_in_smem = b <= 128;
+  if (g_in_smem && residual_correction) {
+    const float4* src = reinterpret_cast<const float4*>(Gset);
+    float4* dst = reinterpret_cast<float4*>(gs);
+    for (int i = tid; i < b * b / 4; i += kAppThreads) dst[i] = src[i];
+  }
+  const KV* kn = k_new + (size_t)unit * BPC_D;
+  const KV* vn = v_new + (size_t)unit * BPC_D;
+  if (tid < BPC_D) {
+    const KV kv = kn[tid];
+    k_s[tid] = to_float(kv);
+    k_cache[((size_t)unit * n_max + n) * BPC_D + tid] = kv;
+  } else if (tid < 2 * BPC_D) {
+    v_cache[((size_t)unit * n_max + n) * BPC_D + (tid - BPC_D)] = vn[tid - BPC_D];
+  }
+  __syncthreads();
+  // t_j = P_h[j] . k
+  {
+    const KV* Pset = Ph + (size_t)set * b * BPC_D;
+    const float k0 = k_s[4 * lane], k1 = k_s[4 * lane + 1], k2 = k_s[4 * lane + 2], k3 = k_s[4 * lane + 3];
+#pragma unroll 4
+    for (int j = warp; j < b; j += kAppThreads / 32) {
+      const KV* row = Pset + (size_t)j * BPC_D + 4 * lane;
+      float s = to_float(row[0]) * k0;
+      s = fmaf(to_float(row[1]), k1, s);
+      s = fmaf(to_float(row[2]), k2, s);
+      s = fmaf(to_float(row[3]), k3, s);
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      if (lane == 0) t_s[j] = s;
+    }
+  }
+  __syncthreads();
+  const int nb = b / 32;
+  const float* Gp = g_in_smem ? gs : Gset;
+  float t = warp < nb ? t_s[32 * warp + lane] : 0.f;
+  float gd[32];                                                      // diagonal block column of this lane
+  if (warp < nb && residual_correction) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) gd[i] = Gp[(size_t)(32 * warp + i) * b + 32 * warp + lane];
+  }
+  for (int blk = 0; blk < nb; ++blk) {
+    if (warp == blk) {
+      uint32_t bits = 0;
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const float ti = __shfl_sync(0xffffffffu, t, i);
+        const bool pos = ti >= 0.f;
+        bits |= (pos ? 1u : 0u) << i;
+        if (residual_correction && lane > i) t -= pos ? gd[i] : -gd[i];
+      }
+      if (lane == 0) {
+        ubits_s[blk] = bits;
+        reinterpret_cast<uint32_t*>(codes + ((size_t)unit * n_max + n) * (b / 64))[blk] = bits;
+      }
+    }
+    __syncthreads();
+    if (residual_correction && warp > blk && warp < nb) {
+      const uint32_t bits = ubits_s[blk];
+      const float* gcol = Gp + (size_t)(32 * blk) * b + 32 * warp + lane;
+      float a = 0.f;
+#pragma unroll 8
+      for (int i = 0; i < 32; ++i) {
+        const float g = gcol[(size_t)i * b];
+        a += ((bits >> i) & 1u) ? g : -g;
+      }
+      t -= a;
+    }
+  }
+  if (tid == 0) unit_lens[unit] = n + 1;
+}
+
+// --------------------------------------------------------------------------- Algorithm 1 (fit)
+// The residual R (fp32) lives in the workspace.  Iteration i is one pass over R:
+//   R_row -= u_{i-1}(row) * v_{i-1}   (skipped at i = 0, where R_row = K_row)
+//   t = R_row . v*_i ; u_i(row) = sign(t) ; partial[c] += u_i(row) * R_row[c]
+// followed by a small deterministic reduction v_i = sum(partials) / N.  One warp handles one row at a
+// time (4 channels per lane, coalesced 512-byte rows).
+constexpr int kFitThreads = 256;
+constexpr int kFitRowsPerBlock = 1024;
+
+template <typename KV>
+__global__ void __launch_bounds__(kFitThreads)
+fit_pass_kernel(const KV* __restrict__ k_cache, float* __restrict__ R, uint8_t* __restrict__ usign,
+                uint32_t* __restrict__ hfit, const float* __restrict__ v_star, const float* __restrict__ P, float* __restrict__ partials,
+                const int32_t* __restrict__ unit_lens, int n_max, int b, int it, int blocks_per_unit) {
+  const int unit = blockIdx.y;
+  const int n = min(unit_lens[unit], n_max);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int row0 = blockIdx.x * kFitRowsPerBlock;
+  __shared__ float red[kFitThreads / 32][BPC_D];
+  const float4 vs = reinterpret_cast<const float4*>(v_star + ((size_t)unit * b + it) * BPC_D)[lane];
+  float4 vp = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (it > 0) vp = reinterpret_cast<const float4*>(P + ((size_t)unit * b + (it - 1)) * BPC_D)[lane];
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  const int row_end = min(n, row0 + kFitRowsPerBlock);
+  for (int r = row0 + warp; r < row_end; r += kFitThreads / 32) {
+    const size_t ro = ((size_t)unit * n_max + r) * BPC_D;
+    float4 x;
+    if (it == 0) {
+      const KV* kr = k_cache + ro + 4 * lane;
+      x = make_float4(to_float(kr[0]), to_float(kr[1]), to_float(kr[2]), to_float(kr[3]));
+    } else {
+      x = reinterpret_cast<const float4*>(R + ro)[lane];
+      const float u = usign[(size_t)unit * n_max + r] ? 1.f : -1.f;
+      x.x = fmaf(-u, vp.x, x.x); x.y = fmaf(-u, vp.y, x.y); x.z = fmaf(-u, vp.z, x.z); x.w = fmaf(-u, vp.w, x.w);
+    }
+    reinterpret_cast<float4*>(R + ro)[lane] = x;
+    float t = x.x * vs.x;
+    t = fmaf(x.y, vs.y, t); t = fmaf(x.z, vs.z, t); t = fmaf(x.w, vs.w, t);
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    const bool pos = t >= 0.f;
+    if (lane == 0) {
+      usign[(size_t)unit * n_max + r] = pos ? 1 : 0;
+      // diagnostic copy of the fitted codes H (Algorithm 1's by-product), packed like the cache codes
+      uint32_t* hw = hfit + ((size_t)unit * n_max + r) * (b / 32) + (it >> 5);
+      const uint32_t prev = (it & 31) ? *hw : 0u;
+      *hw = prev | ((pos ? 1u : 0u) << (it & 31));
+    }
+    if (pos) { acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w; }
+    else     { acc.x -= x.x; acc.y -= x.y; acc.z -= x.z; acc.w -= x.w; }
+  }
+  red[warp][4 * lane] = acc.x; red[warp][4 * lane + 1] = acc.y; red[warp][4 * lane + 2] = acc.z; red[warp][4 * lane + 3] = acc.w;
+  __syncthreads();
+  if (tid < BPC_D) {
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < kFitThreads / 32; ++w) s += red[w][tid];
+    partials[((size_t)unit * blocks_per_unit + blockIdx.x) * BPC_D + tid] = s;
+  }
+}
+
+__global__ void fit_reduce_kernel(const float* __restrict__ partials, float* __restrict__ P,
+                                  const int32_t* __restrict__ unit_lens, int n_max, int b, int it, int blocks_per_unit) {
+  const int unit = blockIdx.x, c = threadIdx.x;
+  const int n = min(unit_lens[unit], n_max);
+  const int nblk = (n + kFitRowsPerBlock - 1) / kFitRowsPerBlock;
+  double s = 0.0;
+  for (int k = 0; k < nblk; ++k) s += (double)partials[((size_t)unit * blocks_per_unit + k) * BPC_D + c];
+  P[((size_t)unit * b + it) * BPC_D + c] = n > 0 ? (float)(s / (double)n) : 0.f;
+}
+
+}  // namespace
+
+// =========================================================================== host launchers
+cudaError_t bpc_launch_finalize_projection(bpc_ctx* ctx, cudaStream_t stream) {
+  const bpc_config& c = ctx->cfg;
+  const size_t n = (size_t)c.hash_sets * c.code_bits * BPC_D;
+  const int th = 256;
+  const unsigned blocks = (unsigned)((n + th - 1) / th);
+  if (c.kv_dtype == BPC_BF16)
+    round_projection_kernel<__nv_bfloat16><<<blocks, th, 0, stream>>>(ctx->P, (__nv_bfloat16*)ctx->P_h, ctx->P_hf, n);
+  else
+    round_projection_kernel<float><<<blocks, th, 0, stream>>>(ctx->P, (float*)ctx->P_h, ctx->P_hf, n);
+  gram_kernel<<<dim3(c.code_bits, c.hash_sets), 128, 0, stream>>>(ctx->P_hf, ctx->gram, c.code_bits);
+  ctx->launches += 2;
+  return cudaGetLastError();
+}
+
+cudaError_t bpc_launch_encode_simple(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStream_t stream) {
+  const bpc_config& c = ctx->cfg;
+  const int b = c.code_bits;
+  const size_t smem = (size_t)128 * BPC_D * 4 + (size_t)b * kEncThreads * 4;
+  const dim3 grid((c.n_max + kEncThreads - 1) / kEncThreads, ctx->units);
+  const int shared_sets = c.hash_sets != ctx->units;
+  cudaError_t e;
+  if (c.kv_dtype == BPC_BF16) {
+    e = cudaFuncSetAttribute(encode_simple_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    encode_simple_kernel<__nv_bfloat16><<<grid, kEncThreads, smem, stream>>>(
+        (const __nv_bfloat16*)k_cache, ctx->P_hf, ctx->gram, ctx->unit_lens, codes, c.n_kv_heads, c.n_max, b, shared_sets,
+        c.residual_correction);
+  } else {
+    e = cudaFuncSetAttribute(encode_simple_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    encode_simple_kernel<float><<<grid, kEncThreads, smem, stream>>>(
+        (const float*)k_cache, ctx->P_hf, ctx->gram, ctx->unit_lens, codes, c.n_kv_heads, c.n_max, b, shared_sets,
+        c.residual_correction);
+  }
+  ctx->launches += 1;
+  return cudaGetLastError();
+}
+
+cudaError_t bpc_launch_append(bpc_ctx* ctx, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                              uint64_t* codes, cudaStream_t stream) {
+  const bpc_config& c = ctx->cfg;
+  const int b = c.code_bits;
+  const size_t smem = b <= 128 ? (size_t)b * b * 4 : 16;
+  const int shared_sets = c.hash_sets != ctx->units;
+  cudaError_t e;
+  if (c.kv_dtype == BPC_BF16) {
+    e = cudaFuncSetAttribute(append_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    append_kernel<__nv_bfloat16><<<ctx->units, kAppThreads, smem, stream>>>(
+        (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, codes,
+        (const __nv_bfloat16*)ctx->P_h, ctx->gram, ctx->unit_lens, ctx->dev_err, c.n_kv_heads, c.n_max, b, shared_sets,
+        c.residual_correction);
+  } else {
+    e = cudaFuncSetAttribute(append_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    append_kernel<float><<<ctx->units, kAppThreads, smem, stream>>>(
+        (const float*)k_new, (const float*)v_new, (float*)k_cache, (float*)v_cache, codes, (const float*)ctx->P_h,
+        ctx->gram, ctx->unit_lens, ctx->dev_err, c.n_kv_heads, c.n_max, b, shared_sets, c.residual_correction);
+  }
+  ctx->launches += 1;
+  return cudaGetLastError();
+}
+
+static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+size_t bpc_fit_workspace_bytes_impl(const bpc_config* c) {
+  const size_t units = (size_t)c->batch * c->n_kv_heads;
+  const size_t bpu = ((size_t)c->n_max + kFitRowsPerBlock - 1) / kFitRowsPerBlock;
+  return align256(units * c->n_max * BPC_D * 4) + align256(units * c->n_max) + align256(units * bpu * BPC_D * 4) +
+         align256(units * c->n_max * (c->code_bits / 8));
+}
+
+size_t bpc_fit_codes_offset_impl(const bpc_config* c) {
+  const size_t units = (size_t)c->batch * c->n_kv_heads;
+  const size_t bpu = ((size_t)c->n_max + kFitRowsPerBlock - 1) / kFitRowsPerBlock;
+  return align256(units * c->n_max * BPC_D * 4) + align256(units * c->n_max) + align256(units * bpu * BPC_D * 4);
+}
+
+cudaError_t bpc_launch_fit(bpc_ctx* ctx, const void* k_cache, const float* v_star, void* workspace,
+                           cudaStream_t stream, int* launches) {
+  const bpc_config& c = ctx->cfg;
+  const size_t units = (size_t)ctx->units;
+  const int bpu = (c.n_max + kFitRowsPerBlock - 1) / kFitRowsPerBlock;
+  unsigned char* ws = (unsigned char*)workspace;
+  float* R = (float*)ws;
+  uint8_t* usign = ws + align256(units * c.n_max * BPC_D * 4);
+  float* partials = (float*)(usign + align256(units * c.n_max));
+  uint32_t* hfit = (uint32_t*)(ws + bpc_fit_codes_offset_impl(&c));
+  const dim3 grid(bpu, ctx->units);
+  for (int it = 0; it < c.code_bits; ++it) {
+    if (c.kv_dtype == BPC_BF16)
+      fit_pass_kernel<__nv_bfloat16><<<grid, kFitThreads, 0, stream>>>((const __nv_bfloat16*)k_cache, R, usign, hfit, v_star, ctx->P,
+                                                                        partials, ctx->unit_lens, c.n_max, c.code_bits, it, bpu);
+    else
+      fit_pass_kernel<float><<<grid, kFitThreads, 0, stream>>>((const float*)k_cache, R, usign, hfit, v_star, ctx->P, partials,
+                                                               ctx->unit_lens, c.n_max, c.code_bits, it, bpu);
+    fit_reduce_kernel<<<ctx->units, BPC_D, 0, stream>>>(partials, ctx->P, ctx->unit_lens, c.n_max, c.code_bits, it, bpu);
+    *launches += 2;
+  }
+  return cudaGetLastError();
+}

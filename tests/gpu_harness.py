@@ -1,0 +1,222 @@
+"""Stage-wise comparison of the CUDA library (through the C-ABI binding) with the CPU checker.
+
+Every stage is checked on the same seeded inputs, and each downstream stage is additionally fed the
+library's own upstream output (its projection, its codes, its index set), so that a legitimately ambiguous
+sign upstream cannot masquerade as a downstream bug.
+
+Tolerances
+  fit      : a fitted sign may differ only where |t| < 1e-5 * ||r|| * ||v*|| (fp32 row dot product);
+             with the library's signs adopted, P must agree to 2e-5 relative per row
+  encode   : bits bit-exact except decisions with |t| < 1e-6 * (||k|| ||P_i|| + sum_{j<i} |G_ji|), counted
+  query    : collapsed weights exact except bits with |p_j| < 1e-6 * ||q|| * ||P_j||, counted
+  scores   : bit-exact given the library's codes and query weights
+  top-k    : index set bit-exact (ascending, lowest-index ties)
+  output   : max-abs 2e-3 (bf16 caches) / 1e-5 (fp32 caches) against the fp64 checker
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import bpc_oracle as O
+from paper_2608_04405_b200 import binding as B
+from paper_2608_04405_b200.inputs import Workload, WorkloadSpec
+
+OUT_TOL = {"bf16": 2e-3, "f32": 1e-5}
+
+
+def _np64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to("cpu", torch.float64).numpy()
+
+
+def codes_to_bits(codes_unit: torch.Tensor, b: int) -> np.ndarray:
+    """codes [n, b/64] int64 (device or host) -> bits [n, b] uint8."""
+    w = codes_unit.detach().cpu().numpy().view(np.uint64)
+    return O.unpack_bits(w, b)
+
+
+class Session:
+    """A workload on the GPU with its library context, fitted and encoded."""
+
+    def __init__(self, spec: WorkloadSpec, gen_device: str = "cpu", salt: int = 0, cluster_size: int = 0,
+                 extra_rows=None):
+        self.spec = spec
+        self.w = Workload(spec, device=gen_device, extra_rows=extra_rows, salt=salt)
+        dev = "cuda"
+        self.k_cache = self.w.k_cache.to(dev)
+        self.v_cache = self.w.v_cache.to(dev)
+        self.v_star = self.w.v_star.to(dev)
+        self.cfg = B.make_config(spec.batch, spec.n_q_heads, spec.n_kv_heads, self.w.n_max, spec.code_bits,
+                                 spec.torch_dtype)
+        self.ctx = B.Context(self.cfg)
+        if cluster_size:
+            self.ctx.set_cluster_size(cluster_size)
+        self.lens = list(self.w.seq_lens)
+        self.ctx.set_seq_lens(self.lens)
+        self.codes = self.ctx.alloc_codes()
+        self.units = spec.batch * spec.n_kv_heads
+        self.fit_ws = None
+
+    def fit(self):
+        self.fit_ws = torch.zeros(self.ctx.fit_workspace_bytes(), dtype=torch.uint8, device="cuda")
+        self.ctx.fit(self.k_cache, self.v_star, self.fit_ws)
+        torch.cuda.synchronize()
+        self.P, self.Ph, self.gram = self.ctx.get_projection()
+        torch.cuda.synchronize()
+
+    def encode(self):
+        self.ctx.encode_keys(self.k_cache, self.codes)
+        torch.cuda.synchronize()
+
+    def unit_views(self, u: int):
+        s = self.spec
+        bi, h = divmod(u, s.n_kv_heads)
+        return bi, h, self.lens[bi]
+
+    def hfit_bits(self, u: int) -> np.ndarray:
+        s = self.spec
+        off = self.ctx.fit_codes_offset()
+        words = s.code_bits // 64
+        n_max = self.w.n_max
+        raw = self.fit_ws[off: off + self.units * n_max * words * 8].view(torch.int64).view(self.units, n_max, words)
+        _, _, n = self.unit_views(u)
+        return codes_to_bits(raw[u, :n], s.code_bits)
+
+
+def check_fit(sess: Session, units, report: dict):
+    s = sess.spec
+    for u in units:
+        bi, h, n = sess.unit_views(u)
+        K = _np64(sess.k_cache[bi, h, :n])
+        vs = _np64(sess.v_star[u])
+        gpuH = sess.hfit_bits(u)
+        gpuP = _np64(sess.P[u])
+        # replay Algorithm 1 in fp64, adopting the library's signs where the decision is within fp32 noise
+        R = K.copy()
+        amb = hard = 0
+        Pref = np.zeros_like(gpuP)
+        for i in range(s.code_bits):
+            t = R @ vs[i]
+            mine = t >= 0
+            theirs = gpuH[:, i].astype(bool)
+            diff = mine != theirs
+            tau = 1e-5 * np.linalg.norm(R, axis=1) * np.linalg.norm(vs[i])
+            hard += int(np.count_nonzero(diff & (np.abs(t) >= tau)))
+            amb += int(np.count_nonzero(diff & (np.abs(t) < tau)))
+            uu = np.where(theirs, 1.0, -1.0)
+            v = (uu @ R) / n
+            R = R - np.outer(uu, v)
+            Pref[i] = v
+        assert hard == 0, "fit: %d sign decisions differ outside the ambiguity band (unit %d)" % (hard, u)
+        rel = np.linalg.norm(gpuP - Pref, axis=1) / np.maximum(np.linalg.norm(Pref, axis=1), 1e-30)
+        assert rel.max() <= 2e-5, "fit: projection rows differ, max relative error %g (unit %d)" % (rel.max(), u)
+        # P_h is P rounded to the cache precision; Gram = P_h P_h^T
+        Ph = O.to_hash_precision(_np64(sess.P[u]), s.dtype)
+        assert np.array_equal(Ph, _np64(sess.Ph[u])), "hash-precision rounding of P differs"
+        Gm = Ph @ Ph.T
+        gerr = np.abs(_np64(sess.gram[u]) - Gm).max() / max(np.abs(Gm).max(), 1e-30)
+        assert gerr <= 1e-6, "Gram matrix differs (%g)" % gerr
+        report["fit_ambiguous_signs"] = report.get("fit_ambiguous_signs", 0) + amb
+        report["fit_max_rel_err"] = max(report.get("fit_max_rel_err", 0.0), float(rel.max()))
+        # pure-checker fit from scratch agrees wherever no sign was ambiguous
+        if amb == 0:
+            P0, _, _ = O.fit(K, vs)
+            rel0 = np.linalg.norm(gpuP - P0, axis=1) / np.maximum(np.linalg.norm(P0, axis=1), 1e-30)
+            assert rel0.max() <= 2e-5
+
+
+def check_encode(sess: Session, units, report: dict, max_keys: int = 0, key_slice=None):
+    s = sess.spec
+    for u in units:
+        bi, h, n = sess.unit_views(u)
+        lo, hi = (0, n) if key_slice is None else key_slice
+        if max_keys and hi - lo > max_keys:
+            hi = lo + max_keys
+        K = _np64(sess.k_cache[bi, h, lo:hi])
+        Ph = _np64(sess.Ph[u if sess.cfg.hash_sets == sess.units else h])
+        bits = codes_to_bits(sess.codes[bi, h, lo:hi], s.code_bits)
+        hard, amb = O.replay_encode_with_adoption(K, Ph, bits)
+        assert not hard.any(), "encode: %d bits differ outside the ambiguity band (unit %d)" % (int(hard.sum()), u)
+        report["encode_ambiguous_bits"] = report.get("encode_ambiguous_bits", 0) + int(amb.sum())
+        report["encode_bits_checked"] = report.get("encode_bits_checked", 0) + int(bits.size)
+        if not amb.any():
+            ref, _ = O.encode(K, Ph)
+            assert np.array_equal(ref, bits)
+
+
+def check_decode(sess: Session, q: torch.Tensor, units, report: dict, budget_ppm=None, budget_count=0):
+    """One decode step through the library, checked stage by stage for the given units."""
+    s = sess.spec
+    ppm = s.budget_ppm if budget_ppm is None else budget_ppm
+    n_max = sess.w.n_max
+    dbg_scores = torch.zeros(sess.units, n_max, dtype=torch.int32, device="cuda")
+    dbg_qw = torch.zeros(sess.units, s.code_bits, dtype=torch.int32, device="cuda")
+    sel = torch.full((sess.units, n_max), -1, dtype=torch.int32, device="cuda")
+    sess.ctx.debug_set_buffers(dbg_scores, dbg_qw)
+    out = sess.ctx.decode_attn(q, sess.k_cache, sess.v_cache, sess.codes, budget_ppm=ppm, budget_count=budget_count,
+                               sel_idx=sel)
+    torch.cuda.synchronize()
+    sess.ctx.debug_set_buffers(None, None)
+    assert sess.ctx.last_device_error() == 0
+    # a second call without the parity buffers and without a caller index list must give the same output
+    out2 = sess.ctx.decode_attn(q, sess.k_cache, sess.v_cache, sess.codes, budget_ppm=ppm, budget_count=budget_count)
+    torch.cuda.synchronize()
+    assert torch.equal(out, out2), "decode is not reproducible between calls"
+    G = s.group
+    tol = OUT_TOL[s.dtype]
+    for u in units:
+        bi, h, n = sess.unit_views(u)
+        Ph = _np64(sess.Ph[u if sess.cfg.hash_sets == sess.units else h])
+        qg = _np64(q[bi, h * G:(h + 1) * G])
+        K = _np64(sess.k_cache[bi, h, :n])
+        V = _np64(sess.v_cache[bi, h, :n])
+        bits = codes_to_bits(sess.codes[bi, h, :n], s.code_bits)
+        # query hash
+        p, sg, a = O.query_hash(qg, Ph, O.HAMMING)
+        A = O.collapsed_weights(sg, a)
+        A_gpu = dbg_qw[u].cpu().numpy().astype(np.int64)
+        if not np.array_equal(A, A_gpu):
+            band = np.stack([O.ambiguity_threshold_query(qg[g], Ph) for g in range(G)])
+            amb_bits = np.abs(p) < band
+            # flipping only ambiguous head signs must be able to explain the difference
+            slack = 2 * (amb_bits * a).sum(axis=0)
+            assert np.all(np.abs(A - A_gpu) <= slack), "query hash differs outside the ambiguity band (unit %d)" % u
+            report["query_ambiguous_bits"] = report.get("query_ambiguous_bits", 0) + int(np.count_nonzero(A != A_gpu))
+        # scores from the library's codes and the library's query weights
+        hpm = 2 * bits.astype(np.int64) - 1
+        sc = hpm @ A_gpu
+        sc_gpu = dbg_scores[u, :n].cpu().numpy().astype(np.int64)
+        assert np.array_equal(sc, sc_gpu), "hash scores differ (unit %d): %d of %d" % (u, int((sc != sc_gpu).sum()), n)
+        if np.array_equal(A, A_gpu):
+            assert np.array_equal(O.hash_scores(bits, sg, a), sc_gpu)
+        # selection
+        k = O.budget(n, ppm, budget_count)
+        idx = O.topk(sc_gpu, k)
+        idx_gpu = sel[u, :k].cpu().numpy().astype(np.int64)
+        assert np.array_equal(idx, idx_gpu), "selected index set differs (unit %d)" % u
+        if k < n_max:
+            assert int(sel[u, k]) == -1, "index list written past k"
+        # attention over the selected rows
+        ref = O.attend(qg, K, V, idx_gpu)
+        got = _np64(out[bi, h * G:(h + 1) * G])
+        err = float(np.abs(ref - got).max())
+        assert err <= tol, "attention output differs: max abs %g > %g (unit %d)" % (err, tol, u)
+        report["out_max_abs_err"] = max(report.get("out_max_abs_err", 0.0), err)
+        report["units_checked"] = report.get("units_checked", 0) + 1
+    return out, sel
+
+
+def check_append(sess: Session, k_new: torch.Tensor, v_new: torch.Tensor, units, report: dict):
+    """bpc_append through the library: rows land at position n, the new code follows Algorithm 2, n advances."""
+    s = sess.spec
+    before = list(sess.lens)
+    sess.ctx.append(k_new, v_new, sess.k_cache, sess.v_cache, sess.codes)
+    torch.cuda.synchronize()
+    assert sess.ctx.last_device_error() == 0
+    sess.lens = [n + 1 for n in before]
+    assert sess.ctx.get_seq_lens() == sess.lens
+    for u in units:
+        bi, h, n1 = sess.unit_views(u)
+        n = n1 - 1
+        assert torch.equal(sess.k_cache[bi, h, n], k_new[bi, h]) and torch.equal(sess.v_cache[bi, h, n], v_new[bi, h])
+        check_encode(sess, [u], report, key_slice=(n, n + 1))

@@ -1,0 +1,182 @@
+"""GPU parity tests: the CUDA library, called through the C-ABI binding, against the CPU checker."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_04405_b200.inputs import CONFIGS
+
+pytestmark = pytest.mark.gpu
+
+
+def _harness():
+    from tests import gpu_harness as H
+    return H
+
+
+def _decode_loop(sess, steps, units, report, H, check_every=1):
+    for step in range(steps):
+        k_new, v_new = sess.w.new_kv(sess.lens)
+        k_new, v_new = k_new.cuda(), v_new.cuda()
+        H.check_append(sess, k_new, v_new, units, report)
+        q, _ = sess.w.queries(sess.lens, k_cache=sess.k_cache.to(sess.w.device))
+        if step % check_every == 0:
+            H.check_decode(sess, q.cuda(), units, report)
+
+
+def test_cfg0_tiny_fp32_all_stages():
+    """Config 0 exactly: 1 head, n=4096, fp32, 64-bit codes, k=82, 16 decode steps with append."""
+    H = _harness()
+    spec = CONFIGS[0]
+    sess = H.Session(spec)
+    rep = {}
+    sess.fit(); H.check_fit(sess, [0], rep)
+    sess.encode(); H.check_encode(sess, [0], rep)
+    _decode_loop(sess, spec.steps, [0], rep, H)
+    assert rep["units_checked"] == spec.steps
+    print(rep)
+
+
+@pytest.mark.parametrize("cluster", [1, 2, 4, 8])
+def test_cluster_sizes_agree_with_checker(cluster):
+    """Ragged length (several tiles plus a tail) at every cluster size, GQA 4, bf16, 128-bit codes."""
+    H = _harness()
+    spec = CONFIGS[1].scaled(n_ctx=5000 + 37 * cluster, n_kv_heads=2, n_q_heads=8, steps=2)
+    sess = H.Session(spec, cluster_size=cluster)
+    rep = {}
+    sess.fit(); H.check_fit(sess, [0], rep)
+    sess.encode(); H.check_encode(sess, [0, 1], rep)
+    _decode_loop(sess, 2, [0, 1], rep, H)
+    print(rep)
+
+
+@pytest.mark.parametrize("bits,group,dtype", [(64, 1, "bf16"), (64, 4, "bf16"), (256, 4, "bf16"), (128, 7, "bf16"),
+                                              (128, 8, "bf16"), (128, 2, "bf16"), (128, 3, "f32"), (256, 1, "f32")])
+def test_code_lengths_and_group_sizes(bits, group, dtype):
+    H = _harness()
+    spec = CONFIGS[1].scaled(n_ctx=3000, n_kv_heads=2, n_q_heads=2 * group, code_bits=bits, dtype=dtype, steps=1,
+                             rope_base=None if dtype == "f32" else 500000.0)
+    sess = H.Session(spec)
+    rep = {}
+    sess.fit(); H.check_fit(sess, [1], rep)
+    sess.encode(); H.check_encode(sess, [0, 1], rep)
+    _decode_loop(sess, 1, [0, 1], rep, H)
+    print(rep)
+
+
+@pytest.mark.parametrize("ppm,count", [(1000000, 0), (10000, 0), (50000, 0), (0, 1), (0, 1024), (1, 0)])
+def test_budgets(ppm, count):
+    """budget = n (dense softmax attention), 1 %, 5 %, a single key, a fixed count, and the smallest fraction."""
+    H = _harness()
+    spec = CONFIGS[1].scaled(n_ctx=2500, n_kv_heads=2, n_q_heads=8, steps=1)
+    sess = H.Session(spec)
+    rep = {}
+    sess.fit(); sess.encode()
+    q, _ = sess.w.queries(sess.lens)
+    out, sel = H.check_decode(sess, q.cuda(), [0, 1], rep, budget_ppm=ppm, budget_count=count)
+    if ppm == 1000000:
+        # every key selected: the result is dense softmax attention
+        bi, h = 0, 1
+        n = sess.lens[0]
+        K = sess.k_cache[bi, h, :n].double().cpu(); V = sess.v_cache[bi, h, :n].double().cpu()
+        qq = q[bi, 4:8].double()
+        ref = torch.softmax(qq @ K.T / 128 ** 0.5, dim=-1) @ V
+        assert (ref - out[bi, 4:8].double().cpu()).abs().max() <= 2e-3
+
+
+def test_ragged_batch_and_empty_sequence():
+    """Different lengths per sequence, one of them empty (output rows are zero, nothing is selected)."""
+    H = _harness()
+    spec = CONFIGS[3].scaled(batch=3, n_ctx=4000, n_ctx_min=700, n_kv_heads=2, n_q_heads=8, steps=1)
+    sess = H.Session(spec)
+    sess.lens[1] = 0
+    sess.ctx.set_seq_lens(sess.lens)
+    rep = {}
+    sess.fit(); sess.encode()
+    lens_q = [max(1, n) for n in sess.lens]
+    q, _ = sess.w.queries(lens_q)
+    out, sel = H.check_decode(sess, q.cuda(), [0, 1, 4, 5], rep)
+    assert torch.count_nonzero(out[1]) == 0
+    H.check_encode(sess, [0, 5], rep)
+
+
+def test_shared_projection_per_kv_head():
+    """An externally supplied projection shared by all sequences (offline calibration flow)."""
+    H = _harness()
+    from paper_2608_04405_b200 import binding as B
+    spec = CONFIGS[1].scaled(batch=2, n_ctx=2000, n_kv_heads=2, n_q_heads=8, steps=1)
+    sess = H.Session(spec)
+    sess.fit()
+    P_unit = sess.P.clone()
+    cfg = B.make_config(spec.batch, spec.n_q_heads, spec.n_kv_heads, sess.w.n_max, spec.code_bits, spec.torch_dtype,
+                        shared_projection=True)
+    ctx2 = B.Context(cfg)
+    ctx2.set_seq_lens(sess.lens)
+    ctx2.set_projection(P_unit[:spec.n_kv_heads].contiguous())
+    sess.ctx, sess.cfg = ctx2, cfg
+    sess.P, sess.Ph, sess.gram = ctx2.get_projection()
+    sess.codes.zero_()
+    rep = {}
+    sess.encode(); H.check_encode(sess, [0, 1, 2, 3], rep)
+    q, _ = sess.w.queries(sess.lens)
+    H.check_decode(sess, q.cuda(), [0, 3], rep)
+
+
+def test_error_paths_do_not_launch():
+    from paper_2608_04405_b200 import binding as B
+    cfg = B.make_config(1, 4, 1, 1024, 128, torch.bfloat16)
+    ctx = B.Context(cfg)
+    k = torch.zeros(1, 1, 1024, 128, dtype=torch.bfloat16, device="cuda")
+    codes = ctx.alloc_codes()
+    q = torch.zeros(1, 4, 128, dtype=torch.bfloat16, device="cuda")
+    before = ctx.launch_count()
+    with pytest.raises(B.BpcError) as e:
+        ctx.decode_attn(q, k, k, codes)
+    assert e.value.status == 4                      # not fitted
+    with pytest.raises(B.BpcError) as e:
+        ctx.encode_keys(k, codes)
+    assert e.value.status == 4
+    with pytest.raises(B.BpcError) as e:
+        ctx.set_seq_lens([2000])
+    assert e.value.status == 3                      # beyond n_max
+    ctx.set_projection(torch.randn(1, 128, 128, device="cuda"))
+    ctx.set_seq_lens([1024])
+    kn = torch.zeros(1, 1, 128, dtype=torch.bfloat16, device="cuda")
+    n0 = ctx.launch_count()
+    with pytest.raises(B.BpcError) as e:
+        ctx.append(kn, kn, k, k, codes)
+    assert e.value.status == 3 and ctx.launch_count() == n0      # capacity: nothing launched
+    with pytest.raises(B.BpcError) as e:
+        ctx.decode_attn(q, k, k, codes, budget_ppm=0, budget_count=0)
+    assert e.value.status == 1
+    for bad in (dict(code_bits=96), dict(n_q_heads=9), dict(head_dim=64)):
+        kw = dict(batch=1, n_q_heads=4, n_kv_heads=1, n_max=1024, code_bits=128, dtype=torch.bfloat16)
+        hd = bad.pop("head_dim", 128)
+        kw.update(bad)
+        with pytest.raises(B.BpcError):
+            B.Context(B.make_config(head_dim=hd, **kw))
+    assert before == 0
+
+
+def test_cfg1_full_size_sampled_units():
+    """Config 1 at full size (32/8 heads, n=32768, 128-bit codes, k=656): every unit's selection and output."""
+    H = _harness()
+    spec = CONFIGS[1]
+    sess = H.Session(spec, gen_device="cuda")
+    rep = {}
+    sess.fit(); H.check_fit(sess, [3], rep)
+    sess.encode(); H.check_encode(sess, [0, 7], rep, max_keys=8192)
+    _decode_loop(sess, 2, list(range(8)), rep, H)
+    print(rep)
+
+
+def test_cfg2_full_size_sampled_units():
+    """Config 2 at full size (batch 4, n=131072) in the launch configuration the benchmark times; sampled units."""
+    H = _harness()
+    spec = CONFIGS[2]
+    sess = H.Session(spec, gen_device="cuda")
+    rep = {}
+    sess.fit()
+    sess.encode(); H.check_encode(sess, [5], rep, key_slice=(120000, 124096))
+    _decode_loop(sess, 1, [0, 13, 31], rep, H)
+    # planted-needle recall of the selection is the same number on both sides because the index sets are identical
+    print(rep)
