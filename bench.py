@@ -1,0 +1,417 @@
+#!/usr/bin/env python
+"""Benchmark of the BinaryPC decode step (append + decode_attn) on synthetic long-context workloads.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload 2]
+
+One step = one pass of the per-token hot path over the whole batch of one attention layer: bpc_append
+(cache write + Algorithm 2 on the new key) followed by bpc_decode_attn (query hash, code scan, top-k,
+gathered softmax attention).  The default workload is the 128K-context configuration (batch 4, 32/8
+heads, 128-bit codes, 2 % budget); `--layers` independent layer replicas are visited round-robin so
+that the codes and selected rows of a step are not left in L2 by the previous one.
+
+The timed region is ONE CUDA graph holding exactly K steps, bracketed by CUDA events on the launching
+stream.  With N > 1 (torchrun) every rank runs its own replica set (the path has no exchange step:
+replicas only) and the step time is the maximum over ranks.
+
+--impl reference times the CPU checker (oracle/) on the host cores on a bounded sample of the same
+workload; it is a deliberately plain program and only a reported baseline.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2608_04405_b200.inputs import CONFIGS, Workload, algorithmic_bytes_per_step
+
+METRIC = "sparse decode-attn tokens/s (one attention layer, append + decode_attn per step)"
+UNIT = "tokens/s"
+
+
+def _measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                        bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+        except Exception:
+            pass
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Polls NVML (read-only) for SM clock and clock-event reasons while a region runs."""
+
+    def __init__(self, index: int):
+        self.samples = []
+        self.reasons = set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thr = None
+        self._h = None
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = index
+            if vis:
+                try:
+                    phys = int(vis.split(",")[index])
+                except Exception:
+                    phys = index
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._h = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20,
+                 "hw_power_brake": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                break
+            time.sleep(0.0005)
+
+    def start(self):
+        if self._h is not None:
+            self._stop.clear()
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+
+    def stop(self):
+        if self._thr is not None:
+            self._stop.set()
+            self._thr.join()
+            self._thr = None
+        return len(self.samples)
+
+    def summary(self, n_timed: int):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0, "samples_in_timed_region": 0}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples), "samples_in_timed_region": n_timed}
+
+
+# ----------------------------------------------------------------------------- our arm
+class Layer:
+    """One attention layer replica: caches, codes, context, per-step inputs (all resident on the device)."""
+
+    def __init__(self, spec, salt, extra_rows, B, fit_ws):
+        w = Workload(spec, device="cuda", extra_rows=extra_rows, salt=salt)
+        self.w = w
+        self.cfg = B.make_config(spec.batch, spec.n_q_heads, spec.n_kv_heads, w.n_max, spec.code_bits, spec.torch_dtype)
+        self.ctx = B.Context(self.cfg)
+        self.lens0 = list(w.seq_lens)
+        self.ctx.set_seq_lens(self.lens0)
+        self.codes = self.ctx.alloc_codes()
+        self.k_cache, self.v_cache = w.k_cache, w.v_cache
+        self.fit_ms = self.encode_ms = None
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        if fit_ws[0] is None or fit_ws[0].numel() < self.ctx.fit_workspace_bytes():
+            fit_ws[0] = torch.empty(self.ctx.fit_workspace_bytes(), dtype=torch.uint8, device="cuda")
+        e0.record()
+        self.ctx.fit(self.k_cache, w.v_star, fit_ws[0])
+        e1.record()
+        self.ctx.encode_keys(self.k_cache, self.codes)
+        e2.record()
+        torch.cuda.synchronize()
+        self.fit_ms, self.encode_ms = e0.elapsed_time(e1), e1.elapsed_time(e2)
+        self.q, _ = w.queries(self.lens0)
+        self.k_new, self.v_new = w.new_kv(self.lens0)
+        self.out = torch.zeros(spec.batch, spec.n_q_heads, spec.head_dim, dtype=torch.float32, device="cuda")
+
+    def step(self):
+        self.ctx.append(self.k_new, self.v_new, self.k_cache, self.v_cache, self.codes)
+        self.ctx.decode_attn(self.q, self.k_cache, self.v_cache, self.codes, budget_ppm=self.w.spec.budget_ppm, out=self.out)
+
+
+def _graph_of(fn):
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        fn()
+    return g
+
+
+def _time_graph(g, dist_barrier):
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dist_barrier()
+    torch.cuda.synchronize()
+    e0.record()
+    g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    dist_barrier()
+    return e0.elapsed_time(e1)
+
+
+def run_ours(args):
+    from paper_2608_04405_b200 import binding as B
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    use_dist = world > 1
+    if use_dist:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if use_dist:
+            dist.barrier()
+
+    def max_over_ranks(x: float) -> float:
+        if not use_dist:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    spec = CONFIGS[args.workload]
+    K, W, L = args.steps, args.warmup, args.layers
+    extra = ((K + W) // L + 2) * 2 + 64
+    fit_ws = [None]
+    layers = [Layer(spec, salt=100 * rank + i, extra_rows=extra, B=B, fit_ws=fit_ws) for i in range(L)]
+    fit_ws[0] = None
+    torch.cuda.empty_cache()
+    peaks = _measured_peaks()
+
+    def set_lens(offset):
+        for ly in layers:
+            ly.ctx.set_seq_lens([n + offset for n in ly.lens0])
+
+    # --- warm-up: W eager steps
+    for s in range(W):
+        layers[s % L].step()
+    torch.cuda.synchronize()
+    per_layer_w = [(W + L - 1 - i) // L for i in range(L)]   # steps each layer has taken so far
+
+    def reset_after_warmup():
+        for ly, c in zip(layers, per_layer_w):
+            ly.ctx.set_seq_lens([n + c for n in ly.lens0])
+
+    # --- the timed region: ONE graph with exactly K steps
+    launches0 = sum(ly.ctx.launch_count() for ly in layers)
+    g_steps = _graph_of(lambda: [layers[(W + s) % L].step() for s in range(K)])
+    launches_per_region = sum(ly.ctx.launch_count() for ly in layers) - launches0
+    reset_after_warmup()
+    g_steps.replay()                      # first replay uploads the graph; not timed
+    torch.cuda.synchronize()
+    reset_after_warmup()
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms_total = _time_graph(g_steps, barrier)
+    n_timed_samples = sampler.stop()
+    ms_total = max_over_ranks(ms_total)
+    ms_step = ms_total / K
+
+    # --- the dominant kernel alone: K decode launches (no append), same round-robin, one graph
+    reset_after_warmup()
+    g_dec = _graph_of(lambda: [layers[(W + s) % L].ctx.decode_attn(
+        layers[(W + s) % L].q, layers[(W + s) % L].k_cache, layers[(W + s) % L].v_cache, layers[(W + s) % L].codes,
+        budget_ppm=spec.budget_ppm, out=layers[(W + s) % L].out) for s in range(K)])
+    g_dec.replay()
+    torch.cuda.synchronize()
+    ms_dec = _time_graph(g_dec, barrier) / K
+    g_app = _graph_of(lambda: [layers[(W + s) % L].ctx.append(
+        layers[(W + s) % L].k_new, layers[(W + s) % L].v_new, layers[(W + s) % L].k_cache, layers[(W + s) % L].v_cache,
+        layers[(W + s) % L].codes) for s in range(K)])
+    reset_after_warmup()
+    g_app.replay()
+    torch.cuda.synchronize()
+    reset_after_warmup()
+    ms_app = _time_graph(g_app, barrier) / K
+    # clocks under the same load, long enough for NVML to see it
+    reset_after_warmup()
+    sampler.start()
+    t_end = time.time() + 0.6
+    while time.time() < t_end:
+        g_dec.replay()
+        torch.cuda.synchronize()
+    sampler.stop()
+    clocks = sampler.summary(n_timed_samples)
+
+    # --- end to end through the public API with host buffers (pinned), result read back every step
+    reset_after_warmup()
+    hq = [ly.q.cpu().pin_memory() for ly in layers]
+    hk = [ly.k_new.cpu().pin_memory() for ly in layers]
+    hv = [ly.v_new.cpu().pin_memory() for ly in layers]
+    hout = torch.zeros_like(layers[0].out, device="cpu").pin_memory()
+    h2d = hq[0].numel() * hq[0].element_size() + 2 * hk[0].numel() * hk[0].element_size()
+    d2h = hout.numel() * 4
+
+    def e2e_step(s):
+        ly = layers[s % L]
+        ly.q.copy_(hq[s % L], non_blocking=True)
+        ly.k_new.copy_(hk[s % L], non_blocking=True)
+        ly.v_new.copy_(hv[s % L], non_blocking=True)
+        ly.step()
+        hout.copy_(ly.out, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    for s in range(min(W, 8)):
+        e2e_step(s)
+    reset_after_warmup()
+    barrier()
+    torch.cuda.synchronize()
+    ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ee0.record()
+    for s in range(K):
+        e2e_step(W + s)
+    ee1.record()
+    torch.cuda.synchronize()
+    barrier()
+    ms_e2e = max_over_ranks(ee0.elapsed_time(ee1)) / K
+
+    err = sum(ly.ctx.last_device_error() for ly in layers)
+    lens_now = [n + per_layer_w[0] for n in layers[0].lens0]
+    alg_bytes = algorithmic_bytes_per_step(spec, lens_now)
+    achieved = alg_bytes / (ms_dec * 1e-3) / 1e9
+    n_keys = sum(spec.n_kv_heads * n for n in layers[0].lens0)
+    enc_ms = statistics.median(ly.encode_ms for ly in layers)
+    fit_ms = statistics.median(ly.fit_ms for ly in layers)
+    enc_flops = 2.0 * n_keys * spec.head_dim * spec.code_bits
+    result = {
+        "metric": METRIC, "value": world * spec.batch / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": K, "warmup": W, "ms_per_step": ms_step, "us_per_step": ms_step * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": spec.name, "batch": spec.batch, "n_q_heads": spec.n_q_heads, "n_kv_heads": spec.n_kv_heads,
+                   "head_dim": spec.head_dim, "context": spec.n_ctx, "code_bits": spec.code_bits,
+                   "budget_ppm": spec.budget_ppm, "layer_replicas": L,
+                   "l2": "inputs larger than L2: %d layer replicas visited round-robin" % L,
+                   "cluster_size": layers[0].ctx.get_cluster_size(), "parallelism": "replicas only"},
+        "clocks": clocks,
+        "e2e": {"value": world * spec.batch / (ms_e2e * 1e-3), "unit": UNIT, "us_per_step": ms_e2e * 1e3,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches_per_region,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"], "of": peaks["source"], "traffic": None,
+                     "kernel": "bpc_decode_kernel", "us_per_launch": ms_dec * 1e3, "algorithmic_bytes": alg_bytes,
+                     "frac_of_nominal_8TBs": achieved / 8000.0,
+                     "whole_step_gbs": alg_bytes / (ms_step * 1e-3) / 1e9},
+        "breakdown_us": {"decode_attn": ms_dec * 1e3, "append": ms_app * 1e3},
+        "prefill": {"fit_ms": fit_ms, "encode_ms": enc_ms, "encode_keys_per_s": n_keys / (enc_ms * 1e-3),
+                    "encode_gemm_tflops": enc_flops / (enc_ms * 1e-3) / 1e12,
+                    "encode_frac_of_bf16_peak": enc_flops / (enc_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]},
+        "device_error_word": err,
+        "paper_context": "paper reports up to 3.56x end-to-end decode speed-up over FlashAttention-2 on 8 data-center GPUs "
+                         "(HF stack, 64-bit codes); context only, not comparable",
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        result["cpu_baseline"] = cpu_baseline(spec, budget_s=args.cpu_budget)
+    if rank == 0:
+        print(json.dumps(result))
+    if use_dist:
+        dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------- CPU checker arm
+def _oracle_unit_setup(spec, seed_salt=0):
+    """One unit of the workload prepared for the checker: keys, values, projection, codes (prefill, untimed)."""
+    from oracle import bpc_oracle as O
+    one = spec.scaled(batch=1, n_kv_heads=1, n_q_heads=spec.group)
+    w = Workload(one, device="cpu", extra_rows=64, salt=seed_salt)
+    n = w.seq_lens[0]
+    K = w.k_cache[0, 0, :n].double().numpy()
+    V = w.v_cache[0, 0, :n].double().numpy()
+    sub = K[:: max(1, n // 4096)][:4096]              # projection fitted on a strided sample of the keys
+    P, _, _ = O.fit(sub, w.v_star[0].double().numpy())
+    Ph = O.to_hash_precision(P, spec.dtype)
+    bits, _ = O.encode(K, Ph)
+    q, _ = w.queries(w.seq_lens)
+    return O, K, V, Ph, bits, q[0].double().numpy()
+
+
+def cpu_baseline(spec, budget_s=15.0):
+    O, K, V, Ph, bits, q = _oracle_unit_setup(spec)
+    units_per_step = spec.batch * spec.n_kv_heads
+    t0, c0 = time.time(), time.process_time()
+    done = 0
+    while done < 2 or (time.time() - t0 < budget_s and done < 64):
+        O.decode_unit(q, K, V, bits, Ph, spec.budget_ppm)
+        done += 1
+    wall, cpu = time.time() - t0, time.process_time() - c0
+    step_s = wall / done * units_per_step
+    return {"value": spec.batch / step_s, "unit": UNIT, "cores": max(1, int(round(cpu / max(wall, 1e-9)))),
+            "host_cores": os.cpu_count(), "kind": "oracle",
+            "sample": "%d single-unit decode steps (query hash, %d-key score, top-k, attention) of %s timed; "
+                      "one step = %d such units, scaled" % (done, K.shape[0], spec.name, units_per_step),
+            "us_per_step_scaled": step_s * 1e6}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    spec = CONFIGS[args.workload]
+    O, K, V, Ph, bits, q = _oracle_unit_setup(spec)
+    units_per_step = spec.batch * spec.n_kv_heads
+    for _ in range(min(args.warmup, 3)):
+        O.decode_unit(q, K, V, bits, Ph, spec.budget_ppm)
+    t0, c0 = time.time(), time.process_time()
+    for _ in range(args.steps):
+        O.decode_unit(q, K, V, bits, Ph, spec.budget_ppm)
+    wall, cpu = time.time() - t0, time.process_time() - c0
+    step_s = wall / args.steps * units_per_step
+    value = spec.batch / step_s
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    sample = ("each step times ONE (sequence, KV head) unit of %s (%d keys) on the host and is scaled by the %d units "
+              "of a full step" % (spec.name, K.shape[0], units_per_step))
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": spec.name, "batch": spec.batch, "n_q_heads": spec.n_q_heads, "n_kv_heads": spec.n_kv_heads,
+                   "head_dim": spec.head_dim, "context": spec.n_ctx, "code_bits": spec.code_bits,
+                   "budget_ppm": spec.budget_ppm},
+        "cpu_baseline": {"value": value, "unit": UNIT, "kind": "oracle", "host_cores": os.cpu_count(),
+                         "cores": max(1, int(round(cpu / max(wall, 1e-9)))), "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=128)
+    ap.add_argument("--warmup", type=int, default=32)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=2)
+    ap.add_argument("--layers", type=int, default=4, help="independent layer replicas visited round-robin (cold L2)")
+    ap.add_argument("--cpu-budget", type=float, default=15.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
