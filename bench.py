@@ -121,10 +121,16 @@ class ClockSampler:
 class Layer:
     """One attention layer replica: caches, codes, context, per-step inputs (all resident on the device)."""
 
-    def __init__(self, spec, salt, extra_rows, B, fit_ws):
+    def __init__(self, spec, salt, extra_rows, B, fit_ws, interleaved):
         w = Workload(spec, device="cuda", extra_rows=extra_rows, salt=salt)
         self.w = w
-        self.cfg = B.make_config(spec.batch, spec.n_q_heads, spec.n_kv_heads, w.n_max, spec.code_bits, spec.torch_dtype)
+        if interleaved:     # one buffer, K and V rows of a token adjacent (row stride 2*head_dim)
+            self.kv_buf, kc, vc = B.interleaved_kv(spec.batch, spec.n_kv_heads, w.n_max, spec.head_dim, spec.torch_dtype)
+            kc.copy_(w.k_cache)
+            vc.copy_(w.v_cache)
+            w.k_cache, w.v_cache = kc, vc
+        self.cfg = B.make_config(spec.batch, spec.n_q_heads, spec.n_kv_heads, w.n_max, spec.code_bits, spec.torch_dtype,
+                                 kv_row_stride=2 * spec.head_dim if interleaved else 0)
         self.ctx = B.Context(self.cfg)
         self.lens0 = list(w.seq_lens)
         self.ctx.set_seq_lens(self.lens0)
@@ -195,7 +201,8 @@ def run_ours(args):
     K, W, L = args.steps, args.warmup, args.layers
     extra = ((K + W) // L + 2) * 2 + 64
     fit_ws = [None]
-    layers = [Layer(spec, salt=100 * rank + i, extra_rows=extra, B=B, fit_ws=fit_ws) for i in range(L)]
+    layers = [Layer(spec, salt=100 * rank + i, extra_rows=extra, B=B, fit_ws=fit_ws, interleaved=not args.separate_kv)
+              for i in range(L)]
     fit_ws[0] = None
     torch.cuda.empty_cache()
     peaks = _measured_peaks()
@@ -208,6 +215,14 @@ def run_ours(args):
     for s in range(W):
         layers[s % L].step()
     torch.cuda.synchronize()
+    if args.profile:                      # plain eager steps for a profiler to capture; no graphs, no other legs
+        for s in range(K):
+            layers[(W + s) % L].step()
+        torch.cuda.synchronize()
+        if rank == 0:
+            print(json.dumps({"profile_run": True, "workload": spec.name, "steps": K, "warmup": W, "layer_replicas": L,
+                              "cluster_size": layers[0].ctx.get_cluster_size()}))
+        return
     per_layer_w = [(W + L - 1 - i) // L for i in range(L)]   # steps each layer has taken so far
 
     def reset_after_warmup():
@@ -303,7 +318,8 @@ def run_ours(args):
                    "head_dim": spec.head_dim, "context": spec.n_ctx, "code_bits": spec.code_bits,
                    "budget_ppm": spec.budget_ppm, "layer_replicas": L,
                    "l2": "inputs larger than L2: %d layer replicas visited round-robin" % L,
-                   "cluster_size": layers[0].ctx.get_cluster_size(), "parallelism": "replicas only"},
+                   "cluster_size": layers[0].ctx.get_cluster_size(), "parallelism": "replicas only",
+                   "kv_layout": "separate k/v arrays" if args.separate_kv else "interleaved k|v rows (row stride 2*head_dim)"},
         "clocks": clocks,
         "e2e": {"value": world * spec.batch / (ms_e2e * 1e-3), "unit": UNIT, "us_per_step": ms_e2e * 1e3,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
@@ -404,6 +420,8 @@ def main():
     ap.add_argument("--layers", type=int, default=4, help="independent layer replicas visited round-robin (cold L2)")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--separate-kv", action="store_true", help="separate K and V arrays instead of interleaved rows")
+    ap.add_argument("--profile", action="store_true", help="warm-up plus K eager steps only (for ncu captures)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

@@ -14,7 +14,11 @@
  *   - Every compute call is asynchronous on `stream` (a cudaStream_t passed as void*; NULL is the
  *     legacy default stream) and returns a bpc_status; nothing aborts, traps or prints.
  *   - Layouts (row-major, contiguous):
- *       k_cache, v_cache : [batch][n_kv_heads][n_max][head_dim]   kv_dtype, base 16-byte aligned
+ *       k_cache, v_cache : [batch][n_kv_heads][n_max] rows of head_dim kv_dtype values, base 16-byte
+ *                          aligned; consecutive rows are kv_row_stride elements apart (head_dim when the
+ *                          caches are separate arrays; 2*head_dim with v_cache = k_cache + head_dim for the
+ *                          interleaved layout, where a token's K and V rows are adjacent in memory and one
+ *                          gather touches 4*head_dim contiguous bytes instead of two separate rows)
  *       codes            : [batch][n_kv_heads][n_max][code_bits/64] uint64
  *                          bit j of a key (Algorithm 2 iteration j+1) is word j/64, bit j%64,
  *                          least significant first; 1 means the component is +1 (decision value >= 0)
@@ -65,6 +69,7 @@ typedef struct {
   float   sm_scale;             /* softmax scale; 0 selects 1/sqrt(head_dim) */
   int32_t hash_sets;            /* batch*n_kv_heads (one projection per unit) or n_kv_heads (shared per KV head) */
   int32_t residual_correction;  /* 1: Algorithm 2 (default). 0: plain sign(k P^T), for comparison only */
+  int32_t kv_row_stride;        /* elements between consecutive cache rows; 0 selects head_dim */
 } bpc_config;
 
 typedef struct bpc_ctx bpc_ctx;
@@ -131,6 +136,12 @@ bpc_status bpc_decode_attn(bpc_ctx* ctx, const void* q, const void* k_cache, con
  * score of every cached key (scores [units][n_max] int32) and the collapsed integer query weights
  * A = sum over the group's heads of sign*magnitude (qweights [units][code_bits] int32). */
 bpc_status bpc_debug_set_buffers(bpc_ctx* ctx, int32_t* scores, int32_t* qweights);
+
+/* Tracing aid.  When set (non-NULL), every thread block of the next bpc_decode_attn calls writes
+ * %globaltimer stamps (ns) at its phase boundaries into a row of 16 slots: 0 start, 1 query hash done,
+ * 2 scan done, 3 selection done, 4 index list visible, 5 attention done, 6 block merge done, 7 end,
+ * 8 histograms complete, 9 threshold known, 10 output offsets known.  stamps [units * cluster_size][16] uint64. */
+bpc_status bpc_debug_set_phase_timer(bpc_ctx* ctx, uint64_t* stamps);
 
 /* Launch geometry of the decode kernel: thread blocks per cluster (0 = choose automatically).
  * Returns BPC_ERR_UNSUPPORTED if n_max does not fit that many blocks. */

@@ -32,7 +32,7 @@ class bpc_config(ctypes.Structure):
     _fields_ = [("batch", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
                 ("head_dim", ctypes.c_int32), ("code_bits", ctypes.c_int32), ("n_max", ctypes.c_int32),
                 ("kv_dtype", ctypes.c_int32), ("score_mode", ctypes.c_int32), ("sm_scale", ctypes.c_float),
-                ("hash_sets", ctypes.c_int32), ("residual_correction", ctypes.c_int32)]
+                ("hash_sets", ctypes.c_int32), ("residual_correction", ctypes.c_int32), ("kv_row_stride", ctypes.c_int32)]
 
 
 def _load() -> ctypes.CDLL:
@@ -57,6 +57,7 @@ def _load() -> ctypes.CDLL:
         "bpc_append": (i32, [vp, vp, vp, vp, vp, vp, vp]),
         "bpc_decode_attn": (i32, [vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]),
         "bpc_debug_set_buffers": (i32, [vp, vp, vp]),
+        "bpc_debug_set_phase_timer": (i32, [vp, vp]),
         "bpc_set_cluster_size": (i32, [vp, i32]),
         "bpc_get_cluster_size": (i32, [vp]),
         "bpc_last_device_error": (i32, [vp, ctypes.POINTER(i32), vp]),
@@ -75,7 +76,8 @@ lib = _load()
 EXPORTS = ["bpc_create", "bpc_destroy", "bpc_codes_bytes", "bpc_fit_workspace_bytes", "bpc_fit_codes_offset",
            "bpc_max_context",
            "bpc_set_seq_lens", "bpc_get_seq_lens", "bpc_fit", "bpc_set_projection", "bpc_get_projection",
-           "bpc_encode_keys", "bpc_append", "bpc_decode_attn", "bpc_debug_set_buffers", "bpc_set_cluster_size",
+           "bpc_encode_keys", "bpc_append", "bpc_decode_attn", "bpc_debug_set_buffers", "bpc_debug_set_phase_timer",
+           "bpc_set_cluster_size",
            "bpc_get_cluster_size", "bpc_last_device_error", "bpc_last_cuda_error", "bpc_launch_count", "bpc_version"]
 
 
@@ -84,6 +86,18 @@ def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
         return None
     assert t.is_contiguous(), "tensor must be contiguous"
     return t.data_ptr()
+
+
+def _cache_ptr(t: torch.Tensor) -> int:
+    """K/V caches may be strided views of one interleaved buffer: rows must be dense, the row stride is in the config."""
+    assert t.stride(-1) == 1, "cache rows must be dense"
+    return t.data_ptr()
+
+
+def interleaved_kv(batch: int, n_kv_heads: int, n_max: int, head_dim: int, dtype: torch.dtype, device="cuda"):
+    """One buffer [batch][n_kv_heads][n_max][2][head_dim]; returns (buffer, k_view, v_view) for kv_row_stride = 2*head_dim."""
+    buf = torch.zeros(batch, n_kv_heads, n_max, 2, head_dim, dtype=dtype, device=device)
+    return buf, buf[:, :, :, 0, :], buf[:, :, :, 1, :]
 
 
 def _stream() -> int:
@@ -97,10 +111,10 @@ def _check(status: int, what: str) -> None:
 
 def make_config(batch: int, n_q_heads: int, n_kv_heads: int, n_max: int, code_bits: int, dtype: torch.dtype,
                 score_mode: int = BPC_SCORE_HAMMING, sm_scale: float = 0.0, shared_projection: bool = False,
-                residual_correction: bool = True, head_dim: int = 128) -> bpc_config:
+                residual_correction: bool = True, head_dim: int = 128, kv_row_stride: int = 0) -> bpc_config:
     return bpc_config(batch, n_q_heads, n_kv_heads, head_dim, code_bits, n_max,
                       BPC_BF16 if dtype == torch.bfloat16 else BPC_F32, score_mode, sm_scale,
-                      n_kv_heads if shared_projection else batch * n_kv_heads, 1 if residual_correction else 0)
+                      n_kv_heads if shared_projection else batch * n_kv_heads, 1 if residual_correction else 0, kv_row_stride)
 
 
 class Context:
@@ -163,7 +177,7 @@ class Context:
     def fit(self, k_cache: torch.Tensor, v_star: torch.Tensor, workspace: Optional[torch.Tensor] = None) -> None:
         if workspace is None:
             workspace = torch.empty(self.fit_workspace_bytes(), dtype=torch.uint8, device=k_cache.device)
-        _check(lib.bpc_fit(self._h, _ptr(k_cache), _ptr(v_star), _ptr(workspace), workspace.numel(), _stream()), "bpc_fit")
+        _check(lib.bpc_fit(self._h, _cache_ptr(k_cache), _ptr(v_star), _ptr(workspace), workspace.numel(), _stream()), "bpc_fit")
 
     def set_projection(self, P: torch.Tensor) -> None:
         assert P.dtype == torch.float32
@@ -178,10 +192,10 @@ class Context:
         return P, Ph, gram
 
     def encode_keys(self, k_cache: torch.Tensor, codes: torch.Tensor) -> None:
-        _check(lib.bpc_encode_keys(self._h, _ptr(k_cache), _ptr(codes), _stream()), "bpc_encode_keys")
+        _check(lib.bpc_encode_keys(self._h, _cache_ptr(k_cache), _ptr(codes), _stream()), "bpc_encode_keys")
 
     def append(self, k_new, v_new, k_cache, v_cache, codes) -> None:
-        _check(lib.bpc_append(self._h, _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), _ptr(codes), _stream()),
+        _check(lib.bpc_append(self._h, _ptr(k_new), _ptr(v_new), _cache_ptr(k_cache), _cache_ptr(v_cache), _ptr(codes), _stream()),
                "bpc_append")
 
     def decode_attn(self, q, k_cache, v_cache, codes, budget_ppm: int = 20000, budget_count: int = 0,
@@ -189,7 +203,7 @@ class Context:
         c = self.cfg
         if out is None:
             out = torch.empty(c.batch, c.n_q_heads, c.head_dim, dtype=torch.float32, device=q.device)
-        _check(lib.bpc_decode_attn(self._h, _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(codes), budget_ppm, budget_count,
+        _check(lib.bpc_decode_attn(self._h, _ptr(q), _cache_ptr(k_cache), _cache_ptr(v_cache), _ptr(codes), budget_ppm, budget_count,
                                    _ptr(out), _ptr(sel_idx), _stream()), "bpc_decode_attn")
         return out
 
@@ -197,6 +211,10 @@ class Context:
     def debug_set_buffers(self, scores: Optional[torch.Tensor], qweights: Optional[torch.Tensor]) -> None:
         self._dbg = (scores, qweights)   # keep alive
         _check(lib.bpc_debug_set_buffers(self._h, _ptr(scores), _ptr(qweights)), "bpc_debug_set_buffers")
+
+    def debug_set_phase_timer(self, stamps: Optional[torch.Tensor]) -> None:
+        self._stamps = stamps
+        _check(lib.bpc_debug_set_phase_timer(self._h, _ptr(stamps)), "bpc_debug_set_phase_timer")
 
     def last_device_error(self) -> int:
         v = ctypes.c_int32(0)

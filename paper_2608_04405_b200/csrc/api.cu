@@ -26,6 +26,7 @@ bpc_status check_cfg(const bpc_config* c) {
   if (c->hash_sets != units && c->hash_sets != c->n_kv_heads) return BPC_ERR_INVALID_ARG;
   if (c->residual_correction != 0 && c->residual_correction != 1) return BPC_ERR_INVALID_ARG;
   if (!(c->sm_scale >= 0.f)) return BPC_ERR_INVALID_ARG;
+  if (c->kv_row_stride != 0 && (c->kv_row_stride < c->head_dim || c->kv_row_stride % 8 != 0)) return BPC_ERR_INVALID_ARG;
   if (c->n_max % 2 != 0) return BPC_ERR_INVALID_ARG;   // keeps every unit's code rows 16-byte aligned at 64 bits
   return BPC_OK;
 }
@@ -36,15 +37,16 @@ bpc_status cuda_fail(bpc_ctx* ctx, cudaError_t e) {
   return BPC_ERR_CUDA;
 }
 
-cudaError_t decode_limits(const bpc_ctx* ctx, int cs, int* max_cluster, int* chunk_cap, size_t* smem) {
-  return ctx->cfg.kv_dtype == BPC_BF16 ? bpc_decode_limits_bf16(ctx, cs, max_cluster, chunk_cap, smem)
-                                       : bpc_decode_limits_f32(ctx, cs, max_cluster, chunk_cap, smem);
-}
-
 int hamming_bins(const bpc_ctx* ctx) {
   const int G = ctx->group;
   const int cs = (G % 2 == 0) ? 1 : 0;
   return ((G * ctx->cfg.code_bits) >> cs) + 1;
+}
+
+cudaError_t decode_limits(const bpc_ctx* ctx, int /*unused*/, int* max_cluster, int* chunk_cap, size_t* smem) {
+  const int nbins = hamming_bins(ctx);
+  return ctx->cfg.kv_dtype == BPC_BF16 ? bpc_decode_limits_bf16(ctx, nbins, max_cluster, chunk_cap, smem)
+                                       : bpc_decode_limits_f32(ctx, nbins, max_cluster, chunk_cap, smem);
 }
 
 int chunk_for(int n_max, int cs) { return (((n_max + cs - 1) / cs) + 63) & ~63; }
@@ -104,9 +106,10 @@ bpc_status bpc_create(const bpc_config* cfg, bpc_ctx** out) {
   if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
   memset(ctx, 0, sizeof(*ctx));
   ctx->cfg = *cfg;
-  if (ctx->cfg.sm_scale == 0.f) ctx->cfg.sm_scale = 0.08838834764831845f;   // 1/sqrt(128)
+  ctx->sm_scale_d = cfg->sm_scale == 0.f ? 0.08838834764831845 : (double)cfg->sm_scale;   // default 1/sqrt(128)
   ctx->units = cfg->batch * cfg->n_kv_heads;
   ctx->group = cfg->n_q_heads / cfg->n_kv_heads;
+  ctx->row_stride = cfg->kv_row_stride == 0 ? cfg->head_dim : cfg->kv_row_stride;
   cudaError_t e = cudaGetDevice(&ctx->device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device);
   const size_t b = cfg->code_bits, hs = cfg->hash_sets;
@@ -270,10 +273,11 @@ bpc_status bpc_decode_attn(bpc_ctx* ctx, const void* q, const void* k_cache, con
   p.q = q; p.k_cache = k_cache; p.v_cache = v_cache; p.codes = codes; p.P_h = ctx->P_h;
   p.unit_lens = ctx->unit_lens; p.out = out;
   p.sel = sel_idx != nullptr ? sel_idx : ctx->sel_scratch;
-  p.dbg_scores = ctx->dbg_scores; p.dbg_qweights = ctx->dbg_qweights; p.err = ctx->dev_err;
-  p.n_kv_heads = c.n_kv_heads; p.group = ctx->group; p.n_max = c.n_max;
+  p.dbg_scores = ctx->dbg_scores; p.dbg_qweights = ctx->dbg_qweights; p.dbg_times = ctx->dbg_times;
+  p.err = ctx->dev_err;
+  p.n_kv_heads = c.n_kv_heads; p.group = ctx->group; p.n_max = c.n_max; p.row_stride = ctx->row_stride;
   p.shared_sets = c.hash_sets != ctx->units;
-  p.budget_ppm = budget_ppm; p.budget_count = budget_count; p.sm_scale = c.sm_scale;
+  p.budget_ppm = budget_ppm; p.budget_count = budget_count; p.sm_scale_d = ctx->sm_scale_d;
   const int chunk = chunk_for(c.n_max, ctx->cluster_size);
   if (chunk > cap) return BPC_ERR_UNSUPPORTED;
   p.chunk_cap = chunk;                                    // shared memory is sized for the largest possible unit
@@ -289,6 +293,12 @@ bpc_status bpc_debug_set_buffers(bpc_ctx* ctx, int32_t* scores, int32_t* qweight
   if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
   ctx->dbg_scores = scores;
   ctx->dbg_qweights = qweights;
+  return BPC_OK;
+}
+
+bpc_status bpc_debug_set_phase_timer(bpc_ctx* ctx, uint64_t* stamps) {
+  if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
+  ctx->dbg_times = reinterpret_cast<unsigned long long*>(stamps);
   return BPC_OK;
 }
 

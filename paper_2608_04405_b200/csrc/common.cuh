@@ -19,6 +19,7 @@ struct bpc_ctx {
   int device;
   int units;                // batch * n_kv_heads
   int group;                // query heads per KV head
+  int row_stride;           // cache elements between consecutive rows
   int cluster_size;         // decode: thread blocks per cluster
   int max_cluster;          // largest cluster size the device schedules for the decode kernel
   int sm_count;
@@ -33,9 +34,11 @@ struct bpc_ctx {
   int32_t* dev_err;         // device error word
   int32_t* dbg_scores;      // caller buffers (may be null)
   int32_t* dbg_qweights;
+  unsigned long long* dbg_times;
   int32_t last_cuda_error;
   int64_t launches;
   int chunk_cap_limit;      // keys one decode block can hold with all opt-in shared memory
+  double sm_scale_d;        // softmax scale in double (exact 1/sqrt(head_dim) by default)
   size_t decode_smem_set;   // non-zero once the decode kernel's function attributes have been set
 };
 
@@ -50,14 +53,17 @@ struct DecodeParams {
   int32_t* sel;              // [units][n_max]
   int32_t* dbg_scores;
   int32_t* dbg_qweights;
+  unsigned long long* dbg_times;   // [blocks][8] phase time stamps (ns), or null
   int32_t* err;
   int n_kv_heads;
   int group;
   int n_max;
+  int row_stride;            // cache elements between consecutive rows
   int shared_sets;           // 1: projection shared per KV head, 0: one per unit
   int budget_ppm;
   int budget_count;
-  float sm_scale;
+  double sm_scale_d;         // softmax scale
+  int stages;                // gather ring depth (2 or 3)
   int chunk_cap;             // keys whose scores one thread block can hold
   int nbins;                 // histogram bins (largest score key + 1)
 };

@@ -8,15 +8,17 @@
 // of the paper's eight packed query words; the score of key h is <A, h>.
 //
 // Phases of a cluster of CS blocks working on one unit with n cached keys:
-//   0  every block hashes the group's queries (fp64 projection, identical in all blocks)
-//   1  block r scans keys [r*chunk, (r+1)*chunk): 128-bit code loads, LOP3+POPC score, 16-bit score
-//      key into shared memory, shared-memory histogram
+//   0  every block hashes the group's queries (identical arithmetic in all blocks)
+//   1  block r scans keys [r*chunk, (r+1)*chunk): 128-bit code loads, LOP3 (+ carry-save compression) and
+//      POPC score, 16-bit score key into shared memory, shared-memory histogram
 //   2  cluster barrier; histograms are summed through distributed shared memory; the threshold key T
 //      and the per-block output offsets follow; each block emits its selected indices in ascending
 //      order (score > T, then the lowest-index ties at T) into the unit's index list
 //   3  cluster barrier; block r runs online-softmax attention over rows [k*r/CS, k*(r+1)/CS) of the
-//      list, gathering K and V rows with 16-byte loads; partial (m, l, acc) are merged inside the
-//      block, then across the cluster through distributed shared memory
+//      list.  Rows are gathered into a shared-memory ring with 16-byte asynchronous copies; bf16 caches
+//      use warp-level tensor-core MMAs (q K^T, then P V with P split in two bf16 halves), fp32 caches use
+//      fp64 arithmetic on the CUDA cores.  Partial (m, l, acc) are merged inside the block, then across
+//      the cluster through distributed shared memory.
 // Scores and gathered rows never touch global memory.
 #pragma once
 #include <cooperative_groups.h>
@@ -28,7 +30,7 @@ namespace cg = cooperative_groups;
 constexpr int kSegKeys = 32;        // score keys per shared-memory segment
 constexpr int kSegSlots = 40;       // 16-bit slots per segment (80 B: conflict-free 16-byte reads)
 constexpr int kMaxBins = 2048;      // histogram bins (score keys are 0..nbins-1)
-constexpr int kIdxTile = 1024;      // selected indices staged per attention tile
+constexpr int kIdxTile = 1024;      // selected indices staged at a time
 constexpr int kMaxPlanes = 10;
 
 template <int GP, int MODE> struct PlaneCount {
@@ -46,28 +48,43 @@ struct SmallState {
   int T, cnt_gt, my_take, my_base, rsum, pad[3];
 };
 
+template <typename KV> struct IsBf16 { static constexpr bool value = false; };
+template <> struct IsBf16<__nv_bfloat16> { static constexpr bool value = true; };
+
+// Shared-memory plan of one block, computed identically on host and device.
 template <typename KV, int GP, int W32>
 struct DecodeSmem {
   typedef typename KvTraits<KV>::acc_t acc_t;
-  static constexpr int NT = (GP <= 4) ? 512 : 256;
+  static constexpr bool kMma = IsBf16<KV>::value;
+  static constexpr int NT = kMma ? 512 : (GP <= 2 ? 512 : 256);
   static constexpr int NW = NT / 32;
   static constexpr int B = W32 * 32;
-  // offsets in bytes
+  static constexpr int kRowBytes = BPC_D * (int)sizeof(KV);
+  // gather staging: bf16 tiles hold 8 rows per warp (K rows, then V rows, 16-byte chunks XOR-swizzled);
+  // fp32 tiles hold 32 rows, each K row followed by its V row
+  static constexpr int kTileRows = kMma ? 8 * NW : 32;
+  static constexpr int kStageBytes = kTileRows * 2 * kRowBytes;
   __host__ __device__ static constexpr size_t a16(size_t x) { return (x + 15) & ~(size_t)15; }
   __host__ __device__ static constexpr size_t part_bytes() { return (size_t)NW * GP * (BPC_D + 2) * sizeof(acc_t); }
-  __host__ __device__ static size_t scores_bytes(int chunk_cap) {
-    size_t s = (size_t)((chunk_cap + kSegKeys - 1) / kSegKeys) * kSegSlots * 2;
-    return a16(s > part_bytes() ? s : part_bytes());
+  __host__ __device__ static constexpr size_t hashpart_bytes() { return (size_t)NT * GP * 8; }
+
+  size_t off_hist, off_tot, off_qf, off_pd, off_idx, off_cta, off_small, off_union, total;
+  __host__ __device__ DecodeSmem(int chunk_cap, int nbins, int stages) {
+    const size_t nb = a16((size_t)nbins * 4);
+    off_hist = 0;
+    off_tot = off_hist + nb;
+    off_qf = off_tot + nb;                                           // float[GP][128]
+    off_pd = off_qf + (size_t)GP * BPC_D * 4;                        // double[GP][B]
+    off_idx = off_pd + (size_t)GP * B * 8;                           // int32[kIdxTile]
+    off_cta = off_idx + kIdxTile * 4;                                // acc_t[GP][130]
+    off_small = a16(off_cta + (size_t)GP * (BPC_D + 2) * sizeof(acc_t));
+    off_union = a16(off_small + sizeof(SmallState));
+    size_t u = (size_t)((chunk_cap + kSegKeys - 1) / kSegKeys) * kSegSlots * 2;   // score keys
+    if (u < part_bytes()) u = part_bytes();                                      // block-level merge
+    if (u < hashpart_bytes()) u = hashpart_bytes();                              // query-hash partial sums
+    if (u < (size_t)stages * kStageBytes) u = (size_t)stages * kStageBytes;      // gather ring
+    total = off_union + a16(u);
   }
-  static constexpr size_t off_hist = 0;                                    // uint32[kMaxBins]
-  static constexpr size_t off_tot = off_hist + kMaxBins * 4;               // uint32[kMaxBins]
-  static constexpr size_t off_qd = off_tot + kMaxBins * 4;                 // double[GP][128]
-  static constexpr size_t off_pd = off_qd + (size_t)GP * BPC_D * 8;        // double[GP][B]
-  static constexpr size_t off_idx = off_pd + (size_t)GP * B * 8;           // int32[kIdxTile]
-  static constexpr size_t off_cta = off_idx + kIdxTile * 4;                // acc_t[GP][130]
-  static constexpr size_t off_small = a16(off_cta + (size_t)GP * (BPC_D + 2) * sizeof(acc_t));
-  static constexpr size_t off_scores = a16(off_small + sizeof(SmallState));
-  __host__ __device__ static size_t total(int chunk_cap) { return off_scores + scores_bytes(chunk_cap); }
 };
 
 __device__ __forceinline__ int score_slot(int i) { return (i >> 5) * kSegSlots + (i & 31); }
@@ -100,20 +117,87 @@ template <typename T> __device__ __forceinline__ T fast_exp2(T x);
 template <> __device__ __forceinline__ float fast_exp2<float>(float x) { return exp2f(x); }
 template <> __device__ __forceinline__ double fast_exp2<double>(double x) { return exp2(x); }
 
-// K/V row fragment of 8 consecutive dims held by one lane
-template <typename KV> struct RowFrag;
-template <> struct RowFrag<__nv_bfloat16> {
-  uint4 w;
-  __device__ __forceinline__ void load(const __nv_bfloat16* row, int hl) { w = ld_stream_v4(row + 8 * hl); }
-  __device__ __forceinline__ void get(float* f) const {
-    f[0] = bf16_lo(w.x); f[1] = bf16_hi(w.x); f[2] = bf16_lo(w.y); f[3] = bf16_hi(w.y);
-    f[4] = bf16_lo(w.z); f[5] = bf16_hi(w.z); f[6] = bf16_lo(w.w); f[7] = bf16_hi(w.w);
+// 16-byte asynchronous global->shared copy (bypasses L1 and registers) and its group bookkeeping
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+  const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+// ---- warp-level tensor-core helpers (legacy mma.sync path; M = 16 is padded query heads)
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void* smem_row) {
+  const unsigned a = (unsigned)__cvta_generic_to_shared(smem_row);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* smem_row) {
+  const unsigned a = (unsigned)__cvta_generic_to_shared(smem_row);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+// D(16x8,f32) += A(16x16,bf16,row) * B(16x8,bf16,col); rows 8..15 of A are zero here (a1 = a3 = 0)
+__device__ __forceinline__ void mma_qk(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+  const uint32_t z = 0u;
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a0), "r"(z), "r"(a2), "r"(z), "r"(b0), "r"(b1));
+}
+// D(16x8,f32) += A(16x8,bf16,row) * B(8x8,bf16,col)
+__device__ __forceinline__ void mma_pv(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
+  asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a0), "r"(a1), "r"(b0));
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// ---- score key of one code: sum over planes of weight * popc(agree & mask); agree = ~(h ^ sign)
+template <int W32, int NP>
+__device__ __forceinline__ int score_key(const uint32_t (&h)[W32], const uint32_t (&sg)[W32], const uint32_t (&mk)[NP][W32]) {
+  int key = 0;
+#pragma unroll
+  for (int pl = 0; pl < NP; ++pl) {
+    int c = 0;
+#pragma unroll
+    for (int w = 0; w < W32; ++w) c += __popc(~(h[w] ^ sg[w]) & mk[pl][w]);
+    key += c << pl;
   }
-};
-template <> struct RowFrag<float> {
+  return key;
+}
+// 128-bit codes with two planes (weights 1 and 2): carry-save adders fold the eight masked words into five
+// before the population counts, which run on the 16-lane pipe
+__device__ __forceinline__ void csa(uint32_t a, uint32_t b, uint32_t c, uint32_t& sum, uint32_t& carry) {
+  sum = a ^ b ^ c;
+  carry = (a & b) | (a & c) | (b & c);
+}
+template <>
+__device__ __forceinline__ int score_key<4, 2>(const uint32_t (&h)[4], const uint32_t (&sg)[4], const uint32_t (&mk)[2][4]) {
+  uint32_t x0[4], x1[4];
+#pragma unroll
+  for (int w = 0; w < 4; ++w) {
+    const uint32_t agree = ~(h[w] ^ sg[w]);
+    x0[w] = agree & mk[0][w];
+    x1[w] = agree & mk[1][w];
+  }
+  uint32_t s0, c0, s1, c1, s2, c2;
+  csa(x0[0], x0[1], x0[2], s0, c0);       // ones -> one ones word + one twos word
+  csa(c0, x1[0], x1[1], s1, c1);          // twos -> twos + fours
+  csa(s1, x1[2], x1[3], s2, c2);
+  return __popc(s0) + __popc(x0[3]) + 2 * __popc(s2) + 4 * (__popc(c1) + __popc(c2));
+}
+
+// K/V row fragment of 8 consecutive dims held by one lane (fp32 caches; read from the staging ring)
+struct RowFragF32 {
   uint4 a, b;
-  __device__ __forceinline__ void load(const float* row, int hl) {
-    a = ld_stream_v4(row + 8 * hl); b = ld_stream_v4(row + 8 * hl + 4);
+  __device__ __forceinline__ void load(const unsigned char* row, int hl) {
+    a = *reinterpret_cast<const uint4*>(row + 32 * hl); b = *reinterpret_cast<const uint4*>(row + 32 * hl + 16);
   }
   __device__ __forceinline__ void get(double* f) const {
     f[0] = __uint_as_float(a.x); f[1] = __uint_as_float(a.y); f[2] = __uint_as_float(a.z); f[3] = __uint_as_float(a.w);
@@ -122,12 +206,13 @@ template <> struct RowFrag<float> {
 };
 
 template <typename KV, int GP, int W32, int MODE>
-__global__ void __launch_bounds__((GP <= 4) ? 512 : 256, 1)
+__global__ void __launch_bounds__((DecodeSmem<KV, GP, W32>::NT), 1)
 bpc_decode_kernel(const DecodeParams p) {
   typedef DecodeSmem<KV, GP, W32> L;
   typedef typename L::acc_t acc_t;
   constexpr int NT = L::NT, NW = L::NW, B = L::B;
   constexpr int NP = PlaneCount<GP, MODE>::value;
+  constexpr int ROWB = L::kRowBytes;
   extern __shared__ __align__(16) unsigned char smem[];
 
   cg::cluster_group cluster = cg::this_cluster();
@@ -160,42 +245,72 @@ bpc_decode_kernel(const DecodeParams p) {
     return;
   }
 
-  uint32_t* hist = reinterpret_cast<uint32_t*>(smem + L::off_hist);
-  uint32_t* tot = reinterpret_cast<uint32_t*>(smem + L::off_tot);
-  double* qd = reinterpret_cast<double*>(smem + L::off_qd);
-  double* pd = reinterpret_cast<double*>(smem + L::off_pd);
-  int32_t* idx_s = reinterpret_cast<int32_t*>(smem + L::off_idx);
-  acc_t* cta_acc = reinterpret_cast<acc_t*>(smem + L::off_cta);        // [GP][128], then m[GP], l[GP]
+  const int nbins = p.nbins;
+  const L plan(p.chunk_cap, nbins, p.stages);
+  uint32_t* hist = reinterpret_cast<uint32_t*>(smem + plan.off_hist);
+  uint32_t* tot = reinterpret_cast<uint32_t*>(smem + plan.off_tot);
+  float* qf_s = reinterpret_cast<float*>(smem + plan.off_qf);
+  double* pd = reinterpret_cast<double*>(smem + plan.off_pd);
+  int32_t* idx_s = reinterpret_cast<int32_t*>(smem + plan.off_idx);
+  acc_t* cta_acc = reinterpret_cast<acc_t*>(smem + plan.off_cta);      // [GP][128], then m[GP], l[GP]
   acc_t* cta_m = cta_acc + GP * BPC_D;
   acc_t* cta_l = cta_m + GP;
-  SmallState* st = reinterpret_cast<SmallState*>(smem + L::off_small);
-  uint16_t* sc = reinterpret_cast<uint16_t*>(smem + L::off_scores);
-  const int nbins = p.nbins;
+  SmallState* st = reinterpret_cast<SmallState*>(smem + plan.off_small);
+  unsigned char* uni = smem + plan.off_union;
+  uint16_t* sc = reinterpret_cast<uint16_t*>(uni);
+#define BPC_STAMP(i) do { if (p.dbg_times != nullptr && tid == 0) p.dbg_times[(size_t)blockIdx.x * 16 + (i)] = global_timer_ns(); } while (0)
+  BPC_STAMP(0);
 
   // ------------------------------------------------------------------ phase 0: query hash
+  // p[g][j] = P_h[j] . q_g.  Thread (part, j) covers a slice of the 128 channels of row j: products are
+  // summed eight at a time in fp32 (exact products for bf16 inputs) and the groups are added in fp64; the
+  // slices are then added in fp64 in a fixed order.  Every block of the cluster gets identical bits.
   const KV* qg = reinterpret_cast<const KV*>(p.q) + ((size_t)seq * p.n_kv_heads + kvh) * (size_t)G * BPC_D;
-  for (int i = tid; i < GP * BPC_D; i += NT) qd[i] = (i >> 7) < G ? (double)to_float(qg[i]) : 0.0;
+  for (int i = tid; i < GP * BPC_D; i += NT) qf_s[i] = (i >> 7) < G ? to_float(qg[i]) : 0.f;
   for (int i = tid; i < nbins; i += NT) hist[i] = 0u;
   if (tid < BPC_MAX_CLUSTER) { st->gt[tid] = 0u; st->eq[tid] = 0u; }
   if (tid == 0) { st->rsum = 0; st->T = 0; st->cnt_gt = 0; }
   __syncthreads();
   {
-    const KV* Ph = reinterpret_cast<const KV*>(p.P_h) + (size_t)(p.shared_sets ? kvh : unit) * B * BPC_D;
-#pragma unroll 4
-    for (int j = warp; j < B; j += NW) {
-      const KV* row = Ph + (size_t)j * BPC_D + 4 * lane;
-      double pv[4];
+    constexpr int PARTS = NT / B;                  // slices per row
+    constexpr int DS = BPC_D / PARTS;              // channels per slice (a multiple of 8)
+    const int j = tid % B, part = tid / B;
+    const KV* row = reinterpret_cast<const KV*>(p.P_h) + ((size_t)(p.shared_sets ? kvh : unit) * B + j) * BPC_D + part * DS;
+    double acc[GP];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) pv[c] = (double)to_float(row[c]);
+    for (int g = 0; g < GP; ++g) acc[g] = 0.0;
+#pragma unroll 2
+    for (int c0 = 0; c0 < DS; c0 += 8) {
+      float pv[8];
+      if (L::kMma) {
+        const uint4 w = *reinterpret_cast<const uint4*>(row + c0);
+        pv[0] = bf16_lo(w.x); pv[1] = bf16_hi(w.x); pv[2] = bf16_lo(w.y); pv[3] = bf16_hi(w.y);
+        pv[4] = bf16_lo(w.z); pv[5] = bf16_hi(w.z); pv[6] = bf16_lo(w.w); pv[7] = bf16_hi(w.w);
+      } else {
+        const float4 w0 = *reinterpret_cast<const float4*>(row + c0);
+        const float4 w1 = *reinterpret_cast<const float4*>(row + c0 + 4);
+        pv[0] = w0.x; pv[1] = w0.y; pv[2] = w0.z; pv[3] = w0.w; pv[4] = w1.x; pv[5] = w1.y; pv[6] = w1.z; pv[7] = w1.w;
+      }
 #pragma unroll
       for (int g = 0; g < GP; ++g) {
-        const double* qq = qd + g * BPC_D + 4 * lane;
-        double s = pv[0] * qq[0];
-        s = fma(pv[1], qq[1], s); s = fma(pv[2], qq[2], s); s = fma(pv[3], qq[3], s);
-#pragma unroll
-        for (int o = 16; o >= 1; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        if (lane == 0) pd[g * B + j] = s;
+        const float4 q0 = *reinterpret_cast<const float4*>(qf_s + g * BPC_D + part * DS + c0);
+        const float4 q1 = *reinterpret_cast<const float4*>(qf_s + g * BPC_D + part * DS + c0 + 4);
+        float s0 = pv[0] * q0.x, s1 = pv[1] * q0.y;
+        s0 = fmaf(pv[2], q0.z, s0); s1 = fmaf(pv[3], q0.w, s1);
+        s0 = fmaf(pv[4], q1.x, s0); s1 = fmaf(pv[5], q1.y, s1);
+        s0 = fmaf(pv[6], q1.z, s0); s1 = fmaf(pv[7], q1.w, s1);
+        acc[g] += (double)s0 + (double)s1;
       }
+    }
+    double* hp = reinterpret_cast<double*>(uni);   // [PARTS][GP][B]
+#pragma unroll
+    for (int g = 0; g < GP; ++g) hp[((size_t)part * GP + g) * B + j] = acc[g];
+    __syncthreads();
+    for (int i = tid; i < GP * B; i += NT) {       // i = g * B + j
+      double s = 0.0;
+#pragma unroll
+      for (int pt = 0; pt < PARTS; ++pt) s += hp[(size_t)pt * GP * B + i];
+      pd[i] = s;
     }
   }
   __syncthreads();
@@ -237,6 +352,7 @@ bpc_decode_kernel(const DecodeParams p) {
   }
   __syncthreads();
 
+  BPC_STAMP(1);
   // ------------------------------------------------------------------ phase 1: scan
   const int c0 = min(n, rank * chunk), c1 = min(n, c0 + chunk);
   {
@@ -250,54 +366,91 @@ bpc_decode_kernel(const DecodeParams p) {
     const int rfull = st->rsum << cs;                       // sum_j |A_j|
     const uint32_t* cu = reinterpret_cast<const uint32_t*>(p.codes) + (size_t)unit * (size_t)p.n_max * W32;
     int32_t* dbg = p.dbg_scores != nullptr ? p.dbg_scores + (size_t)unit * p.n_max : nullptr;
-    constexpr int U = 4;
-    for (int i0 = c0; i0 < c1; i0 += NT * U) {
-      uint32_t h[U][W32];
+    constexpr int U = W32 <= 4 ? 8 : 4;                     // codes in flight per thread and buffer
+    auto load_code = [&](uint32_t (&h)[W32], int i) {
+      const uint32_t* src = cu + (size_t)i * W32;
+      if (W32 == 2) {
+        const uint2 v = ld_stream_v2(src); h[0] = v.x; h[1] = v.y;
+      } else {
 #pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int i = i0 + u * NT + tid;
-        if (i < c1) {
-          const uint32_t* src = cu + (size_t)i * W32;
-          if (W32 == 2) {
-            const uint2 v = ld_stream_v2(src); h[u][0] = v.x; h[u][1] = v.y;
-          } else {
-#pragma unroll
-            for (int w = 0; w < W32; w += 4) {
-              const uint4 v = ld_stream_v4(src + w);
-              h[u][w] = v.x; h[u][w + 1] = v.y; h[u][w + 2] = v.z; h[u][w + 3] = v.w;
-            }
-          }
-        } else {
-#pragma unroll
-          for (int w = 0; w < W32; ++w) h[u][w] = 0u;
+        for (int w = 0; w < W32; w += 4) {
+          const uint4 v = ld_stream_v4(src + w);
+          h[w] = v.x; h[w + 1] = v.y; h[w + 2] = v.z; h[w + 3] = v.w;
         }
       }
+    };
+    auto load_batch = [&](uint32_t (&h)[U][W32], int base) {
+#pragma unroll
+      for (int u = 0; u < U; ++u) load_code(h[u], base + u * NT + tid);
+    };
+    auto score_batch = [&](const uint32_t (&h)[U][W32], int base) {
 #pragma unroll
       for (int u = 0; u < U; ++u) {
-        const int i = i0 + u * NT + tid;
-        if (i < c1) {
-          int key = 0;
-#pragma unroll
-          for (int pl = 0; pl < NP; ++pl) {
-            int c = 0;
-#pragma unroll
-            for (int w = 0; w < W32; ++w) c += __popc(~(h[u][w] ^ sg[w]) & mk[pl][w]);
-            key += c << pl;
-          }
-          sc[score_slot(i - c0)] = (uint16_t)key;
-          atomicAdd(&hist[key], 1u);
-          if (dbg != nullptr) dbg[i] = ((2 * key) << cs) - rfull;
+        const int key = score_key<W32, NP>(h[u], sg, mk);
+        sc[score_slot(base - c0 + u * NT + tid)] = (uint16_t)key;
+        atomicAdd(&hist[key], 1u);
+      }
+    };
+    int i0 = c0;
+    if (dbg == nullptr) {
+      // Full batches without bounds checks, software-pipelined over two register buffers so that the
+      // loads of the next batch are in flight while the current one is scored (a warp's 32 keys share
+      // one score segment).
+      constexpr int STEP = NT * U;
+      if (i0 + STEP <= c1) {
+        uint32_t ha[U][W32], hb[U][W32];
+        load_batch(ha, i0);
+        for (;;) {
+          const bool more_b = i0 + 2 * STEP <= c1;
+          if (more_b) load_batch(hb, i0 + STEP);
+          score_batch(ha, i0);
+          i0 += STEP;
+          if (!more_b) break;
+          const bool more_a = i0 + 2 * STEP <= c1;
+          if (more_a) load_batch(ha, i0 + STEP);
+          score_batch(hb, i0);
+          i0 += STEP;
+          if (!more_a) break;
         }
+      }
+    }
+    for (; i0 < c1; i0 += NT) {                             // tail (and the whole range when scores are exported)
+      const int i = i0 + tid;
+      if (i < c1) {
+        uint32_t h[W32];
+        load_code(h, i);
+        const int key = score_key<W32, NP>(h, sg, mk);
+        sc[score_slot(i - c0)] = (uint16_t)key;
+        atomicAdd(&hist[key], 1u);
+        if (dbg != nullptr) dbg[i] = ((2 * key) << cs) - rfull;
       }
     }
   }
 
+  BPC_STAMP(2);
   // ------------------------------------------------------------------ phase 2: threshold and ordered selection
   cluster.sync();                                            // every block's histogram is complete
-  for (int bin = tid; bin < nbins; bin += NT) {
-    uint32_t s = 0;
-    for (int r = 0; r < CS; ++r) s += cluster.map_shared_rank(hist, r)[bin];
-    tot[bin] = s;
+  BPC_STAMP(8);
+  // Total histogram through distributed shared memory.  With at most one bin per thread (the common case)
+  // the per-block counts of that bin stay in registers and are reused for the per-block offsets below.
+  const bool one_bin = nbins <= NT;
+  uint32_t myv[BPC_MAX_CLUSTER];
+#pragma unroll
+  for (int r = 0; r < BPC_MAX_CLUSTER; ++r) myv[r] = 0u;
+  if (one_bin) {
+    if (tid < nbins) {
+      uint32_t s = 0;
+#pragma unroll
+      for (int r = 0; r < BPC_MAX_CLUSTER; ++r)
+        if (r < CS) { myv[r] = cluster.map_shared_rank(hist, r)[tid]; s += myv[r]; }
+      tot[tid] = s;
+    }
+  } else {
+    for (int bin = tid; bin < nbins; bin += NT) {
+      uint32_t s = 0;
+      for (int r = 0; r < CS; ++r) s += cluster.map_shared_rank(hist, r)[bin];
+      tot[bin] = s;
+    }
   }
   __syncthreads();
   {
@@ -316,14 +469,27 @@ bpc_decode_kernel(const DecodeParams p) {
   }
   __syncthreads();
   const int T = st->T;
-  for (int bin = T + 1 + tid; bin < nbins; bin += NT) {
-    if (tot[bin] == 0u) continue;
-    for (int r = 0; r < CS; ++r) {
-      const uint32_t v = cluster.map_shared_rank(hist, r)[bin];
-      if (v) atomicAdd(&st->gt[r], v);
+  BPC_STAMP(9);
+  if (one_bin) {
+    if (tid < nbins && tid >= T) {
+#pragma unroll
+      for (int r = 0; r < BPC_MAX_CLUSTER; ++r) {
+        if (r < CS) {
+          if (tid == T) st->eq[r] = myv[r];
+          else if (myv[r]) atomicAdd(&st->gt[r], myv[r]);
+        }
+      }
     }
+  } else {
+    for (int bin = T + 1 + tid; bin < nbins; bin += NT) {
+      if (tot[bin] == 0u) continue;
+      for (int r = 0; r < CS; ++r) {
+        const uint32_t v = cluster.map_shared_rank(hist, r)[bin];
+        if (v) atomicAdd(&st->gt[r], v);
+      }
+    }
+    if (tid < CS) st->eq[tid] = cluster.map_shared_rank(hist, tid)[T];
   }
-  if (tid < CS) st->eq[tid] = cluster.map_shared_rank(hist, tid)[T];
   __syncthreads();
   if (tid == 0) {
     const int need = k - st->cnt_gt;                         // ties to take, cluster-wide (>= 1)
@@ -338,42 +504,69 @@ bpc_decode_kernel(const DecodeParams p) {
   }
   __syncthreads();
   int32_t* sel_u = p.sel + (size_t)unit * p.n_max;
+  BPC_STAMP(10);
   {
+    // Each thread owns whole 32-key segments, in ascending order within a pass.  Two keys share a 32-bit
+    // word; adding (0x8000 - T) to both halves raises bit 15 / bit 31 exactly for keys >= T (keys < 2048),
+    // which is shifted into a 32-bit candidate mask without branches.  Only the few candidates are looked
+    // at again (re-read from shared memory) to tell "greater" from "tie".
     const int len = c1 - c0;
     const int nseg = (len + kSegKeys - 1) / kSegKeys;
     const int my_take = st->my_take;
+    const uint32_t cge = (uint32_t)(0x8000 - T) * 0x10001u;
+    constexpr int SPT = 4;                                   // most consecutive segments one thread takes per pass
+    const int spt = min(SPT, (nseg + NT - 1) / NT);
     int run_gt = 0, run_eq = 0;
-    for (int s0 = 0; s0 < nseg; s0 += NT) {
-      const int seg = s0 + tid;
-      uint32_t kw[16];
+    for (int s0 = 0; s0 < nseg; s0 += NT * spt) {
+      uint32_t M[SPT], Mgt[SPT];                             // bit j: key j of the segment is >= T / > T
       int cgt = 0, ceq = 0;
-      if (seg < nseg) {
-        const uint4* src = reinterpret_cast<const uint4*>(sc + (size_t)seg * kSegSlots);
 #pragma unroll
-        for (int v = 0; v < 4; ++v) {
-          const uint4 x = src[v];
-          kw[4 * v] = x.x; kw[4 * v + 1] = x.y; kw[4 * v + 2] = x.z; kw[4 * v + 3] = x.w;
-        }
-        const int valid = min(kSegKeys, len - seg * kSegKeys);
+      for (int q = 0; q < SPT; ++q) {
+        M[q] = 0u; Mgt[q] = 0u;
+        const int seg = s0 + tid * spt + q;
+        if (q < spt && seg < nseg) {
+          const uint4* src = reinterpret_cast<const uint4*>(sc + (size_t)seg * kSegSlots);
+          uint32_t kw[16];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const int key = (int)((kw[j >> 1] >> ((j & 1) * 16)) & 0xffffu);
-          if (j < valid) { cgt += key > T; ceq += key == T; }
+          for (int v = 0; v < 4; ++v) {
+            const uint4 x = src[v];
+            kw[4 * v] = x.x; kw[4 * v + 1] = x.y; kw[4 * v + 2] = x.z; kw[4 * v + 3] = x.w;
+          }
+          uint32_t m = 0;
+#pragma unroll
+          for (int w = 0; w < 16; ++w) {
+            const uint32_t gq = kw[w] + cge;
+            m |= (2 * w <= 15 ? (gq >> (15 - 2 * w)) : (gq << (2 * w - 15))) & (1u << (2 * w));
+            m |= (gq >> (30 - 2 * w)) & (2u << (2 * w));
+          }
+          const int valid = len - seg * kSegKeys;
+          if (valid < kSegKeys) m &= (1u << valid) - 1u;     // slots past the end of the chunk hold stale bytes
+          uint32_t rem = m, mg = 0;
+          while (rem) {
+            const int j = __ffs(rem) - 1;
+            rem &= rem - 1;
+            if ((int)sc[(size_t)seg * kSegSlots + j] > T) mg |= 1u << j;
+          }
+          M[q] = m; Mgt[q] = mg;
+          cgt += __popc(mg);
+          ceq += __popc(m) - __popc(mg);
         }
       }
       uint32_t total;
       const uint32_t ex = block_excl_scan<NT>((uint32_t)cgt | ((uint32_t)ceq << 16), st->wscan, &total);
-      if (seg < nseg && (cgt | ceq)) {
+      if (cgt | ceq) {
         int eqb = run_eq + (int)(ex >> 16);
         int pos = st->my_base + run_gt + (int)(ex & 0xffffu) + min(eqb, my_take);
-        const int valid = min(kSegKeys, len - seg * kSegKeys);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const int key = (int)((kw[j >> 1] >> ((j & 1) * 16)) & 0xffffu);
-          if (j < valid) {
-            if (key > T) {
+        for (int q = 0; q < SPT; ++q) {
+          const int seg = s0 + tid * spt + q;
+          uint32_t rem = M[q];
+          while (rem) {
+            const int j = __ffs(rem) - 1;
+            rem &= rem - 1;
+            if ((Mgt[q] >> j) & 1u) {
               sel_u[pos++] = c0 + seg * kSegKeys + j;
-            } else if (key == T) {
+            } else {
               if (eqb < my_take) sel_u[pos++] = c0 + seg * kSegKeys + j;
               ++eqb;
             }
@@ -384,113 +577,247 @@ bpc_decode_kernel(const DecodeParams p) {
       run_eq += (int)(total >> 16);
     }
   }
+  BPC_STAMP(3);
   __threadfence();
   cluster.sync();                                            // the unit's index list is complete and visible
+  BPC_STAMP(4);
 
   // ------------------------------------------------------------------ phase 3: gathered attention
-  const int hl = lane & 15, half = lane >> 4;
   const int lo = (int)(((long long)k * rank) / CS), hi = (int)(((long long)k * (rank + 1)) / CS);
-  acc_t qf[GP][8], acc[GP][8], m_run[GP], l_run[GP];
-  {
-    const double scale = (double)p.sm_scale * 1.4426950408889634;   // logits in base-2 exponent units
-#pragma unroll
-    for (int g = 0; g < GP; ++g) {
-#pragma unroll
-      for (int c = 0; c < 8; ++c) { qf[g][c] = (acc_t)(qd[g * BPC_D + 8 * hl + c] * scale); acc[g][c] = (acc_t)0; }
-      m_run[g] = (acc_t)-1e30; l_run[g] = (acc_t)0;
-    }
-  }
-  const KV* Ku = reinterpret_cast<const KV*>(p.k_cache) + (size_t)unit * (size_t)p.n_max * BPC_D;
-  const KV* Vu = reinterpret_cast<const KV*>(p.v_cache) + (size_t)unit * (size_t)p.n_max * BPC_D;
+  const size_t rstride = (size_t)p.row_stride * sizeof(KV);   // bytes between consecutive cache rows
+  const unsigned char* Ku = reinterpret_cast<const unsigned char*>(p.k_cache) + (size_t)unit * (size_t)p.n_max * rstride;
+  const unsigned char* Vu = reinterpret_cast<const unsigned char*>(p.v_cache) + (size_t)unit * (size_t)p.n_max * rstride;
+  constexpr int TR = L::kTileRows, CPR = ROWB / 16;
+  const int NS = p.stages;
+  unsigned char* stg = uni;
+  acc_t* part = reinterpret_cast<acc_t*>(uni);               // [NW][GP][130]; aliases the ring (used after it)
+  const float scale2 = (float)(p.sm_scale_d * 1.4426950408889634);   // logits in base-2 exponent units
 
-  auto process = [&](const RowFrag<KV>& kf, const RowFrag<KV>& vf, bool valid) {
-    acc_t kv8[8], s[GP];
-    kf.get(kv8);
+  if constexpr (L::kMma) {
+    // ---- bf16: tensor-core path.  Warp w owns rows 8w..8w+7 of every tile.
+    //   S^T[head][key] = Q (16 x 128, rows >= G zero) . K_tile^T : 8 MMAs m16n8k16 per 8 keys
+    //   O[head][dim]  += P (16 x 8; rows 0-7 = bf16(p), rows 8-15 = bf16(p - bf16(p))) . V_tile : 16 MMAs m16n8k8
+    // Lane (g = lane/4, t = lane%4) holds the logits of head g for keys 2t, 2t+1 and, in every 8-dim output
+    // tile, dims 2t, 2t+1 of head g (high part in d[0..1], low part in d[2..3]).
+    const int g = lane >> 2, t = lane & 3;
+    uint32_t qa0[8], qa2[8];
+    {
+      const uint32_t* qw = reinterpret_cast<const uint32_t*>(qg + (size_t)g * BPC_D);
 #pragma unroll
-    for (int g = 0; g < GP; ++g) {
-      acc_t d = qf[g][0] * kv8[0];
-#pragma unroll
-      for (int c = 1; c < 8; ++c) d = fma(qf[g][c], kv8[c], d);
-      s[g] = d;
+      for (int s = 0; s < 8; ++s) {
+        qa0[s] = g < G ? qw[8 * s + t] : 0u;                 // dims 16s + 2t, +1
+        qa2[s] = g < G ? qw[8 * s + 4 + t] : 0u;             // dims 16s + 8 + 2t, +1
+      }
     }
+    float o[16][4];
 #pragma unroll
-    for (int o = 8; o >= 1; o >>= 1) {
+    for (int j = 0; j < 16; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
+    float m_run = -1e30f, l_run = 0.f;
+    const int lrow = lane & 7, lmat = lane >> 3;             // ldmatrix: lane supplies row lrow of matrix lmat
+
+    // Every warp runs its own gather ring (no block barriers): it owns the 8-row blocks warp, warp+NW, ... of
+    // the block's slice, copies a block's K and V rows with one 16-byte asynchronous copy per lane and row
+    // (lanes 0-15 the K row, lanes 16-31 the V row; chunks XOR-swizzled by the row number so that ldmatrix
+    // reads are conflict-free), keeps NS-1 blocks in flight and multiplies the oldest one.
+    constexpr int WSTG = 8 * 2 * ROWB;                       // bytes of one 8-row stage (K rows, then V rows)
+    unsigned char* wst = stg + (size_t)warp * NS * WSTG;
+    const int nblk = (hi - lo + 7) >> 3;
+    const int isv = lane >> 4, ch = lane & 15;
+    const unsigned char* srcbase = (isv ? Vu : Ku) + (size_t)ch * 16;
+    auto issue = [&](int bi) {
+      const int blk = warp + bi * NW;
+      if (blk < nblk) {
+        const int rbase = lo + 8 * blk;
+        int myidx = -1;
+        if (lane < 8 && rbase + lane < hi) myidx = min(max(sel_u[rbase + lane], 0), p.n_max - 1);
+        unsigned char* dst = wst + (size_t)(bi % NS) * WSTG + (size_t)isv * (8 * ROWB);
 #pragma unroll
-      for (int g = 0; g < GP; ++g) s[g] += __shfl_xor_sync(0xffffffffu, s[g], o);
-    }
-    bool grow = false;
-#pragma unroll
-    for (int g = 0; g < GP; ++g) grow |= (s[g] > m_run[g]);
-    grow &= valid;
-    if (__any_sync(0xffffffffu, grow)) {
-      if (valid) {
-#pragma unroll
-        for (int g = 0; g < GP; ++g) {
-          if (s[g] > m_run[g]) {
-            const acc_t corr = fast_exp2<acc_t>(m_run[g] - s[g]);
-            l_run[g] *= corr;
-#pragma unroll
-            for (int c = 0; c < 8; ++c) acc[g][c] *= corr;
-            m_run[g] = s[g];
+        for (int it = 0; it < 8; ++it) {
+          const int idx = __shfl_sync(0xffffffffu, myidx, it);
+          unsigned char* d = dst + it * ROWB + ((ch ^ it) << 4);
+          if (idx >= 0) {
+            cp_async16(d, srcbase + (size_t)idx * rstride);
+          } else {
+            // rows past the end of the list get zeros: their probabilities are zero, and 0 * stale NaN
+            // must not reach the accumulators
+            *reinterpret_cast<uint4*>(d) = make_uint4(0u, 0u, 0u, 0u);
           }
         }
       }
+      cp_async_commit();
+    };
+    for (int tt = 0; tt < NS - 1; ++tt) issue(tt);
+    for (int bi = 0; warp + bi * NW < nblk; ++bi) {
+      if (NS == 2) cp_async_wait<0>(); else cp_async_wait<1>();   // this lane's copies for block bi have landed
+      __syncwarp();                                          // ... and every lane's
+      issue(bi + NS - 1);                                    // refill the stage consumed in the previous round
+      const int rbase = lo + 8 * (warp + bi * NW);
+      const unsigned char* ks = wst + (size_t)(bi % NS) * WSTG;
+      const unsigned char* vs = ks + 8 * ROWB;
+      float s[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int jj = 0; jj < 4; ++jj) {                       // 32 dims per ldmatrix.x4: chunks 4jj .. 4jj+3
+        uint32_t b[4];
+        ldmatrix_x4(b, ks + (size_t)lrow * ROWB + (((4 * jj + lmat) ^ lrow) << 4));
+        mma_qk(s, qa0[2 * jj], qa2[2 * jj], b[0], b[1]);
+        mma_qk(s, qa0[2 * jj + 1], qa2[2 * jj + 1], b[2], b[3]);
+      }
+      const bool v0 = rbase + 2 * t < hi, v1 = rbase + 2 * t + 1 < hi;
+      const float s0 = v0 ? s[0] * scale2 : -1e30f, s1 = v1 ? s[1] * scale2 : -1e30f;
+      float tmax = fmaxf(s0, s1);
+      tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+      tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+      if (__any_sync(0xffffffffu, tmax > m_run)) {
+        if (tmax > m_run) {
+          const float corr = exp2f(m_run - tmax);
+          l_run *= corr;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) { o[j][0] *= corr; o[j][1] *= corr; o[j][2] *= corr; o[j][3] *= corr; }
+          m_run = tmax;
+        }
+      }
+      const float p0 = v0 ? exp2f(s0 - m_run) : 0.f, p1 = v1 ? exp2f(s1 - m_run) : 0.f;
+      l_run += p0 + p1;
+      const __nv_bfloat162 hi2 = __floats2bfloat162_rn(p0, p1);
+      const float r0f = p0 - __low2float(hi2), r1f = p1 - __high2float(hi2);
+      const uint32_t pa0 = *reinterpret_cast<const uint32_t*>(&hi2);
+      const uint32_t pa1 = pack_bf16x2(r0f, r1f);
+#pragma unroll
+      for (int jj = 0; jj < 4; ++jj) {
+        uint32_t b[4];
+        ldmatrix_x4_trans(b, vs + (size_t)lrow * ROWB + (((4 * jj + lmat) ^ lrow) << 4));
+        mma_pv(o[4 * jj], pa0, pa1, b[0]);
+        mma_pv(o[4 * jj + 1], pa0, pa1, b[1]);
+        mma_pv(o[4 * jj + 2], pa0, pa1, b[2]);
+        mma_pv(o[4 * jj + 3], pa0, pa1, b[3]);
+      }
+      __syncwarp();
     }
-    vf.get(kv8);
-#pragma unroll
-    for (int g = 0; g < GP; ++g) {
-      const acc_t pr = valid ? fast_exp2<acc_t>(s[g] - m_run[g]) : (acc_t)0;
-      l_run[g] += pr;
-#pragma unroll
-      for (int c = 0; c < 8; ++c) acc[g][c] = fma(pr, kv8[c], acc[g][c]);
-    }
-  };
-
-  for (int t0 = lo; t0 < hi; t0 += kIdxTile) {
-    const int tn = min(kIdxTile, hi - t0);
-    __syncthreads();
-    for (int i = tid; i < tn; i += NT) idx_s[i] = sel_u[t0 + i];
-    __syncthreads();
-    // a warp handles two rows per pass (one per half warp), two passes per iteration
-    for (int rp = warp; 2 * rp < tn; rp += 2 * NW) {
-      const int r0 = 2 * rp + half, r1 = 2 * (rp + NW) + half;
-      const bool v0 = r0 < tn, v1 = r1 < tn;
-      const int i0 = min(max(idx_s[v0 ? r0 : 0], 0), p.n_max - 1);
-      const int i1 = min(max(idx_s[v1 ? r1 : 0], 0), p.n_max - 1);
-      RowFrag<KV> k0, vv0, k1, vv1;
-      k0.load(Ku + (size_t)i0 * BPC_D, hl); vv0.load(Vu + (size_t)i0 * BPC_D, hl);
-      k1.load(Ku + (size_t)i1 * BPC_D, hl); vv1.load(Vu + (size_t)i1 * BPC_D, hl);
-      process(k0, vv0, v0);
-      process(k1, vv1, v1);
-    }
-  }
-
-  // merge the two half warps, then the warps of the block
-  acc_t* part = reinterpret_cast<acc_t*>(sc);                // [NW][GP][130]: the score storage is free now
-#pragma unroll
-  for (int g = 0; g < GP; ++g) {
-    const acc_t om = __shfl_xor_sync(0xffffffffu, m_run[g], 16);
-    const acc_t ol = __shfl_xor_sync(0xffffffffu, l_run[g], 16);
-    const acc_t mm = om > m_run[g] ? om : m_run[g];
-    const acc_t ws = fast_exp2<acc_t>(m_run[g] - mm), wo = fast_exp2<acc_t>(om - mm);
-    l_run[g] = l_run[g] * ws + ol * wo;
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      const acc_t oa = __shfl_xor_sync(0xffffffffu, acc[g][c], 16);
-      acc[g][c] = acc[g][c] * ws + oa * wo;
-    }
-    m_run[g] = mm;
-  }
-  __syncthreads();                                           // all reads of the score storage are done
-  if (half == 0) {
-#pragma unroll
-    for (int g = 0; g < GP; ++g) {
+    cp_async_wait<0>();
+    // lanes of one head (same g) hold partial sums of l over their keys
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+    __syncthreads();                                         // the ring is no longer read: reuse it for the merge
+    if (g < GP) {
       acc_t* dst = part + ((size_t)warp * GP + g) * (BPC_D + 2);
 #pragma unroll
-      for (int c = 0; c < 8; ++c) dst[8 * hl + c] = acc[g][c];
-      if (hl == 0) { dst[BPC_D] = m_run[g]; dst[BPC_D + 1] = l_run[g]; }
+      for (int j = 0; j < 16; ++j) {
+        dst[8 * j + 2 * t] = o[j][0] + o[j][2];
+        dst[8 * j + 2 * t + 1] = o[j][1] + o[j][3];
+      }
+      if (t == 0) { dst[BPC_D] = m_run; dst[BPC_D + 1] = l_run; }
+    }
+  } else {
+    // ---- fp32 caches: fp64 logits and averages on the CUDA cores, half a warp per row
+    const int hl = lane & 15, half = lane >> 4;
+    acc_t qf[GP][8], acc[GP][8], m_run[GP], l_run[GP];
+#pragma unroll
+    for (int gg = 0; gg < GP; ++gg) {
+#pragma unroll
+      for (int c = 0; c < 8; ++c) { qf[gg][c] = (acc_t)qf_s[gg * BPC_D + 8 * hl + c] * (acc_t)(p.sm_scale_d * 1.4426950408889634); acc[gg][c] = (acc_t)0; }
+      m_run[gg] = (acc_t)-1e30; l_run[gg] = (acc_t)0;
+    }
+    auto process = [&](const RowFragF32& kf, const RowFragF32& vf, bool valid) {
+      acc_t kv8[8], s[GP];
+      kf.get(kv8);
+#pragma unroll
+      for (int gg = 0; gg < GP; ++gg) {
+        acc_t d = qf[gg][0] * kv8[0];
+#pragma unroll
+        for (int c = 1; c < 8; ++c) d = fma(qf[gg][c], kv8[c], d);
+        s[gg] = d;
+      }
+#pragma unroll
+      for (int o = 8; o >= 1; o >>= 1) {
+#pragma unroll
+        for (int gg = 0; gg < GP; ++gg) s[gg] += __shfl_xor_sync(0xffffffffu, s[gg], o);
+      }
+      if (valid) {                                           // rows past the tile's end hold stale bytes
+#pragma unroll
+        for (int gg = 0; gg < GP; ++gg) {
+          if (s[gg] > m_run[gg]) {
+            const acc_t corr = fast_exp2<acc_t>(m_run[gg] - s[gg]);
+            l_run[gg] *= corr;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) acc[gg][c] *= corr;
+            m_run[gg] = s[gg];
+          }
+        }
+        vf.get(kv8);
+#pragma unroll
+        for (int gg = 0; gg < GP; ++gg) {
+          const acc_t pr = fast_exp2<acc_t>(s[gg] - m_run[gg]);
+          l_run[gg] += pr;
+#pragma unroll
+          for (int c = 0; c < 8; ++c) acc[gg][c] = fma(pr, kv8[c], acc[gg][c]);
+        }
+      }
+    };
+    for (int t0 = lo; t0 < hi; t0 += kIdxTile) {
+      const int tn = min(kIdxTile, hi - t0);
+      __syncthreads();
+      for (int i = tid; i < tn; i += NT) idx_s[i] = min(max(sel_u[t0 + i], 0), p.n_max - 1);
+      __syncthreads();
+      const int ntile = (tn + TR - 1) / TR;
+      auto issue = [&](int tile) {
+        if (tile < ntile) {
+          unsigned char* dst = stg + (size_t)(tile % NS) * L::kStageBytes;
+          const int r0 = tile * TR;
+          for (int c = tid; c < TR * 2 * CPR; c += NT) {
+            const int row = c / (2 * CPR), within = c % (2 * CPR);
+            const int isv = within / CPR, ch = within % CPR;
+            if (r0 + row < tn) {
+              const size_t off = (size_t)idx_s[r0 + row] * rstride + (size_t)ch * 16;
+              cp_async16(dst + (size_t)row * 2 * ROWB + isv * ROWB + ch * 16, (isv ? Vu : Ku) + off);
+            }
+          }
+        }
+        cp_async_commit();
+      };
+      for (int tt = 0; tt < NS - 1; ++tt) issue(tt);
+      for (int tile = 0; tile < ntile; ++tile) {
+        if (NS == 2) cp_async_wait<0>(); else cp_async_wait<1>();
+        __syncthreads();
+        issue(tile + NS - 1);
+        const unsigned char* src = stg + (size_t)(tile % NS) * L::kStageBytes;
+        const int r0 = tile * TR;
+        for (int rp = warp; 2 * rp < TR; rp += NW) {
+          const int r = 2 * rp + half;
+          RowFragF32 kf, vf;
+          kf.load(src + (size_t)r * 2 * ROWB, hl);
+          vf.load(src + (size_t)r * 2 * ROWB + ROWB, hl);
+          process(kf, vf, r0 + r < tn);
+        }
+      }
+      cp_async_wait<0>();
+    }
+    // merge the two half warps
+#pragma unroll
+    for (int gg = 0; gg < GP; ++gg) {
+      const acc_t om = __shfl_xor_sync(0xffffffffu, m_run[gg], 16);
+      const acc_t ol = __shfl_xor_sync(0xffffffffu, l_run[gg], 16);
+      const acc_t mm = om > m_run[gg] ? om : m_run[gg];
+      const acc_t ws = fast_exp2<acc_t>(m_run[gg] - mm), wo = fast_exp2<acc_t>(om - mm);
+      l_run[gg] = l_run[gg] * ws + ol * wo;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const acc_t oa = __shfl_xor_sync(0xffffffffu, acc[gg][c], 16);
+        acc[gg][c] = acc[gg][c] * ws + oa * wo;
+      }
+      m_run[gg] = mm;
+    }
+    __syncthreads();                                         // the ring is no longer read: reuse it for the merge
+    if (half == 0) {
+#pragma unroll
+      for (int gg = 0; gg < GP; ++gg) {
+        acc_t* dst = part + ((size_t)warp * GP + gg) * (BPC_D + 2);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) dst[8 * hl + c] = acc[gg][c];
+        if (hl == 0) { dst[BPC_D] = m_run[gg]; dst[BPC_D + 1] = l_run[gg]; }
+      }
     }
   }
+  BPC_STAMP(5);
   __syncthreads();
   for (int o = tid; o < GP * BPC_D; o += NT) {
     const int g = o >> 7, d = o & 127;
@@ -509,6 +836,7 @@ bpc_decode_kernel(const DecodeParams p) {
     cta_acc[o] = num;
     if (d == 0) { cta_m[g] = mm; cta_l[g] = den; }
   }
+  BPC_STAMP(6);
   cluster.sync();                                            // every block's partial result is published
   {
     const int nout = G * BPC_D;
@@ -531,6 +859,8 @@ bpc_decode_kernel(const DecodeParams p) {
     }
   }
   cluster.sync();                                            // keep shared memory alive until all peers have read it
+  BPC_STAMP(7);
+#undef BPC_STAMP
 }
 
 }  // namespace bpcdev

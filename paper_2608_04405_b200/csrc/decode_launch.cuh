@@ -18,10 +18,15 @@ static cudaError_t configure_kernel(int device) {
 }
 
 template <typename KV, int GP, int W32, int MODE>
-static cudaError_t launch_one(bpc_ctx* ctx, const DecodeParams& p, cudaStream_t stream) {
+static cudaError_t launch_one(bpc_ctx* ctx, const DecodeParams& p_in, cudaStream_t stream) {
   typedef DecodeSmem<KV, GP, W32> L;
-  const size_t smem = L::total(p.chunk_cap);
-  cudaError_t e = cudaSuccess;
+  DecodeParams p = p_in;
+  int optin = 0;
+  cudaError_t e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, ctx->device);
+  if (e != cudaSuccess) return e;
+  p.stages = L(p.chunk_cap, p.nbins, 3).total <= (size_t)optin ? 3 : 2;
+  const size_t smem = L(p.chunk_cap, p.nbins, p.stages).total;
+  if (smem > (size_t)optin) return cudaErrorInvalidConfiguration;
   if (ctx->decode_smem_set == 0) {                          // function attributes are sticky: set them once
     e = configure_kernel<KV, GP, W32, MODE>(ctx->device);
     if (e != cudaSuccess) return e;
@@ -42,31 +47,30 @@ static cudaError_t launch_one(bpc_ctx* ctx, const DecodeParams& p, cudaStream_t 
   return cudaLaunchKernelEx(&lc, bpc_decode_kernel<KV, GP, W32, MODE>, p);
 }
 
-// Largest cluster size (power of two) the device can schedule with `smem` bytes per block, and the
-// shared-memory budget of one block.
+// Largest cluster size (power of two) the device can schedule with a full-size block, and the number of
+// score keys one block can hold next to a two-stage gather ring.
 template <typename KV, int GP, int W32, int MODE>
-static cudaError_t limits_one(const bpc_ctx* ctx, int cluster_size, int* max_cluster, int* chunk_cap, size_t* smem_bytes) {
+static cudaError_t limits_one(const bpc_ctx* ctx, int nbins, int* max_cluster, int* chunk_cap, size_t* smem_bytes) {
   typedef DecodeSmem<KV, GP, W32> L;
   int dev = ctx->device, optin = 0;
   cudaError_t e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   if (e != cudaSuccess) return e;
-  // score capacity of one block: what is left of the opt-in shared memory after the fixed regions
-  const size_t fixed = L::off_scores;
-  size_t avail = (size_t)optin > fixed + 1024 ? (size_t)optin - fixed - 1024 : 0;
+  const size_t fixed = L(0, nbins, 2).off_union;
+  const size_t avail = (size_t)optin > fixed + 64 ? (size_t)optin - fixed - 64 : 0;
   int cap = (int)((avail / (kSegSlots * 2)) * kSegKeys);
   cap &= ~63;
+  if (L(cap, nbins, 2).total > (size_t)optin) cap = 0;
   if (chunk_cap) *chunk_cap = cap;
   if (smem_bytes) *smem_bytes = (size_t)optin;
   if (max_cluster) {
     int best = 1;
+    e = configure_kernel<KV, GP, W32, MODE>(dev);
+    if (e != cudaSuccess) return e;
     for (int cs = 2; cs <= BPC_MAX_CLUSTER; cs *= 2) {
-      const size_t smem = L::total(cap);
-      e = configure_kernel<KV, GP, W32, MODE>(dev);
-      if (e != cudaSuccess) return e;
       cudaLaunchConfig_t lc = {};
       lc.gridDim = dim3((unsigned)cs, 1, 1);
       lc.blockDim = dim3(L::NT, 1, 1);
-      lc.dynamicSmemBytes = smem;
+      lc.dynamicSmemBytes = (size_t)optin;
       cudaLaunchAttribute at[1];
       at[0].id = cudaLaunchAttributeClusterDimension;
       at[0].val.clusterDim.x = (unsigned)cs; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
@@ -79,7 +83,6 @@ static cudaError_t limits_one(const bpc_ctx* ctx, int cluster_size, int* max_clu
     }
     *max_cluster = best;
   }
-  (void)cluster_size;
   return cudaSuccess;
 }
 
@@ -103,9 +106,9 @@ static cudaError_t launch_dtype(bpc_ctx* ctx, const DecodeParams& p, cudaStream_
   BPC_DISPATCH_G(KV, 0, launch_one, ctx, p, stream)
 }
 template <typename KV>
-static cudaError_t limits_dtype(const bpc_ctx* ctx, int cluster_size, int* max_cluster, int* chunk_cap, size_t* smem) {
+static cudaError_t limits_dtype(const bpc_ctx* ctx, int nbins, int* max_cluster, int* chunk_cap, size_t* smem) {
   if (ctx->cfg.score_mode != BPC_SCORE_HAMMING) return cudaErrorNotSupported;
-  BPC_DISPATCH_G(KV, 0, limits_one, ctx, cluster_size, max_cluster, chunk_cap, smem)
+  BPC_DISPATCH_G(KV, 0, limits_one, ctx, nbins, max_cluster, chunk_cap, smem)
 }
 
 }  // namespace bpcdev

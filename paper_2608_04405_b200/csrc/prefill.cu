@@ -51,7 +51,7 @@ template <typename KV>
 __global__ void __launch_bounds__(kEncThreads)
 encode_simple_kernel(const KV* __restrict__ k_cache, const float* __restrict__ Phf, const float* __restrict__ gram,
                      const int32_t* __restrict__ unit_lens, uint64_t* __restrict__ codes, int n_kv_heads, int n_max,
-                     int b, int shared_sets, int residual_correction) {
+                     int row_stride, int b, int shared_sets, int residual_correction) {
   extern __shared__ __align__(16) unsigned char smem[];
   float* ps = reinterpret_cast<float*>(smem);                       // [128 rows of P][128]
   float* ts = ps + 128 * BPC_D;                                      // [b][kEncThreads]
@@ -65,7 +65,7 @@ encode_simple_kernel(const KV* __restrict__ k_cache, const float* __restrict__ P
   const bool live = key < n;
   float kr[BPC_D];
   {
-    const KV* row = k_cache + ((size_t)unit * n_max + (live ? key : 0)) * BPC_D;
+    const KV* row = k_cache + ((size_t)unit * n_max + (live ? key : 0)) * row_stride;
 #pragma unroll
     for (int c = 0; c < BPC_D; ++c) kr[c] = to_float(row[c]);
   }
@@ -116,8 +116,8 @@ template <typename KV>
 __global__ void __launch_bounds__(kAppThreads)
 append_kernel(const KV* __restrict__ k_new, const KV* __restrict__ v_new, KV* __restrict__ k_cache, KV* __restrict__ v_cache,
               uint64_t* __restrict__ codes, const KV* __restrict__ Ph, const float* __restrict__ gram,
-              int32_t* __restrict__ unit_lens, int32_t* __restrict__ err, int n_kv_heads, int n_max, int b,
-              int shared_sets, int residual_correction) {
+              int32_t* __restrict__ unit_lens, int32_t* __restrict__ err, int n_kv_heads, int n_max, int row_stride,
+              int b, int shared_sets, int residual_correction) {
   extern __shared__ __align__(16) unsigned char smem[];
   float* gs = reinterpret_cast<float*>(smem);                        // [b][b] when b <= 128
   __shared__ float t_s[256];
@@ -143,9 +143,9 @@ append_kernel(const KV* __restrict__ k_new, const KV* __restrict__ v_new, KV* __
   if (tid < BPC_D) {
     const KV kv = kn[tid];
     k_s[tid] = to_float(kv);
-    k_cache[((size_t)unit * n_max + n) * BPC_D + tid] = kv;
+    k_cache[((size_t)unit * n_max + n) * row_stride + tid] = kv;
   } else if (tid < 2 * BPC_D) {
-    v_cache[((size_t)unit * n_max + n) * BPC_D + (tid - BPC_D)] = vn[tid - BPC_D];
+    v_cache[((size_t)unit * n_max + n) * row_stride + (tid - BPC_D)] = vn[tid - BPC_D];
   }
   __syncthreads();
   // t_j = P_h[j] . k
@@ -217,7 +217,7 @@ template <typename KV>
 __global__ void __launch_bounds__(kFitThreads)
 fit_pass_kernel(const KV* __restrict__ k_cache, float* __restrict__ R, uint8_t* __restrict__ usign,
                 uint32_t* __restrict__ hfit, const float* __restrict__ v_star, const float* __restrict__ P, float* __restrict__ partials,
-                const int32_t* __restrict__ unit_lens, int n_max, int b, int it, int blocks_per_unit) {
+                const int32_t* __restrict__ unit_lens, int n_max, int row_stride, int b, int it, int blocks_per_unit) {
   const int unit = blockIdx.y;
   const int n = min(unit_lens[unit], n_max);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -232,7 +232,7 @@ fit_pass_kernel(const KV* __restrict__ k_cache, float* __restrict__ R, uint8_t* 
     const size_t ro = ((size_t)unit * n_max + r) * BPC_D;
     float4 x;
     if (it == 0) {
-      const KV* kr = k_cache + ro + 4 * lane;
+      const KV* kr = k_cache + ((size_t)unit * n_max + r) * row_stride + 4 * lane;
       x = make_float4(to_float(kr[0]), to_float(kr[1]), to_float(kr[2]), to_float(kr[3]));
     } else {
       x = reinterpret_cast<const float4*>(R + ro)[lane];
@@ -303,13 +303,13 @@ cudaError_t bpc_launch_encode_simple(bpc_ctx* ctx, const void* k_cache, uint64_t
     e = cudaFuncSetAttribute(encode_simple_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     encode_simple_kernel<__nv_bfloat16><<<grid, kEncThreads, smem, stream>>>(
-        (const __nv_bfloat16*)k_cache, ctx->P_hf, ctx->gram, ctx->unit_lens, codes, c.n_kv_heads, c.n_max, b, shared_sets,
+        (const __nv_bfloat16*)k_cache, ctx->P_hf, ctx->gram, ctx->unit_lens, codes, c.n_kv_heads, c.n_max, ctx->row_stride, b, shared_sets,
         c.residual_correction);
   } else {
     e = cudaFuncSetAttribute(encode_simple_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     encode_simple_kernel<float><<<grid, kEncThreads, smem, stream>>>(
-        (const float*)k_cache, ctx->P_hf, ctx->gram, ctx->unit_lens, codes, c.n_kv_heads, c.n_max, b, shared_sets,
+        (const float*)k_cache, ctx->P_hf, ctx->gram, ctx->unit_lens, codes, c.n_kv_heads, c.n_max, ctx->row_stride, b, shared_sets,
         c.residual_correction);
   }
   ctx->launches += 1;
@@ -328,14 +328,15 @@ cudaError_t bpc_launch_append(bpc_ctx* ctx, const void* k_new, const void* v_new
     if (e != cudaSuccess) return e;
     append_kernel<__nv_bfloat16><<<ctx->units, kAppThreads, smem, stream>>>(
         (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, codes,
-        (const __nv_bfloat16*)ctx->P_h, ctx->gram, ctx->unit_lens, ctx->dev_err, c.n_kv_heads, c.n_max, b, shared_sets,
+        (const __nv_bfloat16*)ctx->P_h, ctx->gram, ctx->unit_lens, ctx->dev_err, c.n_kv_heads, c.n_max, ctx->row_stride, b, shared_sets,
         c.residual_correction);
   } else {
     e = cudaFuncSetAttribute(append_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     append_kernel<float><<<ctx->units, kAppThreads, smem, stream>>>(
         (const float*)k_new, (const float*)v_new, (float*)k_cache, (float*)v_cache, codes, (const float*)ctx->P_h,
-        ctx->gram, ctx->unit_lens, ctx->dev_err, c.n_kv_heads, c.n_max, b, shared_sets, c.residual_correction);
+        ctx->gram, ctx->unit_lens, ctx->dev_err, c.n_kv_heads, c.n_max, ctx->row_stride, b, shared_sets,
+        c.residual_correction);
   }
   ctx->launches += 1;
   return cudaGetLastError();
@@ -370,10 +371,10 @@ cudaError_t bpc_launch_fit(bpc_ctx* ctx, const void* k_cache, const float* v_sta
   for (int it = 0; it < c.code_bits; ++it) {
     if (c.kv_dtype == BPC_BF16)
       fit_pass_kernel<__nv_bfloat16><<<grid, kFitThreads, 0, stream>>>((const __nv_bfloat16*)k_cache, R, usign, hfit, v_star, ctx->P,
-                                                                        partials, ctx->unit_lens, c.n_max, c.code_bits, it, bpu);
+                                                                        partials, ctx->unit_lens, c.n_max, ctx->row_stride, c.code_bits, it, bpu);
     else
       fit_pass_kernel<float><<<grid, kFitThreads, 0, stream>>>((const float*)k_cache, R, usign, hfit, v_star, ctx->P, partials,
-                                                               ctx->unit_lens, c.n_max, c.code_bits, it, bpu);
+                                                               ctx->unit_lens, c.n_max, ctx->row_stride, c.code_bits, it, bpu);
     fit_reduce_kernel<<<ctx->units, BPC_D, 0, stream>>>(partials, ctx->P, ctx->unit_lens, c.n_max, c.code_bits, it, bpu);
     *launches += 2;
   }

@@ -39,15 +39,21 @@ class Session:
     """A workload on the GPU with its library context, fitted and encoded."""
 
     def __init__(self, spec: WorkloadSpec, gen_device: str = "cpu", salt: int = 0, cluster_size: int = 0,
-                 extra_rows=None):
+                 extra_rows=None, interleaved: bool = False):
         self.spec = spec
         self.w = Workload(spec, device=gen_device, extra_rows=extra_rows, salt=salt)
         dev = "cuda"
-        self.k_cache = self.w.k_cache.to(dev)
-        self.v_cache = self.w.v_cache.to(dev)
+        if interleaved:       # K and V rows of a token adjacent in one buffer; the caches are strided views of it
+            self.kv_buf, self.k_cache, self.v_cache = B.interleaved_kv(spec.batch, spec.n_kv_heads, self.w.n_max,
+                                                                        spec.head_dim, spec.torch_dtype)
+            self.k_cache.copy_(self.w.k_cache)
+            self.v_cache.copy_(self.w.v_cache)
+        else:
+            self.k_cache = self.w.k_cache.to(dev)
+            self.v_cache = self.w.v_cache.to(dev)
         self.v_star = self.w.v_star.to(dev)
         self.cfg = B.make_config(spec.batch, spec.n_q_heads, spec.n_kv_heads, self.w.n_max, spec.code_bits,
-                                 spec.torch_dtype)
+                                 spec.torch_dtype, kv_row_stride=2 * spec.head_dim if interleaved else 0)
         self.ctx = B.Context(self.cfg)
         if cluster_size:
             self.ctx.set_cluster_size(cluster_size)

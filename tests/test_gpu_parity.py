@@ -63,6 +63,21 @@ def test_code_lengths_and_group_sizes(bits, group, dtype):
     print(rep)
 
 
+@pytest.mark.parametrize("dtype,bits", [("bf16", 128), ("f32", 64)])
+def test_interleaved_kv_layout(dtype, bits):
+    """K and V rows of a token adjacent in one buffer (row stride 2*head_dim): same results as separate arrays."""
+    H = _harness()
+    spec = CONFIGS[1].scaled(n_ctx=4500, n_kv_heads=2, n_q_heads=8, steps=2, dtype=dtype, code_bits=bits)
+    sess = H.Session(spec, interleaved=True)
+    rep = {}
+    sess.fit(); H.check_fit(sess, [1], rep)
+    sess.encode(); H.check_encode(sess, [0, 1], rep)
+    _decode_loop(sess, 2, [0, 1], rep, H)
+    ref = H.Session(spec)
+    ref.fit(); ref.encode()
+    assert torch.equal(ref.codes[:, :, :4500], sess.codes[:, :, :4500])
+
+
 @pytest.mark.parametrize("ppm,count", [(1000000, 0), (10000, 0), (50000, 0), (0, 1), (0, 1024), (1, 0)])
 def test_budgets(ppm, count):
     """budget = n (dense softmax attention), 1 %, 5 %, a single key, a fixed count, and the smallest fraction."""
