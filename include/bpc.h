@@ -48,7 +48,8 @@ typedef enum {
   BPC_ERR_CAPACITY = 3,      /* a sequence would exceed n_max; nothing was written */
   BPC_ERR_NOT_FITTED = 4,    /* a call needs the projection before bpc_fit / bpc_set_projection */
   BPC_ERR_CUDA = 5,          /* a CUDA runtime call failed (see bpc_last_cuda_error) */
-  BPC_ERR_DEVICE = 6         /* a kernel reported an internal error through the device error word */
+  BPC_ERR_DEVICE = 6,        /* a kernel reported an internal error through the device error word */
+  BPC_ERR_SCRATCH_LIMIT = 7  /* bpc_decode_attn_static only: the shape needs more than the built-in scratch array */
 } bpc_status;
 
 typedef enum { BPC_BF16 = 0, BPC_F32 = 1 } bpc_dtype;
@@ -131,6 +132,36 @@ bpc_status bpc_append(bpc_ctx* ctx, const void* k_new, const void* v_new,
 bpc_status bpc_decode_attn(bpc_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
                            const uint64_t* codes, int32_t budget_ppm, int32_t budget_count,
                            float* out, int32_t* sel_idx, void* stream);
+
+/* The same decode step for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this is a property of the library, not of the method.)
+ *
+ * Who needs it: a plug-in inside a serving process whose memory pool has already taken the whole device, or
+ * code that may run while another thread has a stream capture open; neither can call cudaMalloc, so neither
+ * can use bpc_create.  This call takes no context, makes no cudaMalloc / cudaFree / allocating library call,
+ * and keeps the two things the regular call gets from its context - the selected-index list and the device
+ * error word - in a fixed array compiled into the library (4 MiB + 256 B, held by every device that loads the
+ * library until the process exits).
+ *
+ * The caller passes every input and the output: cfg (host; same meaning and limits as for bpc_create, Hamming
+ * scores only), q, k_cache, v_cache, codes, out as for bpc_decode_attn; P_hash = the hash projection rounded to
+ * the cache dtype, [hash_sets][code_bits][head_dim] kv_dtype (what bpc_get_projection reports as P_hash_out,
+ * stored in kv_dtype); unit_lens = number of cached keys per unit, [batch*n_kv_heads] int32 on the device.
+ *
+ * Limits and hazards
+ *   - batch * n_kv_heads * n_max must not exceed bpc_static_scratch_entries() (1 Mi index entries); larger
+ *     shapes return BPC_ERR_SCRATCH_LIMIT and launch nothing.
+ *   - All calls on one device share the array.  Calls that can overlap on the GPU (different streams without
+ *     an ordering between them) race on it; order them on one stream or with events.
+ *   - The array keeps the previous call's contents.  The call clears the error word itself (asynchronously, on
+ *     `stream`) before launching; the index list needs no clearing because each unit's entries are written
+ *     before they are read.
+ *   - The first call on each device looks up the array's device address and sets the kernel's launch
+ *     attributes; make that first call outside any stream capture. */
+bpc_status bpc_decode_attn_static(const bpc_config* host_cfg, const void* q, const void* k_cache, const void* v_cache,
+                                  const uint64_t* codes, const void* P_hash, const int32_t* unit_lens,
+                                  int32_t budget_ppm, int32_t budget_count, float* out, void* stream);
+size_t     bpc_static_scratch_entries(void);
 
 /* Parity aids.  When set (non-NULL), the next bpc_decode_attn calls also write the integer hash
  * score of every cached key (scores [units][n_max] int32) and the collapsed integer query weights

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libbpc.so")
 
 BPC_OK = 0
 STATUS_NAMES = {0: "BPC_OK", 1: "BPC_ERR_INVALID_ARG", 2: "BPC_ERR_UNSUPPORTED", 3: "BPC_ERR_CAPACITY",
-                4: "BPC_ERR_NOT_FITTED", 5: "BPC_ERR_CUDA", 6: "BPC_ERR_DEVICE"}
+                4: "BPC_ERR_NOT_FITTED", 5: "BPC_ERR_CUDA", 6: "BPC_ERR_DEVICE", 7: "BPC_ERR_SCRATCH_LIMIT"}
 BPC_BF16, BPC_F32 = 0, 1
 BPC_SCORE_HAMMING, BPC_SCORE_WEIGHTED7 = 0, 1
 
@@ -56,6 +56,8 @@ def _load() -> ctypes.CDLL:
         "bpc_encode_keys": (i32, [vp, vp, vp, vp]),
         "bpc_append": (i32, [vp, vp, vp, vp, vp, vp, vp]),
         "bpc_decode_attn": (i32, [vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]),
+        "bpc_decode_attn_static": (i32, [cfgp, vp, vp, vp, vp, vp, vp, i32, i32, vp, vp]),
+        "bpc_static_scratch_entries": (sz, []),
         "bpc_debug_set_buffers": (i32, [vp, vp, vp]),
         "bpc_debug_set_phase_timer": (i32, [vp, vp]),
         "bpc_set_cluster_size": (i32, [vp, i32]),
@@ -76,7 +78,8 @@ lib = _load()
 EXPORTS = ["bpc_create", "bpc_destroy", "bpc_codes_bytes", "bpc_fit_workspace_bytes", "bpc_fit_codes_offset",
            "bpc_max_context",
            "bpc_set_seq_lens", "bpc_get_seq_lens", "bpc_fit", "bpc_set_projection", "bpc_get_projection",
-           "bpc_encode_keys", "bpc_append", "bpc_decode_attn", "bpc_debug_set_buffers", "bpc_debug_set_phase_timer",
+           "bpc_encode_keys", "bpc_append", "bpc_decode_attn", "bpc_decode_attn_static", "bpc_static_scratch_entries",
+           "bpc_debug_set_buffers", "bpc_debug_set_phase_timer",
            "bpc_set_cluster_size",
            "bpc_get_cluster_size", "bpc_last_device_error", "bpc_last_cuda_error", "bpc_launch_count", "bpc_version"]
 
@@ -233,6 +236,19 @@ def bpc_decode_attn(ctx: Context, q, k_cache, v_cache, codes, budget) -> torch.T
     if isinstance(budget, float):
         return ctx.decode_attn(q, k_cache, v_cache, codes, budget_ppm=int(round(budget * 1e6)))
     return ctx.decode_attn(q, k_cache, v_cache, codes, budget_ppm=0, budget_count=int(budget))
+
+
+def bpc_decode_attn_static(cfg: bpc_config, q, k_cache, v_cache, codes, P_hash, unit_lens, budget_ppm: int = 20000,
+                           budget_count: int = 0, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Decode step without a context and without any allocation inside the library (see bpc.h).  P_hash is the hash
+    projection in the cache dtype, unit_lens an int32 device tensor with one length per (sequence, KV head)."""
+    if out is None:
+        out = torch.empty(cfg.batch, cfg.n_q_heads, cfg.head_dim, dtype=torch.float32, device=q.device)
+    assert unit_lens.dtype == torch.int32
+    _check(lib.bpc_decode_attn_static(ctypes.byref(cfg), _ptr(q), _cache_ptr(k_cache), _cache_ptr(v_cache), _ptr(codes),
+                                      _ptr(P_hash), _ptr(unit_lens), budget_ppm, budget_count, _ptr(out), _stream()),
+           "bpc_decode_attn_static")
+    return out
 
 
 def bpc_fit(ctx: Context, k_cache, v_star, workspace=None) -> None:
