@@ -35,6 +35,7 @@ import numpy as np
 import torch
 
 from paper_2608_04405_b200.inputs import CONFIGS, Workload, algorithmic_bytes_per_step
+from paper_2608_04405_b200 import replicas
 
 METRIC = "sparse decode-attn tokens/s (one attention layer, append + decode_attn per step)"
 UNIT = "tokens/s"
@@ -191,17 +192,13 @@ def run_ours(args):
             dist.barrier()
 
     def max_over_ranks(x: float) -> float:
-        if not use_dist:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return replicas.max_over_ranks(x, device="cuda")
 
     spec = CONFIGS[args.workload]
     K, W, L = args.steps, args.warmup, args.layers
     extra = ((K + W) // L + 2) * 2 + 64
     fit_ws = [None]
-    layers = [Layer(spec, salt=100 * rank + i, extra_rows=extra, B=B, fit_ws=fit_ws, interleaved=not args.separate_kv)
+    layers = [Layer(spec, salt=replicas.replica_salt(rank, i), extra_rows=extra, B=B, fit_ws=fit_ws, interleaved=not args.separate_kv)
               for i in range(L)]
     fit_ws[0] = None
     torch.cuda.empty_cache()
@@ -311,7 +308,7 @@ def run_ours(args):
     fit_ms = statistics.median(ly.fit_ms for ly in layers)
     enc_flops = 2.0 * n_keys * spec.head_dim * spec.code_bits
     result = {
-        "metric": METRIC, "value": world * spec.batch / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": replicas.whole_job_tokens_per_s(spec.batch, world, ms_step), "unit": UNIT, "n_gpus": world,
         "steps": K, "warmup": W, "ms_per_step": ms_step, "us_per_step": ms_step * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": spec.name, "batch": spec.batch, "n_q_heads": spec.n_q_heads, "n_kv_heads": spec.n_kv_heads,
