@@ -133,6 +133,15 @@ bpc_status bpc_decode_attn(bpc_ctx* ctx, const void* q, const void* k_cache, con
                            const uint64_t* codes, int32_t budget_ppm, int32_t budget_count,
                            float* out, int32_t* sel_idx, void* stream);
 
+/* bpc_append followed by bpc_decode_attn as ONE launch (the two calls of a decode step, fused): the block of
+ * each unit's cluster that owns the new position writes the (k, v) rows, codes the new key in one of its warps
+ * while the other warps scan the old codes, scores it, and advances the length; the step's selection and
+ * attention then see n+1 keys exactly as after a separate bpc_append.  Same arguments, layouts, limits and
+ * errors as the two calls it replaces (BPC_ERR_CAPACITY, with nothing launched, if any sequence is at n_max). */
+bpc_status bpc_append_decode_attn(bpc_ctx* ctx, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                                  uint64_t* codes, const void* q, int32_t budget_ppm, int32_t budget_count,
+                                  float* out, int32_t* sel_idx, void* stream);
+
 /* The same decode step for callers that cannot allocate device memory.  (The paper has no counterpart:
  * this is a property of the library, not of the method.)
  *

@@ -56,6 +56,7 @@ def _load() -> ctypes.CDLL:
         "bpc_encode_keys": (i32, [vp, vp, vp, vp]),
         "bpc_append": (i32, [vp, vp, vp, vp, vp, vp, vp]),
         "bpc_decode_attn": (i32, [vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]),
+        "bpc_append_decode_attn": (i32, [vp, vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]),
         "bpc_decode_attn_static": (i32, [cfgp, vp, vp, vp, vp, vp, vp, i32, i32, vp, vp]),
         "bpc_static_scratch_entries": (sz, []),
         "bpc_debug_set_buffers": (i32, [vp, vp, vp]),
@@ -78,7 +79,7 @@ lib = _load()
 EXPORTS = ["bpc_create", "bpc_destroy", "bpc_codes_bytes", "bpc_fit_workspace_bytes", "bpc_fit_codes_offset",
            "bpc_max_context",
            "bpc_set_seq_lens", "bpc_get_seq_lens", "bpc_fit", "bpc_set_projection", "bpc_get_projection",
-           "bpc_encode_keys", "bpc_append", "bpc_decode_attn", "bpc_decode_attn_static", "bpc_static_scratch_entries",
+           "bpc_encode_keys", "bpc_append", "bpc_decode_attn", "bpc_append_decode_attn", "bpc_decode_attn_static", "bpc_static_scratch_entries",
            "bpc_debug_set_buffers", "bpc_debug_set_phase_timer",
            "bpc_set_cluster_size",
            "bpc_get_cluster_size", "bpc_last_device_error", "bpc_last_cuda_error", "bpc_launch_count", "bpc_version"]
@@ -208,6 +209,16 @@ class Context:
             out = torch.empty(c.batch, c.n_q_heads, c.head_dim, dtype=torch.float32, device=q.device)
         _check(lib.bpc_decode_attn(self._h, _ptr(q), _cache_ptr(k_cache), _cache_ptr(v_cache), _ptr(codes), budget_ppm, budget_count,
                                    _ptr(out), _ptr(sel_idx), _stream()), "bpc_decode_attn")
+        return out
+
+    def append_decode_attn(self, k_new, v_new, k_cache, v_cache, codes, q, budget_ppm: int = 20000, budget_count: int = 0,
+                           out: Optional[torch.Tensor] = None, sel_idx: Optional[torch.Tensor] = None) -> torch.Tensor:
+        c = self.cfg
+        if out is None:
+            out = torch.empty(c.batch, c.n_q_heads, c.head_dim, dtype=torch.float32, device=q.device)
+        _check(lib.bpc_append_decode_attn(self._h, _ptr(k_new), _ptr(v_new), _cache_ptr(k_cache), _cache_ptr(v_cache),
+                                          _ptr(codes), _ptr(q), budget_ppm, budget_count, _ptr(out), _ptr(sel_idx), _stream()),
+               "bpc_append_decode_attn")
         return out
 
     # -- parity aids and diagnostics

@@ -255,8 +255,10 @@ bpc_status bpc_append(bpc_ctx* ctx, const void* k_new, const void* v_new, void* 
   return BPC_OK;
 }
 
-bpc_status bpc_decode_attn(bpc_ctx* ctx, const void* q, const void* k_cache, const void* v_cache, const uint64_t* codes,
-                           int32_t budget_ppm, int32_t budget_count, float* out, int32_t* sel_idx, void* stream) {
+static bpc_status decode_common(bpc_ctx* ctx, const void* k_new, const void* v_new, void* k_cache_w, void* v_cache_w,
+                                uint64_t* codes_w, const void* q, const void* k_cache, const void* v_cache,
+                                const uint64_t* codes, int32_t budget_ppm, int32_t budget_count, float* out,
+                                int32_t* sel_idx, void* stream) {
   if (ctx == nullptr || q == nullptr || k_cache == nullptr || v_cache == nullptr || codes == nullptr || out == nullptr)
     return BPC_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(codes) || !aligned16(out))
@@ -272,6 +274,8 @@ bpc_status bpc_decode_attn(bpc_ctx* ctx, const void* q, const void* k_cache, con
   memset(&p, 0, sizeof(p));
   p.q = q; p.k_cache = k_cache; p.v_cache = v_cache; p.codes = codes; p.P_h = ctx->P_h;
   p.unit_lens = ctx->unit_lens; p.out = out;
+  p.k_new = k_new; p.v_new = v_new; p.k_cache_w = k_cache_w; p.v_cache_w = v_cache_w; p.codes_w = codes_w;
+  p.unit_lens_w = ctx->unit_lens; p.gram = ctx->gram; p.residual_correction = c.residual_correction;
   p.sel = sel_idx != nullptr ? sel_idx : ctx->sel_scratch;
   p.dbg_scores = ctx->dbg_scores; p.dbg_qweights = ctx->dbg_qweights; p.dbg_times = ctx->dbg_times;
   p.err = ctx->dev_err;
@@ -286,6 +290,27 @@ bpc_status bpc_decode_attn(bpc_ctx* ctx, const void* q, const void* k_cache, con
                              : bpc_launch_decode_f32(ctx, p, (cudaStream_t)stream);
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   ctx->launches += 1;
+  return BPC_OK;
+}
+
+bpc_status bpc_decode_attn(bpc_ctx* ctx, const void* q, const void* k_cache, const void* v_cache, const uint64_t* codes,
+                           int32_t budget_ppm, int32_t budget_count, float* out, int32_t* sel_idx, void* stream) {
+  return decode_common(ctx, nullptr, nullptr, nullptr, nullptr, nullptr, q, k_cache, v_cache, codes, budget_ppm,
+                       budget_count, out, sel_idx, stream);
+}
+
+bpc_status bpc_append_decode_attn(bpc_ctx* ctx, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                                  uint64_t* codes, const void* q, int32_t budget_ppm, int32_t budget_count, float* out,
+                                  int32_t* sel_idx, void* stream) {
+  if (ctx == nullptr || k_new == nullptr || v_new == nullptr || k_cache == nullptr || v_cache == nullptr || codes == nullptr)
+    return BPC_ERR_INVALID_ARG;
+  if (!aligned16(k_new) || !aligned16(v_new)) return BPC_ERR_INVALID_ARG;
+  for (int i = 0; i < ctx->cfg.batch; ++i)
+    if (ctx->host_lens[i] >= ctx->cfg.n_max) return BPC_ERR_CAPACITY;
+  bpc_status s = decode_common(ctx, k_new, v_new, k_cache, v_cache, codes, q, k_cache, v_cache, codes, budget_ppm,
+                               budget_count, out, sel_idx, stream);
+  if (s != BPC_OK) return s;
+  for (int i = 0; i < ctx->cfg.batch; ++i) ctx->host_lens[i] += 1;
   return BPC_OK;
 }
 

@@ -49,6 +49,15 @@ struct DecodeParams {
   const uint64_t* codes;
   const void* P_h;
   const int32_t* unit_lens;
+  // fused cache write (all null / unused when the launch only decodes)
+  const void* k_new;
+  const void* v_new;
+  void* k_cache_w;
+  void* v_cache_w;
+  uint64_t* codes_w;
+  int32_t* unit_lens_w;
+  const float* gram;
+  int residual_correction;
   float* out;
   int32_t* sel;              // [units][n_max]
   int32_t* dbg_scores;

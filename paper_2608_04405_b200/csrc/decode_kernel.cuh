@@ -46,6 +46,7 @@ struct SmallState {
   uint32_t wscan[32];
   double pmax[BPC_MAX_GROUP];
   int T, cnt_gt, my_take, my_base, rsum, pad[3];
+  uint32_t newcode[8];                   // code of the key appended by this launch
 };
 
 template <typename KV> struct IsBf16 { static constexpr bool value = false; };
@@ -66,16 +67,17 @@ struct DecodeSmem {
   static constexpr int kStageBytes = kTileRows * 2 * kRowBytes;
   __host__ __device__ static constexpr size_t a16(size_t x) { return (x + 15) & ~(size_t)15; }
   __host__ __device__ static constexpr size_t part_bytes() { return (size_t)NW * GP * (BPC_D + 2) * sizeof(acc_t); }
-  __host__ __device__ static constexpr size_t hashpart_bytes() { return (size_t)NT * GP * 8; }
+  static constexpr int GV = GP + 1;      // vectors projected in phase 0: the group's queries and the appended key
+  __host__ __device__ static constexpr size_t hashpart_bytes() { return (size_t)NT * GV * 8; }
 
   size_t off_hist, off_tot, off_qf, off_pd, off_idx, off_cta, off_small, off_union, total;
   __host__ __device__ DecodeSmem(int chunk_cap, int nbins, int stages) {
     const size_t nb = a16((size_t)nbins * 4);
     off_hist = 0;
     off_tot = off_hist + nb;
-    off_qf = off_tot + nb;                                           // float[GP][128]
-    off_pd = off_qf + (size_t)GP * BPC_D * 4;                        // double[GP][B]
-    off_idx = off_pd + (size_t)GP * B * 8;                           // int32[kIdxTile]
+    off_qf = off_tot + nb;                                           // float[GP+1][128]
+    off_pd = off_qf + (size_t)GV * BPC_D * 4;                        // double[GP+1][B]
+    off_idx = off_pd + (size_t)GV * B * 8;                           // int32[kIdxTile]
     off_cta = off_idx + kIdxTile * 4;                                // acc_t[GP][130]
     off_small = a16(off_cta + (size_t)GP * (BPC_D + 2) * sizeof(acc_t));
     off_union = a16(off_small + sizeof(SmallState));
@@ -226,6 +228,13 @@ bpc_decode_kernel(const DecodeParams p) {
 
   int n = p.unit_lens[unit];
   n = max(0, min(n, p.n_max));
+  // Fused cache write: this launch also appends one (k, v) row per unit at position n, codes it and counts it.
+  bool fused = p.k_new != nullptr;
+  if (fused && n >= p.n_max) {                               // full: nothing is written, the step runs on n keys
+    if (tid == 0 && rank == 0) atomicOr(p.err, BPC_DEVERR_APPEND_CAP);
+    fused = false;
+  }
+  if (fused) n += 1;
   long long kk = p.budget_count > 0 ? (long long)p.budget_count
                                     : ((long long)n * (long long)p.budget_ppm + 999999LL) / 1000000LL;
   if (kk < 0) kk = 0;
@@ -260,6 +269,8 @@ bpc_decode_kernel(const DecodeParams p) {
   uint16_t* sc = reinterpret_cast<uint16_t*>(uni);
 #define BPC_STAMP(i) do { if (p.dbg_times != nullptr && tid == 0) p.dbg_times[(size_t)blockIdx.x * 16 + (i)] = global_timer_ns(); } while (0)
   BPC_STAMP(0);
+  // the block whose key range holds the appended key (index n-1) does the append work in its last warp
+  const bool appender = fused && rank == (n - 1) / chunk;
 
   // ------------------------------------------------------------------ phase 0: query hash
   // p[g][j] = P_h[j] . q_g.  Thread (part, j) covers a slice of the 128 channels of row j: products are
@@ -267,6 +278,8 @@ bpc_decode_kernel(const DecodeParams p) {
   // slices are then added in fp64 in a fixed order.  Every block of the cluster gets identical bits.
   const KV* qg = reinterpret_cast<const KV*>(p.q) + ((size_t)seq * p.n_kv_heads + kvh) * (size_t)G * BPC_D;
   for (int i = tid; i < GP * BPC_D; i += NT) qf_s[i] = (i >> 7) < G ? to_float(qg[i]) : 0.f;
+  if (tid < BPC_D)                                           // slot GP: the appended key (its decision values P_h k)
+    qf_s[GP * BPC_D + tid] = appender ? to_float(reinterpret_cast<const KV*>(p.k_new)[(size_t)unit * BPC_D + tid]) : 0.f;
   for (int i = tid; i < nbins; i += NT) hist[i] = 0u;
   if (tid < BPC_MAX_CLUSTER) { st->gt[tid] = 0u; st->eq[tid] = 0u; }
   if (tid == 0) { st->rsum = 0; st->T = 0; st->cnt_gt = 0; }
@@ -276,9 +289,10 @@ bpc_decode_kernel(const DecodeParams p) {
     constexpr int DS = BPC_D / PARTS;              // channels per slice (a multiple of 8)
     const int j = tid % B, part = tid / B;
     const KV* row = reinterpret_cast<const KV*>(p.P_h) + ((size_t)(p.shared_sets ? kvh : unit) * B + j) * BPC_D + part * DS;
-    double acc[GP];
+    constexpr int GV = L::GV;
+    double acc[GV];
 #pragma unroll
-    for (int g = 0; g < GP; ++g) acc[g] = 0.0;
+    for (int g = 0; g < GV; ++g) acc[g] = 0.0;
 #pragma unroll 2
     for (int c0 = 0; c0 < DS; c0 += 8) {
       float pv[8];
@@ -292,7 +306,7 @@ bpc_decode_kernel(const DecodeParams p) {
         pv[0] = w0.x; pv[1] = w0.y; pv[2] = w0.z; pv[3] = w0.w; pv[4] = w1.x; pv[5] = w1.y; pv[6] = w1.z; pv[7] = w1.w;
       }
 #pragma unroll
-      for (int g = 0; g < GP; ++g) {
+      for (int g = 0; g < GV; ++g) {
         const float4 q0 = *reinterpret_cast<const float4*>(qf_s + g * BPC_D + part * DS + c0);
         const float4 q1 = *reinterpret_cast<const float4*>(qf_s + g * BPC_D + part * DS + c0 + 4);
         float s0 = pv[0] * q0.x, s1 = pv[1] * q0.y;
@@ -302,14 +316,14 @@ bpc_decode_kernel(const DecodeParams p) {
         acc[g] += (double)s0 + (double)s1;
       }
     }
-    double* hp = reinterpret_cast<double*>(uni);   // [PARTS][GP][B]
+    double* hp = reinterpret_cast<double*>(uni);   // [PARTS][GV][B]
 #pragma unroll
-    for (int g = 0; g < GP; ++g) hp[((size_t)part * GP + g) * B + j] = acc[g];
+    for (int g = 0; g < GV; ++g) hp[((size_t)part * GV + g) * B + j] = acc[g];
     __syncthreads();
-    for (int i = tid; i < GP * B; i += NT) {       // i = g * B + j
+    for (int i = tid; i < GV * B; i += NT) {       // i = g * B + j
       double s = 0.0;
 #pragma unroll
-      for (int pt = 0; pt < PARTS; ++pt) s += hp[(size_t)pt * GP * B + i];
+      for (int pt = 0; pt < PARTS; ++pt) s += hp[(size_t)pt * GV * B + i];
       pd[i] = s;
     }
   }
@@ -355,7 +369,11 @@ bpc_decode_kernel(const DecodeParams p) {
   BPC_STAMP(1);
   // ------------------------------------------------------------------ phase 1: scan
   const int c0 = min(n, rank * chunk), c1 = min(n, c0 + chunk);
-  {
+  // In the appending block the last warp codes the new key while the other warps scan; the new key's code is
+  // not in memory yet, so the scan stops one key short and the key is scored separately below.
+  const int nts = appender ? NT - 32 : NT;
+  const int c1s = appender ? c1 - 1 : c1;
+  if (tid < nts) {
     uint32_t sg[W32], mk[NP][W32];
 #pragma unroll
     for (int w = 0; w < W32; ++w) {
@@ -381,13 +399,13 @@ bpc_decode_kernel(const DecodeParams p) {
     };
     auto load_batch = [&](uint32_t (&h)[U][W32], int base) {
 #pragma unroll
-      for (int u = 0; u < U; ++u) load_code(h[u], base + u * NT + tid);
+      for (int u = 0; u < U; ++u) load_code(h[u], base + u * nts + tid);
     };
     auto score_batch = [&](const uint32_t (&h)[U][W32], int base) {
 #pragma unroll
       for (int u = 0; u < U; ++u) {
         const int key = score_key<W32, NP>(h[u], sg, mk);
-        sc[score_slot(base - c0 + u * NT + tid)] = (uint16_t)key;
+        sc[score_slot(base - c0 + u * nts + tid)] = (uint16_t)key;
         atomicAdd(&hist[key], 1u);
       }
     };
@@ -396,17 +414,17 @@ bpc_decode_kernel(const DecodeParams p) {
       // Full batches without bounds checks, software-pipelined over two register buffers so that the
       // loads of the next batch are in flight while the current one is scored (a warp's 32 keys share
       // one score segment).
-      constexpr int STEP = NT * U;
-      if (i0 + STEP <= c1) {
+      const int STEP = nts * U;
+      if (i0 + STEP <= c1s) {
         uint32_t ha[U][W32], hb[U][W32];
         load_batch(ha, i0);
         for (;;) {
-          const bool more_b = i0 + 2 * STEP <= c1;
+          const bool more_b = i0 + 2 * STEP <= c1s;
           if (more_b) load_batch(hb, i0 + STEP);
           score_batch(ha, i0);
           i0 += STEP;
           if (!more_b) break;
-          const bool more_a = i0 + 2 * STEP <= c1;
+          const bool more_a = i0 + 2 * STEP <= c1s;
           if (more_a) load_batch(ha, i0 + STEP);
           score_batch(hb, i0);
           i0 += STEP;
@@ -414,9 +432,9 @@ bpc_decode_kernel(const DecodeParams p) {
         }
       }
     }
-    for (; i0 < c1; i0 += NT) {                             // tail (and the whole range when scores are exported)
+    for (; i0 < c1s; i0 += nts) {                           // tail (and the whole range when scores are exported)
       const int i = i0 + tid;
-      if (i < c1) {
+      if (i < c1s) {
         uint32_t h[W32];
         load_code(h, i);
         const int key = score_key<W32, NP>(h, sg, mk);
@@ -425,12 +443,86 @@ bpc_decode_kernel(const DecodeParams p) {
         if (dbg != nullptr) dbg[i] = ((2 * key) << cs) - rfull;
       }
     }
+  } else {
+    // ---- appending warp (Algorithm 2 on the new key, Gram form): cache rows, sign sweep, code words.
+    // Lane l holds the decision values of bits l, 32+l, ...; bit i is decided by a shuffle from its owner
+    // lane and every later column is corrected with G[i][.], read from global memory two steps ahead.
+    const size_t rstride_e = (size_t)p.row_stride;
+    const KV* kn = reinterpret_cast<const KV*>(p.k_new) + (size_t)unit * BPC_D;
+    const KV* vn = reinterpret_cast<const KV*>(p.v_new) + (size_t)unit * BPC_D;
+    KV* krow = reinterpret_cast<KV*>(p.k_cache_w) + ((size_t)unit * p.n_max + (n - 1)) * rstride_e;
+    KV* vrow = reinterpret_cast<KV*>(p.v_cache_w) + ((size_t)unit * p.n_max + (n - 1)) * rstride_e;
+    constexpr int CPL = ROWB / 16 / 16;                      // 16-byte chunks per lane and row (1 bf16, 2 fp32)
+#pragma unroll
+    for (int c = 0; c < CPL; ++c) {
+      const int chn = (lane & 15) * CPL + c;
+      if (lane < 16) reinterpret_cast<uint4*>(krow)[chn] = reinterpret_cast<const uint4*>(kn)[chn];
+      else           reinterpret_cast<uint4*>(vrow)[chn] = reinterpret_cast<const uint4*>(vn)[chn];
+    }
+    constexpr int NB = W32;                                  // 32-bit column blocks
+    float t[NB];
+#pragma unroll
+    for (int c = 0; c < NB; ++c) t[c] = (float)pd[GP * B + 32 * c + lane];
+    const float* Gs = p.gram + (size_t)(p.shared_sets ? kvh : unit) * B * B;
+    const bool rc = p.residual_correction != 0;
+    uint32_t* code_dst = reinterpret_cast<uint32_t*>(p.codes_w) + ((size_t)unit * p.n_max + (n - 1)) * W32;
+    constexpr int PF = 4;                                    // Gram rows per prefetch group
+#pragma unroll
+    for (int bi = 0; bi < NB; ++bi) {
+      uint32_t wbits = 0;
+      float ga[PF][NB], gb[PF][NB];
+      auto fetch = [&](float (&gq)[PF][NB], int ii) {
+#pragma unroll
+        for (int r = 0; r < PF; ++r)
+#pragma unroll
+          for (int c = bi; c < NB; ++c) gq[r][c] = rc ? __ldg(Gs + (size_t)(32 * bi + ii + r) * B + 32 * c + lane) : 0.f;
+      };
+      auto sweep = [&](const float (&gq)[PF][NB], int ii) {
+#pragma unroll
+        for (int r = 0; r < PF; ++r) {
+          const int i = ii + r;
+          const float ti = __shfl_sync(0xffffffffu, t[bi], i);
+          const bool pos = ti >= 0.f;
+          wbits |= (pos ? 1u : 0u) << i;
+          const float u = pos ? 1.f : -1.f;
+          if (lane > i) t[bi] -= u * gq[r][bi];
+#pragma unroll
+          for (int c = bi + 1; c < NB; ++c) t[c] -= u * gq[r][c];
+        }
+      };
+      fetch(ga, 0);
+#pragma unroll 1
+      for (int ii = 0; ii < 32; ii += 2 * PF) {
+        fetch(gb, ii + PF);
+        sweep(ga, ii);
+        if (ii + 2 * PF < 32) fetch(ga, ii + 2 * PF);
+        sweep(gb, ii + PF);
+      }
+      if (lane == 0) { st->newcode[bi] = wbits; code_dst[bi] = wbits; }
+    }
+  }
+  if (appender) {
+    __syncthreads();                                         // the new code is in shared memory; the scan is done
+    if (tid == 0) {
+      uint32_t sg[W32], mk[NP][W32], h[W32];
+#pragma unroll
+      for (int w = 0; w < W32; ++w) {
+        sg[w] = st->signw[w]; h[w] = st->newcode[w];
+#pragma unroll
+        for (int pl = 0; pl < NP; ++pl) mk[pl][w] = st->mask[pl][w];
+      }
+      const int key = score_key<W32, NP>(h, sg, mk);
+      sc[score_slot(n - 1 - c0)] = (uint16_t)key;
+      atomicAdd(&hist[key], 1u);
+      if (p.dbg_scores != nullptr) p.dbg_scores[(size_t)unit * p.n_max + (n - 1)] = ((2 * key) << cs) - (st->rsum << cs);
+    }
   }
 
   BPC_STAMP(2);
   // ------------------------------------------------------------------ phase 2: threshold and ordered selection
   cluster.sync();                                            // every block's histogram is complete
   BPC_STAMP(8);
+  if (appender && tid == 0) p.unit_lens_w[unit] = n;         // every block of the cluster has read the old length
   // Total histogram through distributed shared memory.  With at most one bin per thread (the common case)
   // the per-block counts of that bin stay in registers and are reused for the per-block offsets below.
   const bool one_bin = nbins <= NT;

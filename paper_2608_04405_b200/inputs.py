@@ -169,7 +169,10 @@ class Workload:
             n = int(cur_lens[bi])
             for hq in range(s.n_q_heads):
                 h = hq // s.group
-                p = torch.randperm(n, generator=self._g, device=self.device)[: s.needles]
+                if n >= s.needles:
+                    p = torch.randperm(n, generator=self._g, device=self.device)[: s.needles]
+                else:                      # fewer cached keys than needles: draw with replacement
+                    p = torch.randint(0, n, (s.needles,), generator=self._g, device=self.device)
                 pos[bi, hq] = p
                 vec = kc[bi, h, p].float().sum(0)
                 vec = vec + 0.1 * torch.randn(s.head_dim, generator=self._g, device=self.device)

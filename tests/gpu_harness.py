@@ -150,8 +150,12 @@ def check_encode(sess: Session, units, report: dict, max_keys: int = 0, key_slic
             assert np.array_equal(ref, bits)
 
 
-def check_decode(sess: Session, q: torch.Tensor, units, report: dict, budget_ppm=None, budget_count=0):
-    """One decode step through the library, checked stage by stage for the given units."""
+def check_decode(sess: Session, q: torch.Tensor, units, report: dict, budget_ppm=None, budget_count=0, append=None):
+    """One decode step through the library, checked stage by stage for the given units.
+
+    With append=(k_new, v_new) the step goes through the fused bpc_append_decode_attn call; the cache rows, the
+    new key's code and the advanced lengths are checked as for bpc_append, and the plain decode call that
+    follows must reproduce the fused call's output bit for bit."""
     s = sess.spec
     ppm = s.budget_ppm if budget_ppm is None else budget_ppm
     n_max = sess.w.n_max
@@ -159,11 +163,23 @@ def check_decode(sess: Session, q: torch.Tensor, units, report: dict, budget_ppm
     dbg_qw = torch.zeros(sess.units, s.code_bits, dtype=torch.int32, device="cuda")
     sel = torch.full((sess.units, n_max), -1, dtype=torch.int32, device="cuda")
     sess.ctx.debug_set_buffers(dbg_scores, dbg_qw)
-    out = sess.ctx.decode_attn(q, sess.k_cache, sess.v_cache, sess.codes, budget_ppm=ppm, budget_count=budget_count,
-                               sel_idx=sel)
+    if append is None:
+        out = sess.ctx.decode_attn(q, sess.k_cache, sess.v_cache, sess.codes, budget_ppm=ppm, budget_count=budget_count,
+                                   sel_idx=sel)
+    else:
+        k_new, v_new = append
+        out = sess.ctx.append_decode_attn(k_new, v_new, sess.k_cache, sess.v_cache, sess.codes, q, budget_ppm=ppm,
+                                          budget_count=budget_count, sel_idx=sel)
     torch.cuda.synchronize()
     sess.ctx.debug_set_buffers(None, None)
     assert sess.ctx.last_device_error() == 0
+    if append is not None:
+        sess.lens = [n + 1 for n in sess.lens]
+        assert sess.ctx.get_seq_lens() == sess.lens
+        for u in units:
+            bi, h, n1 = sess.unit_views(u)
+            assert torch.equal(sess.k_cache[bi, h, n1 - 1], k_new[bi, h]) and torch.equal(sess.v_cache[bi, h, n1 - 1], v_new[bi, h])
+            check_encode(sess, [u], report, key_slice=(n1 - 1, n1))
     # a second call without the parity buffers and without a caller index list must give the same output
     out2 = sess.ctx.decode_attn(q, sess.k_cache, sess.v_cache, sess.codes, budget_ppm=ppm, budget_count=budget_count)
     torch.cuda.synchronize()

@@ -13,14 +13,21 @@ def _harness():
     return H
 
 
-def _decode_loop(sess, steps, units, report, H, check_every=1):
+def _decode_loop(sess, steps, units, report, H, check_every=1, fused="alternate"):
+    """Decode steps with a cache write each: even steps use bpc_append + bpc_decode_attn, odd steps the fused call."""
     for step in range(steps):
         k_new, v_new = sess.w.new_kv(sess.lens)
         k_new, v_new = k_new.cuda(), v_new.cuda()
-        H.check_append(sess, k_new, v_new, units, report)
-        q, _ = sess.w.queries(sess.lens, k_cache=sess.k_cache.to(sess.w.device))
-        if step % check_every == 0:
-            H.check_decode(sess, q.cuda(), units, report)
+        use_fused = fused is True or (fused == "alternate" and step % 2 == 1)
+        if use_fused:
+            # the query is planted on keys cached before this step, as for the two-call sequence
+            q, _ = sess.w.queries(sess.lens, k_cache=sess.k_cache.to(sess.w.device))
+            H.check_decode(sess, q.cuda(), units, report, append=(k_new, v_new))
+        else:
+            H.check_append(sess, k_new, v_new, units, report)
+            q, _ = sess.w.queries(sess.lens, k_cache=sess.k_cache.to(sess.w.device))
+            if step % check_every == 0:
+                H.check_decode(sess, q.cuda(), units, report)
 
 
 def test_cfg0_tiny_fp32_all_stages():
@@ -59,7 +66,7 @@ def test_code_lengths_and_group_sizes(bits, group, dtype):
     rep = {}
     sess.fit(); H.check_fit(sess, [1], rep)
     sess.encode(); H.check_encode(sess, [0, 1], rep)
-    _decode_loop(sess, 1, [0, 1], rep, H)
+    _decode_loop(sess, 2, [0, 1], rep, H)
     print(rep)
 
 
@@ -134,6 +141,24 @@ def test_shared_projection_per_kv_head():
     sess.encode(); H.check_encode(sess, [0, 1, 2, 3], rep)
     q, _ = sess.w.queries(sess.lens)
     H.check_decode(sess, q.cuda(), [0, 3], rep)
+
+
+def test_fused_append_decode_tiny_and_boundary_lengths():
+    """Fused cache write at lengths where the new key opens a new chunk / a new 32-key segment, and from n = 0."""
+    H = _harness()
+    for n0 in (0, 1, 63, 64, 255, 256, 2047):
+        spec = CONFIGS[1].scaled(n_ctx=max(n0, 1), n_kv_heads=2, n_q_heads=8, steps=3)
+        sess = H.Session(spec, extra_rows=64)
+        sess.fit(); sess.encode()            # projection fitted on max(n0, 1) keys
+        if n0 == 0:
+            sess.lens = [0]
+            sess.ctx.set_seq_lens(sess.lens)
+        rep = {}
+        for step in range(3):
+            k_new, v_new = sess.w.new_kv(sess.lens)
+            q, _ = sess.w.queries([max(1, n) for n in sess.lens], k_cache=sess.k_cache.to(sess.w.device))
+            H.check_decode(sess, q.cuda(), [0, 1], rep, append=(k_new.cuda(), v_new.cuda()), budget_ppm=200000)
+        assert sess.lens == [n0 + 3]
 
 
 def test_error_paths_do_not_launch():
