@@ -1,5 +1,6 @@
 // C-ABI entry points: argument validation, context life cycle, stream plumbing.
 #include <new>
+#include <stdlib.h>
 #include <string.h>
 #include "common.cuh"
 
@@ -109,6 +110,10 @@ bpc_status bpc_create(const bpc_config* cfg, bpc_ctx** out) {
   ctx->sm_scale_d = cfg->sm_scale == 0.f ? 0.08838834764831845 : (double)cfg->sm_scale;   // default 1/sqrt(128)
   ctx->units = cfg->batch * cfg->n_kv_heads;
   ctx->group = cfg->n_q_heads / cfg->n_kv_heads;
+  {
+    const char* no_pdl = getenv("BPC_NO_PDL");          // diagnostic switch: plain stream-ordered launches
+    ctx->use_pdl = !(no_pdl != nullptr && no_pdl[0] == '1');
+  }
   ctx->row_stride = cfg->kv_row_stride == 0 ? cfg->head_dim : cfg->kv_row_stride;
   cudaError_t e = cudaGetDevice(&ctx->device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device);

@@ -24,6 +24,7 @@ struct bpc_ctx {
   int max_cluster;          // largest cluster size the device schedules for the decode kernel
   int sm_count;
   bool fitted;
+  bool use_pdl;             // launch the decode kernel with programmatic stream serialization
   float* P;                 // [hash_sets][b][D] float
   void*  P_h;               // [hash_sets][b][D] cache dtype (the hash function)
   float* P_hf;              // P_h as float values

@@ -226,6 +226,12 @@ bpc_decode_kernel(const DecodeParams p) {
   const int kvh = unit % p.n_kv_heads;
   const int seq = unit / p.n_kv_heads;
 
+  // Programmatic dependent launch: when this grid was launched early (while its predecessor in the stream
+  // was still running) nothing of the predecessor's output may be read before this point; afterwards the
+  // successor's blocks may be scheduled as ours drain.  Both are no-ops for an ordinary launch.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
   int n = p.unit_lens[unit];
   n = max(0, min(n, p.n_max));
   // Fused cache write: this launch also appends one (k, v) row per unit at position n, codes it and counts it.
@@ -271,6 +277,22 @@ bpc_decode_kernel(const DecodeParams p) {
   BPC_STAMP(0);
   // the block whose key range holds the appended key (index n-1) does the append work in its last warp
   const bool appender = fused && rank == (n - 1) / chunk;
+
+  // The appending block stages the Gram matrix in the part of the shared-memory union that the score keys do
+  // not reach (free until the gather ring starts), so that the sequential sign decisions of Algorithm 2 cost a
+  // shuffle and a few FMAs each.  Shapes where it does not fit read it from global memory instead.
+  const float* gsm = nullptr;
+  if (appender && p.residual_correction != 0) {
+    const size_t union_bytes = plan.total - plan.off_union;
+    const size_t score_bytes = (size_t)((p.chunk_cap + kSegKeys - 1) / kSegKeys) * kSegSlots * 2;
+    if (score_bytes + (size_t)B * B * 4 <= union_bytes && L::hashpart_bytes() + (size_t)B * B * 4 <= union_bytes) {
+      float* dstg = reinterpret_cast<float*>(uni + union_bytes - (size_t)B * B * 4);
+      const float* Gs = p.gram + (size_t)(p.shared_sets ? kvh : unit) * B * B;
+      for (int c = tid; c < B * B / 4; c += NT) cp_async16(dstg + 4 * c, Gs + 4 * c);
+      gsm = dstg;
+    }
+  }
+  cp_async_commit();
 
   // ------------------------------------------------------------------ phase 0: query hash
   // p[g][j] = P_h[j] . q_g.  Thread (part, j) covers a slice of the 128 channels of row j: products are
@@ -364,6 +386,7 @@ bpc_decode_kernel(const DecodeParams p) {
     if (lane == 0) atomicAdd(&st->rsum, rs);
     if (p.dbg_qweights != nullptr && rank == 0) p.dbg_qweights[(size_t)unit * B + tid] = A;
   }
+  cp_async_wait<0>();                                        // Gram staging (appending block only) has landed
   __syncthreads();
 
   BPC_STAMP(1);
@@ -432,17 +455,32 @@ bpc_decode_kernel(const DecodeParams p) {
         }
       }
     }
-    for (; i0 < c1s; i0 += nts) {                           // tail (and the whole range when scores are exported)
-      const int i = i0 + tid;
-      if (i < c1s) {
-        uint32_t h[W32];
-        load_code(h, i);
-        const int key = score_key<W32, NP>(h, sg, mk);
-        sc[score_slot(i - c0)] = (uint16_t)key;
-        atomicAdd(&hist[key], 1u);
-        if (dbg != nullptr) dbg[i] = ((2 * key) << cs) - rfull;
+    // remainder (and the whole range when scores are exported): the same batches with per-key bounds checks,
+    // so that the loads of a batch are still in flight together
+    for (; i0 < c1s; i0 += nts * U) {
+      uint32_t h[U][W32];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int i = i0 + u * nts + tid;
+        if (i < c1s) {
+          load_code(h[u], i);
+        } else {
+#pragma unroll
+          for (int w = 0; w < W32; ++w) h[u][w] = 0u;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int i = i0 + u * nts + tid;
+        if (i < c1s) {
+          const int key = score_key<W32, NP>(h[u], sg, mk);
+          sc[score_slot(i - c0)] = (uint16_t)key;
+          atomicAdd(&hist[key], 1u);
+          if (dbg != nullptr) dbg[i] = ((2 * key) << cs) - rfull;
+        }
       }
     }
+    if (p.dbg_times != nullptr && tid == 0) p.dbg_times[(size_t)blockIdx.x * 16 + 13] = global_timer_ns();
   } else {
     // ---- appending warp (Algorithm 2 on the new key, Gram form): cache rows, sign sweep, code words.
     // Lane l holds the decision values of bits l, 32+l, ...; bit i is decided by a shuffle from its owner
@@ -466,28 +504,30 @@ bpc_decode_kernel(const DecodeParams p) {
     const float* Gs = p.gram + (size_t)(p.shared_sets ? kvh : unit) * B * B;
     const bool rc = p.residual_correction != 0;
     uint32_t* code_dst = reinterpret_cast<uint32_t*>(p.codes_w) + ((size_t)unit * p.n_max + (n - 1)) * W32;
-    constexpr int PF = 4;                                    // Gram rows per prefetch group
+    constexpr int PF = 8;                                    // Gram rows per prefetch group
 #pragma unroll
     for (int bi = 0; bi < NB; ++bi) {
-      uint32_t wbits = 0;
+      // After step i lane i of the diagonal block is never corrected again (its Gram entries are masked to
+      // zero at fetch time), so at the end its t holds its own decision value and one ballot yields the word.
       float ga[PF][NB], gb[PF][NB];
       auto fetch = [&](float (&gq)[PF][NB], int ii) {
 #pragma unroll
         for (int r = 0; r < PF; ++r)
 #pragma unroll
-          for (int c = bi; c < NB; ++c) gq[r][c] = rc ? __ldg(Gs + (size_t)(32 * bi + ii + r) * B + 32 * c + lane) : 0.f;
+          for (int c = bi; c < NB; ++c) {
+            const size_t gi = (size_t)(32 * bi + ii + r) * B + 32 * c + lane;
+            float gv = !rc ? 0.f : (gsm != nullptr ? gsm[gi] : __ldg(Gs + gi));
+            if (c == bi && lane <= ii + r) gv = 0.f;
+            gq[r][c] = gv;
+          }
       };
       auto sweep = [&](const float (&gq)[PF][NB], int ii) {
 #pragma unroll
         for (int r = 0; r < PF; ++r) {
-          const int i = ii + r;
-          const float ti = __shfl_sync(0xffffffffu, t[bi], i);
-          const bool pos = ti >= 0.f;
-          wbits |= (pos ? 1u : 0u) << i;
-          const float u = pos ? 1.f : -1.f;
-          if (lane > i) t[bi] -= u * gq[r][bi];
+          const float ti = __shfl_sync(0xffffffffu, t[bi], ii + r);
+          const float u = ti >= 0.f ? 1.f : -1.f;
 #pragma unroll
-          for (int c = bi + 1; c < NB; ++c) t[c] -= u * gq[r][c];
+          for (int c = bi; c < NB; ++c) t[c] = fmaf(-u, gq[r][c], t[c]);
         }
       };
       fetch(ga, 0);
@@ -498,8 +538,10 @@ bpc_decode_kernel(const DecodeParams p) {
         if (ii + 2 * PF < 32) fetch(ga, ii + 2 * PF);
         sweep(gb, ii + PF);
       }
+      const uint32_t wbits = __ballot_sync(0xffffffffu, t[bi] >= 0.f);
       if (lane == 0) { st->newcode[bi] = wbits; code_dst[bi] = wbits; }
     }
+    if (p.dbg_times != nullptr && lane == 0) p.dbg_times[(size_t)blockIdx.x * 16 + 11] = global_timer_ns();
   }
   if (appender) {
     __syncthreads();                                         // the new code is in shared memory; the scan is done

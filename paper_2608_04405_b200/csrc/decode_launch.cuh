@@ -37,13 +37,17 @@ static cudaError_t launch_one(bpc_ctx* ctx, const DecodeParams& p_in, cudaStream
   lc.blockDim = dim3(L::NT, 1, 1);
   lc.dynamicSmemBytes = smem;
   lc.stream = stream;
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = (unsigned)ctx->cluster_size;
   at[0].val.clusterDim.y = 1;
   at[0].val.clusterDim.z = 1;
+  // let the grid be scheduled while the previous kernel of the stream drains (the kernel waits for that
+  // kernel's completion itself before it reads anything)
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = at;
-  lc.numAttrs = 1;
+  lc.numAttrs = ctx->use_pdl ? 2 : 1;
   return cudaLaunchKernelEx(&lc, bpc_decode_kernel<KV, GP, W32, MODE>, p);
 }
 
