@@ -161,6 +161,34 @@ def test_fused_append_decode_tiny_and_boundary_lengths():
         assert sess.lens == [n0 + 3]
 
 
+@pytest.mark.parametrize("bits", [64, 128])
+def test_tensor_core_encode_agrees_with_cuda_core_encode(bits):
+    """bpc_encode_keys on the tcgen05 path and on the CUDA-core path (diagnostic switch) against each other and
+    against the checker: ragged length with a partial last tile, several tiles per block."""
+    import os
+    H = _harness()
+    spec = CONFIGS[1].scaled(n_ctx=128 * 37 + 5, n_kv_heads=2, n_q_heads=8, code_bits=bits, steps=1)
+    sess = H.Session(spec)
+    sess.fit()
+    sess.encode()                                   # tensor-core path (bf16, 64/128 bits)
+    tc = sess.codes.clone()
+    rep = {}
+    H.check_encode(sess, [0, 1], rep)
+    os.environ["BPC_NO_TC_ENCODE"] = "1"
+    try:
+        sess.codes.zero_()
+        sess.encode()
+    finally:
+        del os.environ["BPC_NO_TC_ENCODE"]
+    H.check_encode(sess, [0, 1], rep)
+    n = sess.lens[0]
+    diff = (tc[:, :, :n] != sess.codes[:, :, :n]).any(dim=-1).sum().item()
+    # both paths were checked against the fp64 replay above; they may differ from each other only on keys with an
+    # ambiguous decision (fp32 tensor-core sums vs fp64 sums), which are rare
+    assert diff <= max(2, n // 2000), "%d keys differ between the two encode paths" % diff
+    assert torch.count_nonzero(tc[:, :, n:]) == 0   # nothing written past the cached keys
+
+
 def test_error_paths_do_not_launch():
     from paper_2608_04405_b200 import binding as B
     cfg = B.make_config(1, 4, 1, 1024, 128, torch.bfloat16)
