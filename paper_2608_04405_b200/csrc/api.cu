@@ -8,6 +8,10 @@ cudaError_t bpc_launch_decode_bf16(bpc_ctx*, const DecodeParams&, cudaStream_t);
 cudaError_t bpc_launch_decode_f32(bpc_ctx*, const DecodeParams&, cudaStream_t);
 cudaError_t bpc_decode_limits_bf16(const bpc_ctx*, int, int*, int*, size_t*);
 cudaError_t bpc_decode_limits_f32(const bpc_ctx*, int, int*, int*, size_t*);
+cudaError_t bpc_launch_decode_bf16_w7(bpc_ctx*, const DecodeParams&, cudaStream_t);
+cudaError_t bpc_launch_decode_f32_w7(bpc_ctx*, const DecodeParams&, cudaStream_t);
+cudaError_t bpc_decode_limits_bf16_w7(const bpc_ctx*, int, int*, int*, size_t*);
+cudaError_t bpc_decode_limits_f32_w7(const bpc_ctx*, int, int*, int*, size_t*);
 
 namespace {
 
@@ -22,7 +26,8 @@ bpc_status check_cfg(const bpc_config* c) {
   if (c->n_q_heads / c->n_kv_heads > BPC_MAX_GROUP) return BPC_ERR_UNSUPPORTED;
   if (c->kv_dtype != BPC_BF16 && c->kv_dtype != BPC_F32) return BPC_ERR_UNSUPPORTED;
   if (c->score_mode != BPC_SCORE_HAMMING && c->score_mode != BPC_SCORE_WEIGHTED7) return BPC_ERR_INVALID_ARG;
-  if (c->score_mode == BPC_SCORE_WEIGHTED7) return BPC_ERR_UNSUPPORTED;   // not built yet
+  // weighted scores are kept as 16-bit keys: the largest possible score 127 * G * b must fit
+  if (c->score_mode == BPC_SCORE_WEIGHTED7 && 127LL * (c->n_q_heads / c->n_kv_heads) * c->code_bits > 65535) return BPC_ERR_UNSUPPORTED;
   const long long units = (long long)c->batch * c->n_kv_heads;
   if (c->hash_sets != units && c->hash_sets != c->n_kv_heads) return BPC_ERR_INVALID_ARG;
   if (c->residual_correction != 0 && c->residual_correction != 1) return BPC_ERR_INVALID_ARG;
@@ -38,14 +43,25 @@ bpc_status cuda_fail(bpc_ctx* ctx, cudaError_t e) {
   return BPC_ERR_CUDA;
 }
 
-int hamming_bins(const bpc_ctx* ctx) {
-  const int G = ctx->group;
-  const int cs = (G % 2 == 0) ? 1 : 0;
-  return ((G * ctx->cfg.code_bits) >> cs) + 1;
+// Largest score key (sum of |A_j| after removing the common factor), the shift that maps keys to at most 2048
+// histogram bins, and the number of bins.
+int max_score_key(const bpc_ctx* ctx) {
+  const int G = ctx->group, b = ctx->cfg.code_bits;
+  if (ctx->cfg.score_mode == BPC_SCORE_WEIGHTED7) return 127 * G * b;
+  return (G * b) >> ((G % 2 == 0) ? 1 : 0);
 }
+int hist_shift(const bpc_ctx* ctx) {
+  int s = 0;
+  while ((max_score_key(ctx) >> s) >= 2048) ++s;
+  return s;
+}
+int hist_bins(const bpc_ctx* ctx) { return (max_score_key(ctx) >> hist_shift(ctx)) + 1; }
 
 cudaError_t decode_limits(const bpc_ctx* ctx, int /*unused*/, int* max_cluster, int* chunk_cap, size_t* smem) {
-  const int nbins = hamming_bins(ctx);
+  const int nbins = hist_bins(ctx);
+  if (ctx->cfg.score_mode == BPC_SCORE_WEIGHTED7)
+    return ctx->cfg.kv_dtype == BPC_BF16 ? bpc_decode_limits_bf16_w7(ctx, nbins, max_cluster, chunk_cap, smem)
+                                         : bpc_decode_limits_f32_w7(ctx, nbins, max_cluster, chunk_cap, smem);
   return ctx->cfg.kv_dtype == BPC_BF16 ? bpc_decode_limits_bf16(ctx, nbins, max_cluster, chunk_cap, smem)
                                        : bpc_decode_limits_f32(ctx, nbins, max_cluster, chunk_cap, smem);
 }
@@ -141,7 +157,7 @@ bpc_status bpc_create(const bpc_config* cfg, bpc_ctx** out) {
   ctx->chunk_cap_limit = cap;
   ctx->cluster_size = choose_cluster(ctx, cap, ctx->max_cluster);
   if (ctx->cluster_size == 0) { bpc_destroy(ctx); return BPC_ERR_UNSUPPORTED; }
-  if (hamming_bins(ctx) > 2048) { bpc_destroy(ctx); return BPC_ERR_UNSUPPORTED; }
+  if (hist_bins(ctx) > 2048 || hist_shift(ctx) > 5) { bpc_destroy(ctx); return BPC_ERR_UNSUPPORTED; }
   *out = ctx;
   return BPC_OK;
 }
@@ -290,9 +306,14 @@ static bpc_status decode_common(bpc_ctx* ctx, const void* k_new, const void* v_n
   const int chunk = chunk_for(c.n_max, ctx->cluster_size);
   if (chunk > cap) return BPC_ERR_UNSUPPORTED;
   p.chunk_cap = chunk;                                    // shared memory is sized for the largest possible unit
-  p.nbins = hamming_bins(ctx);
-  e = c.kv_dtype == BPC_BF16 ? bpc_launch_decode_bf16(ctx, p, (cudaStream_t)stream)
-                             : bpc_launch_decode_f32(ctx, p, (cudaStream_t)stream);
+  p.nbins = hist_bins(ctx);
+  p.hist_shift = hist_shift(ctx);
+  if (c.score_mode == BPC_SCORE_WEIGHTED7)
+    e = c.kv_dtype == BPC_BF16 ? bpc_launch_decode_bf16_w7(ctx, p, (cudaStream_t)stream)
+                               : bpc_launch_decode_f32_w7(ctx, p, (cudaStream_t)stream);
+  else
+    e = c.kv_dtype == BPC_BF16 ? bpc_launch_decode_bf16(ctx, p, (cudaStream_t)stream)
+                               : bpc_launch_decode_f32(ctx, p, (cudaStream_t)stream);
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   ctx->launches += 1;
   return BPC_OK;

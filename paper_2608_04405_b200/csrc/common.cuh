@@ -75,7 +75,8 @@ struct DecodeParams {
   double sm_scale_d;         // softmax scale
   int stages;                // gather ring depth (2 or 3)
   int chunk_cap;             // keys whose scores one thread block can hold
-  int nbins;                 // histogram bins (largest score key + 1)
+  int nbins;                 // histogram bins
+  int hist_shift;            // histogram bin = score key >> hist_shift
 };
 
 // ---- launchers implemented in the per-dtype translation units

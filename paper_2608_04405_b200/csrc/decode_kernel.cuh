@@ -261,6 +261,7 @@ bpc_decode_kernel(const DecodeParams p) {
   }
 
   const int nbins = p.nbins;
+  const int hsh = p.hist_shift;                              // histogram bin = score key >> hsh (0 in Hamming mode)
   const L plan(p.chunk_cap, nbins, p.stages);
   uint32_t* hist = reinterpret_cast<uint32_t*>(smem + plan.off_hist);
   uint32_t* tot = reinterpret_cast<uint32_t*>(smem + plan.off_tot);
@@ -429,7 +430,7 @@ bpc_decode_kernel(const DecodeParams p) {
       for (int u = 0; u < U; ++u) {
         const int key = score_key<W32, NP>(h[u], sg, mk);
         sc[score_slot(base - c0 + u * nts + tid)] = (uint16_t)key;
-        atomicAdd(&hist[key], 1u);
+        atomicAdd(&hist[key >> hsh], 1u);
       }
     };
     int i0 = c0;
@@ -475,7 +476,7 @@ bpc_decode_kernel(const DecodeParams p) {
         if (i < c1s) {
           const int key = score_key<W32, NP>(h[u], sg, mk);
           sc[score_slot(i - c0)] = (uint16_t)key;
-          atomicAdd(&hist[key], 1u);
+          atomicAdd(&hist[key >> hsh], 1u);
           if (dbg != nullptr) dbg[i] = ((2 * key) << cs) - rfull;
         }
       }
@@ -555,7 +556,7 @@ bpc_decode_kernel(const DecodeParams p) {
       }
       const int key = score_key<W32, NP>(h, sg, mk);
       sc[score_slot(n - 1 - c0)] = (uint16_t)key;
-      atomicAdd(&hist[key], 1u);
+      atomicAdd(&hist[key >> hsh], 1u);
       if (p.dbg_scores != nullptr) p.dbg_scores[(size_t)unit * p.n_max + (n - 1)] = ((2 * key) << cs) - (st->rsum << cs);
     }
   }
@@ -625,6 +626,59 @@ bpc_decode_kernel(const DecodeParams p) {
     if (tid < CS) st->eq[tid] = cluster.map_shared_rank(hist, tid)[T];
   }
   __syncthreads();
+  int T_exact = T;
+  if (hsh > 0) {
+    // Weighted scores have more distinct values than histogram bins: the search above found the coarse bin
+    // that holds the k-th score.  A second, small histogram over the low bits of the keys inside that bin (again
+    // summed across the cluster) yields the exact threshold and corrects the per-block counts.
+    const int FB = 1 << hsh;                                 // at most 32 fine bins
+    uint32_t* fine = tot;
+    if (tid < FB) fine[tid] = 0u;
+    __syncthreads();
+    {
+      const int len = c1 - c0;
+      for (int i = tid; i < len; i += NT) {
+        const int key = (int)sc[score_slot(i)];
+        if ((key >> hsh) == T) atomicAdd(&fine[key & (FB - 1)], 1u);
+      }
+    }
+    cluster.sync();                                          // every block's fine histogram is complete
+    if (warp == 0) {
+      uint32_t fr[BPC_MAX_CLUSTER];
+      uint32_t f = 0;
+#pragma unroll
+      for (int r = 0; r < BPC_MAX_CLUSTER; ++r) {
+        fr[r] = (r < CS && lane < FB) ? cluster.map_shared_rank(fine, r)[lane] : 0u;
+        f += fr[r];
+      }
+      // suffix sums over lanes: above = number of keys of the coarse bin with larger low bits
+      uint32_t incl = f;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_down_sync(0xffffffffu, incl, o);
+        if (lane + o < 32) incl += v;
+      }
+      const uint32_t above = incl - f;
+      const uint32_t need_c = (uint32_t)(k - st->cnt_gt);    // keys still to take from the coarse bin (>= 1)
+      const bool mine = above < need_c && above + f >= need_c;
+      const int vstar = __ffs(__ballot_sync(0xffffffffu, mine)) - 1;
+      const uint32_t above_star = __shfl_sync(0xffffffffu, above, vstar);
+#pragma unroll
+      for (int r = 0; r < BPC_MAX_CLUSTER; ++r) {
+        if (r < CS) {
+          // per block: keys of the coarse bin strictly above the exact threshold, and ties at it
+          uint32_t g = lane > vstar ? fr[r] : 0u;
+#pragma unroll
+          for (int o = 16; o >= 1; o >>= 1) g += __shfl_xor_sync(0xffffffffu, g, o);
+          const uint32_t e = __shfl_sync(0xffffffffu, fr[r], vstar);
+          if (lane == 0) { st->gt[r] += g; st->eq[r] = e; }
+        }
+      }
+      if (lane == 0) { st->T = (T << hsh) | vstar; st->cnt_gt += (int)above_star; }
+    }
+    __syncthreads();
+    T_exact = st->T;
+  }
   if (tid == 0) {
     const int need = k - st->cnt_gt;                         // ties to take, cluster-wide (>= 1)
     int tie_base = 0, out_base = 0;
@@ -647,6 +701,7 @@ bpc_decode_kernel(const DecodeParams p) {
     const int len = c1 - c0;
     const int nseg = (len + kSegKeys - 1) / kSegKeys;
     const int my_take = st->my_take;
+    const int T = T_exact;                                   // shadows the coarse bin: from here on the exact key
     const uint32_t cge = (uint32_t)(0x8000 - T) * 0x10001u;
     constexpr int SPT = 4;                                   // most consecutive segments one thread takes per pass
     const int spt = min(SPT, (nseg + NT - 1) / NT);
@@ -669,9 +724,14 @@ bpc_decode_kernel(const DecodeParams p) {
           uint32_t m = 0;
 #pragma unroll
           for (int w = 0; w < 16; ++w) {
-            const uint32_t gq = kw[w] + cge;
-            m |= (2 * w <= 15 ? (gq >> (15 - 2 * w)) : (gq << (2 * w - 15))) & (1u << (2 * w));
-            m |= (gq >> (30 - 2 * w)) & (2u << (2 * w));
+            if (MODE == 0) {                                 // keys < 2048: both halves compared with one addition
+              const uint32_t gq = kw[w] + cge;
+              m |= (2 * w <= 15 ? (gq >> (15 - 2 * w)) : (gq << (2 * w - 15))) & (1u << (2 * w));
+              m |= (gq >> (30 - 2 * w)) & (2u << (2 * w));
+            } else {                                         // keys up to 65535: compare the halves separately
+              m |= ((int)(kw[w] & 0xffffu) >= T ? 1u : 0u) << (2 * w);
+              m |= ((int)(kw[w] >> 16) >= T ? 2u : 0u) << (2 * w);
+            }
           }
           const int valid = len - seg * kSegKeys;
           if (valid < kSegKeys) m &= (1u << valid) - 1u;     // slots past the end of the chunk hold stale bytes

@@ -104,15 +104,14 @@ static cudaError_t limits_one(const bpc_ctx* ctx, int nbins, int* max_cluster, i
   else if (ctx->group <= 4) { BPC_DISPATCH_W(KV, 4, MODE, FN, __VA_ARGS__) }         \
   else                      { BPC_DISPATCH_W(KV, 8, MODE, FN, __VA_ARGS__) }
 
-template <typename KV>
+// One translation unit per (cache dtype, score mode): MODE 0 = Hamming, MODE 1 = sign + 7 magnitude planes.
+template <typename KV, int MODE>
 static cudaError_t launch_dtype(bpc_ctx* ctx, const DecodeParams& p, cudaStream_t stream) {
-  if (ctx->cfg.score_mode != BPC_SCORE_HAMMING) return cudaErrorNotSupported;
-  BPC_DISPATCH_G(KV, 0, launch_one, ctx, p, stream)
+  BPC_DISPATCH_G(KV, MODE, launch_one, ctx, p, stream)
 }
-template <typename KV>
+template <typename KV, int MODE>
 static cudaError_t limits_dtype(const bpc_ctx* ctx, int nbins, int* max_cluster, int* chunk_cap, size_t* smem) {
-  if (ctx->cfg.score_mode != BPC_SCORE_HAMMING) return cudaErrorNotSupported;
-  BPC_DISPATCH_G(KV, 0, limits_one, ctx, nbins, max_cluster, chunk_cap, smem)
+  BPC_DISPATCH_G(KV, MODE, limits_one, ctx, nbins, max_cluster, chunk_cap, smem)
 }
 
 }  // namespace bpcdev

@@ -161,6 +161,32 @@ def test_fused_append_decode_tiny_and_boundary_lengths():
         assert sess.lens == [n0 + 3]
 
 
+@pytest.mark.parametrize("bits,group,dtype,n", [(128, 4, "bf16", 9000), (64, 8, "bf16", 3000), (256, 1, "bf16", 3000),
+                                                 (64, 2, "f32", 2500), (128, 3, "bf16", 40000)])
+def test_weighted_scores_seven_magnitude_planes(bits, group, dtype, n):
+    """Algorithm 3 as printed (sign + 7 magnitude planes per head): scores, selection with the two-level
+    histogram, output; separate calls and the fused cache write."""
+    H = _harness()
+    from paper_2608_04405_b200 import binding as B
+    spec = CONFIGS[1].scaled(n_ctx=n, n_kv_heads=2, n_q_heads=2 * group, code_bits=bits, dtype=dtype, steps=2,
+                             rope_base=None if dtype == "f32" else 500000.0)
+    sess = H.Session(spec, score_mode=B.BPC_SCORE_WEIGHTED7)
+    rep = {}
+    sess.fit(); sess.encode()
+    _decode_loop(sess, 2, [0, 1], rep, H)
+    q, _ = sess.w.queries(sess.lens)
+    H.check_decode(sess, q.cuda(), [0, 1], rep, budget_ppm=1000000)      # every key selected
+    H.check_decode(sess, q.cuda(), [0], rep, budget_ppm=0, budget_count=1)
+    print(rep)
+
+
+def test_weighted_scores_reject_shapes_whose_scores_exceed_16_bits():
+    from paper_2608_04405_b200 import binding as B
+    with pytest.raises(B.BpcError) as e:
+        B.Context(B.make_config(1, 28, 4, 4096, 128, torch.bfloat16, score_mode=B.BPC_SCORE_WEIGHTED7))   # 127*7*128
+    assert e.value.status == 2
+
+
 @pytest.mark.parametrize("bits", [64, 128])
 def test_tensor_core_encode_agrees_with_cuda_core_encode(bits):
     """bpc_encode_keys on the tcgen05 path and on the CUDA-core path (diagnostic switch) against each other and
