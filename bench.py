@@ -369,7 +369,10 @@ def run_ours(args):
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches_per_region,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": achieved / peaks["hbm_gbs"], "of": peaks["source"], "traffic": None,
+                     "frac": achieved / peaks["hbm_gbs"], "of": peaks["source"],
+                     # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the committed ncu capture of this
+                     # workload (profiles/decode_fused_cfg2_ncu.md); only quoted for the configuration it was taken on
+                     "traffic": 117.8e6 if (args.workload == 2 and not args.separate_kv) else None,
                      "kernel": "bpc_decode_kernel (fused cache write + decode, one launch per step)",
                      "us_per_launch": ms_step * 1e3, "algorithmic_bytes": alg_bytes,
                      "frac_of_nominal_8TBs": achieved / 8000.0},
