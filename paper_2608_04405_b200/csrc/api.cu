@@ -68,19 +68,31 @@ cudaError_t decode_limits(const bpc_ctx* ctx, int /*unused*/, int* max_cluster, 
 
 int chunk_for(int n_max, int cs) { return (((n_max + cs - 1) / cs) + 63) & ~63; }
 
-// Smallest power-of-two cluster whose blocks can hold n_max scores; then grow it while the whole grid
-// still fits one wave of the device.
+// Smallest power-of-two cluster whose blocks can hold n_max scores; then grow it while all clusters of the grid
+// can still be resident at the same time (one wave) and a block keeps at least 1024 keys.
 int choose_cluster(const bpc_ctx* ctx, int chunk_cap, int max_cluster) {
-  int cs = 1;
-  while (cs <= max_cluster && chunk_for(ctx->cfg.n_max, cs) > chunk_cap) cs *= 2;
+  int cs = 1, li = 0;
+  while (cs <= max_cluster && chunk_for(ctx->cfg.n_max, cs) > chunk_cap) { cs *= 2; ++li; }
   if (cs > max_cluster) return 0;
-  while (cs * 2 <= max_cluster && (long long)ctx->units * cs * 2 <= ctx->sm_count &&
-         chunk_for(ctx->cfg.n_max, cs * 2) >= 1024)
+  while (cs * 2 <= max_cluster && ctx->units <= ctx->max_active[li + 1] && chunk_for(ctx->cfg.n_max, cs * 2) >= 1024) {
     cs *= 2;
+    ++li;
+  }
   return cs;
 }
 
 }  // namespace
+
+cudaError_t bpc_plan_decode_geometry(bpc_ctx* ctx) {
+  int mc[6] = {1, 0, 0, 0, 0, 0}, cap = 0;
+  cudaError_t e = decode_limits(ctx, 0, mc, &cap, nullptr);
+  if (e != cudaSuccess) return e;
+  ctx->max_cluster = mc[0];
+  for (int i = 0; i < 5; ++i) ctx->max_active[i] = mc[1 + i];
+  ctx->chunk_cap_limit = cap;
+  ctx->cluster_size = choose_cluster(ctx, cap, ctx->max_cluster);
+  return cudaSuccess;
+}
 
 extern "C" {
 #pragma GCC visibility push(default)
@@ -109,9 +121,8 @@ int64_t bpc_max_context(const bpc_config* c) {
   tmp.cfg = *c;
   tmp.group = c->n_q_heads / c->n_kv_heads;
   if (cudaGetDevice(&tmp.device) != cudaSuccess) return 0;
-  int max_cluster = 1, cap = 0;
-  if (decode_limits(&tmp, 0, &max_cluster, &cap, nullptr) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
-  return (int64_t)max_cluster * cap;
+  if (bpc_plan_decode_geometry(&tmp) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+  return (int64_t)tmp.max_cluster * tmp.chunk_cap_limit;
 }
 
 bpc_status bpc_create(const bpc_config* cfg, bpc_ctx** out) {
@@ -151,11 +162,8 @@ bpc_status bpc_create(const bpc_config* cfg, bpc_ctx** out) {
     (void)cudaGetLastError();
     return BPC_ERR_CUDA;
   }
-  int cap = 0;
-  e = decode_limits(ctx, 0, &ctx->max_cluster, &cap, nullptr);
+  e = bpc_plan_decode_geometry(ctx);
   if (e != cudaSuccess) { bpc_destroy(ctx); (void)cudaGetLastError(); return BPC_ERR_CUDA; }
-  ctx->chunk_cap_limit = cap;
-  ctx->cluster_size = choose_cluster(ctx, cap, ctx->max_cluster);
   if (ctx->cluster_size == 0) { bpc_destroy(ctx); return BPC_ERR_UNSUPPORTED; }
   if (hist_bins(ctx) > 2048 || hist_shift(ctx) > 5) { bpc_destroy(ctx); return BPC_ERR_UNSUPPORTED; }
   *out = ctx;

@@ -22,6 +22,7 @@ struct bpc_ctx {
   int row_stride;           // cache elements between consecutive rows
   int cluster_size;         // decode: thread blocks per cluster
   int max_cluster;          // largest cluster size the device schedules for the decode kernel
+  int max_active[5];        // clusters of size 1, 2, 4, 8, 16 that can be resident at once
   int sm_count;
   bool fitted;
   bool use_pdl;             // launch the decode kernel with programmatic stream serialization
@@ -80,6 +81,9 @@ struct DecodeParams {
 };
 
 // ---- launchers implemented in the per-dtype translation units
+
+// ---- launch geometry (api.cu): fills max_cluster, max_active, chunk_cap_limit and picks cluster_size (0 = none fits)
+cudaError_t bpc_plan_decode_geometry(bpc_ctx* ctx);
 
 // ---- prefill-side launchers (prefill.cu)
 cudaError_t bpc_launch_finalize_projection(bpc_ctx* ctx, cudaStream_t stream);

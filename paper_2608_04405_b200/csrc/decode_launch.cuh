@@ -67,10 +67,12 @@ static cudaError_t limits_one(const bpc_ctx* ctx, int nbins, int* max_cluster, i
   if (chunk_cap) *chunk_cap = cap;
   if (smem_bytes) *smem_bytes = (size_t)optin;
   if (max_cluster) {
+    // max_cluster[0] = largest schedulable cluster size; max_cluster[1 + log2(cs)] = clusters of that size that
+    // can be resident at once (a grid with more clusters than that runs in several waves)
     int best = 1;
     e = configure_kernel<KV, GP, W32, MODE>(dev);
     if (e != cudaSuccess) return e;
-    for (int cs = 2; cs <= BPC_MAX_CLUSTER; cs *= 2) {
+    for (int cs = 1, li = 0; cs <= BPC_MAX_CLUSTER; cs *= 2, ++li) {
       cudaLaunchConfig_t lc = {};
       lc.gridDim = dim3((unsigned)cs, 1, 1);
       lc.blockDim = dim3(L::NT, 1, 1);
@@ -81,11 +83,11 @@ static cudaError_t limits_one(const bpc_ctx* ctx, int nbins, int* max_cluster, i
       lc.attrs = at; lc.numAttrs = 1;
       int nclusters = 0;
       cudaError_t q = cudaOccupancyMaxActiveClusters(&nclusters, bpc_decode_kernel<KV, GP, W32, MODE>, &lc);
-      if (q != cudaSuccess) { (void)cudaGetLastError(); break; }
-      if (nclusters < 1) break;
-      best = cs;
+      if (q != cudaSuccess) { (void)cudaGetLastError(); nclusters = 0; }
+      max_cluster[1 + li] = nclusters;
+      if (nclusters >= 1) best = cs;
     }
-    *max_cluster = best;
+    max_cluster[0] = best;
   }
   return cudaSuccess;
 }

@@ -15,8 +15,6 @@
 
 cudaError_t bpc_launch_decode_bf16(bpc_ctx*, const DecodeParams&, cudaStream_t);
 cudaError_t bpc_launch_decode_f32(bpc_ctx*, const DecodeParams&, cudaStream_t);
-cudaError_t bpc_decode_limits_bf16(const bpc_ctx*, int, int*, int*, size_t*);
-cudaError_t bpc_decode_limits_f32(const bpc_ctx*, int, int*, int*, size_t*);
 
 #define BPC_STATIC_HEADER_BYTES 256                       // error word, padded to the array's alignment
 #define BPC_STATIC_LIST_BYTES (4u << 20)                  // index list: up to 1 Mi int32 entries (units * n_max)
@@ -98,17 +96,10 @@ bpc_status bpc_decode_attn_static(const bpc_config* cfg, const void* q, const vo
 
   const int nbins = ((group * cfg->code_bits) >> ((group % 2 == 0) ? 1 : 0)) + 1;
   if (nbins > 2048) return BPC_ERR_UNSUPPORTED;
-  int max_cluster = 1, cap = 0;
-  e = cfg->kv_dtype == BPC_BF16 ? bpc_decode_limits_bf16(&tmp, nbins, &max_cluster, &cap, nullptr)
-                                : bpc_decode_limits_f32(&tmp, nbins, &max_cluster, &cap, nullptr);
+  e = bpc_plan_decode_geometry(&tmp);                       // occupancy queries only; nothing is allocated
   if (e != cudaSuccess) { (void)cudaGetLastError(); return BPC_ERR_CUDA; }
-  int cs = 1;
-  while (cs <= max_cluster && chunk_for(cfg->n_max, cs) > cap) cs *= 2;
-  if (cs > max_cluster) return BPC_ERR_UNSUPPORTED;
-  while (cs * 2 <= max_cluster && units * cs * 2 <= tmp.sm_count && chunk_for(cfg->n_max, cs * 2) >= 1024) cs *= 2;
-  tmp.cluster_size = cs;
-  tmp.max_cluster = max_cluster;
-  tmp.chunk_cap_limit = cap;
+  if (tmp.cluster_size == 0) return BPC_ERR_UNSUPPORTED;
+  const int cs = tmp.cluster_size;
 
   // the error word accumulates with atomicOr, so it has to start at zero; the list is overwritten before use
   e = cudaMemsetAsync(scratch, 0, BPC_STATIC_HEADER_BYTES, (cudaStream_t)stream);

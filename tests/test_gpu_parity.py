@@ -274,3 +274,45 @@ def test_cfg2_full_size_sampled_units():
     _decode_loop(sess, 1, [0, 13, 31], rep, H)
     # planted-needle recall of the selection is the same number on both sides because the index sets are identical
     print(rep)
+
+
+@pytest.mark.parametrize("bits", [64, 128, 256])
+def test_cfg3_ragged_sweep_code_length_and_budget(bits):
+    """Config 3's sweep (code length x budget) on a ragged batch with lengths in [16384, 65536]; batch reduced to 4,
+    the full-batch launch geometry is covered by the next test."""
+    H = _harness()
+    spec = CONFIGS[3].scaled(batch=4, code_bits=bits, steps=2)
+    sess = H.Session(spec, gen_device="cuda", interleaved=True)
+    rep = {}
+    sess.fit()
+    sess.encode(); H.check_encode(sess, [3], rep, max_keys=4096)
+    q, _ = sess.w.queries(sess.lens)
+    for ppm in (10000, 20000, 50000):
+        H.check_decode(sess, q.cuda(), [1, 30], rep, budget_ppm=ppm)
+    k_new, v_new = sess.w.new_kv(sess.lens)
+    H.check_decode(sess, q.cuda(), [9, 22], rep, append=(k_new.cuda(), v_new.cuda()))
+    print(sess.lens, rep)
+
+
+def test_cfg3_full_batch_sampled_units():
+    """Config 3 at full size (batch 16, 128 units, one block per unit) in the benchmark's launch configuration."""
+    H = _harness()
+    spec = CONFIGS[3]
+    sess = H.Session(spec, gen_device="cuda", interleaved=True)
+    rep = {}
+    sess.fit(); sess.encode()
+    _decode_loop(sess, 2, [0, 77, 127], rep, H, fused=True)
+    print(sess.ctx.get_cluster_size(), rep)
+
+
+def test_cfg4_full_size_sampled_units():
+    """Config 4 at full size (batch 8, 28/4 heads: 7 query heads per KV head, n = 131072): prefill fit + encode, then
+    fused decode steps; sampled units."""
+    H = _harness()
+    spec = CONFIGS[4]
+    sess = H.Session(spec, gen_device="cuda", interleaved=True)
+    rep = {}
+    sess.fit(); H.check_fit(sess, [17], rep)
+    sess.encode(); H.check_encode(sess, [2, 31], rep, key_slice=(60000, 64096))
+    _decode_loop(sess, 2, [0, 19, 31], rep, H, fused=True)
+    print(rep)
