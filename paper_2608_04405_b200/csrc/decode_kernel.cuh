@@ -232,6 +232,27 @@ bpc_decode_kernel(const DecodeParams p) {
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
+  // The projection slice and the queries do not depend on the sequence length: their (cold) loads are issued
+  // first so that they overlap the length read and the set-up below.
+  constexpr int HPARTS = NT / B;                 // slices per projection row in the query hash
+  constexpr int HDS = BPC_D / HPARTS;            // channels per slice (a multiple of 8)
+  constexpr int HV = HDS * (int)sizeof(KV) / 16; // 16-byte vectors per slice
+  uint4 prow[HV];
+  {
+    const int j = tid % B, part = tid / B;
+    const uint4* row = reinterpret_cast<const uint4*>(reinterpret_cast<const KV*>(p.P_h) +
+                                                      ((size_t)(p.shared_sets ? kvh : unit) * B + j) * BPC_D + part * HDS);
+#pragma unroll
+    for (int v = 0; v < HV; ++v) prow[v] = row[v];
+  }
+  const KV* qg = reinterpret_cast<const KV*>(p.q) + ((size_t)seq * p.n_kv_heads + kvh) * (size_t)G * BPC_D;
+  KV qreg[(GP * BPC_D + NT - 1) / NT];
+#pragma unroll
+  for (int v = 0; v < (GP * BPC_D + NT - 1) / NT; ++v) {
+    const int i = tid + v * NT;
+    qreg[v] = (i < GP * BPC_D && (i >> 7) < G) ? qg[i] : (KV)0.f;
+  }
+
   int n = p.unit_lens[unit];
   n = max(0, min(n, p.n_max));
   // Fused cache write: this launch also appends one (k, v) row per unit at position n, codes it and counts it.
@@ -295,12 +316,44 @@ bpc_decode_kernel(const DecodeParams p) {
   }
   cp_async_commit();
 
+  // ---- scan set-up, hoisted above the query hash so that the first batch of codes is already in flight
+  const int c0 = min(n, rank * chunk), c1 = min(n, c0 + chunk);
+  // In the appending block the last warp codes the new key while the other warps scan; the new key's code is
+  // not in memory yet, so the scan stops one key short and the key is scored separately below.
+  const int nts = appender ? NT - 32 : NT;
+  const int c1s = appender ? c1 - 1 : c1;
+  const uint32_t* cu = reinterpret_cast<const uint32_t*>(p.codes) + (size_t)unit * (size_t)p.n_max * W32;
+  int32_t* dbg = p.dbg_scores != nullptr ? p.dbg_scores + (size_t)unit * p.n_max : nullptr;
+  constexpr int U = W32 <= 4 ? 8 : 4;                       // codes in flight per thread and buffer
+  auto load_code = [&](uint32_t (&h)[W32], int i) {
+    const uint32_t* src = cu + (size_t)i * W32;
+    if (W32 == 2) {
+      const uint2 v = ld_stream_v2(src); h[0] = v.x; h[1] = v.y;
+    } else {
+#pragma unroll
+      for (int w = 0; w < W32; w += 4) {
+        const uint4 v = ld_stream_v4(src + w);
+        h[w] = v.x; h[w + 1] = v.y; h[w + 2] = v.z; h[w + 3] = v.w;
+      }
+    }
+  };
+  auto load_batch = [&](uint32_t (&h)[U][W32], int base) {
+#pragma unroll
+    for (int u = 0; u < U; ++u) load_code(h[u], base + u * nts + tid);
+  };
+  uint32_t ha[U][W32], hb[U][W32];
+  const bool pipelined = tid < nts && dbg == nullptr && c0 + nts * U <= c1s;   // at least one full batch
+  if (pipelined) load_batch(ha, c0);
+
   // ------------------------------------------------------------------ phase 0: query hash
   // p[g][j] = P_h[j] . q_g.  Thread (part, j) covers a slice of the 128 channels of row j: products are
   // summed eight at a time in fp32 (exact products for bf16 inputs) and the groups are added in fp64; the
   // slices are then added in fp64 in a fixed order.  Every block of the cluster gets identical bits.
-  const KV* qg = reinterpret_cast<const KV*>(p.q) + ((size_t)seq * p.n_kv_heads + kvh) * (size_t)G * BPC_D;
-  for (int i = tid; i < GP * BPC_D; i += NT) qf_s[i] = (i >> 7) < G ? to_float(qg[i]) : 0.f;
+#pragma unroll
+  for (int v = 0; v < (GP * BPC_D + NT - 1) / NT; ++v) {
+    const int i = tid + v * NT;
+    if (i < GP * BPC_D) qf_s[i] = to_float(qreg[v]);
+  }
   if (tid < BPC_D)                                           // slot GP: the appended key (its decision values P_h k)
     qf_s[GP * BPC_D + tid] = appender ? to_float(reinterpret_cast<const KV*>(p.k_new)[(size_t)unit * BPC_D + tid]) : 0.f;
   for (int i = tid; i < nbins; i += NT) hist[i] = 0u;
@@ -308,25 +361,23 @@ bpc_decode_kernel(const DecodeParams p) {
   if (tid == 0) { st->rsum = 0; st->T = 0; st->cnt_gt = 0; }
   __syncthreads();
   {
-    constexpr int PARTS = NT / B;                  // slices per row
-    constexpr int DS = BPC_D / PARTS;              // channels per slice (a multiple of 8)
+    constexpr int PARTS = HPARTS, DS = HDS;
     const int j = tid % B, part = tid / B;
-    const KV* row = reinterpret_cast<const KV*>(p.P_h) + ((size_t)(p.shared_sets ? kvh : unit) * B + j) * BPC_D + part * DS;
     constexpr int GV = L::GV;
     double acc[GV];
 #pragma unroll
     for (int g = 0; g < GV; ++g) acc[g] = 0.0;
-#pragma unroll 2
+#pragma unroll
     for (int c0 = 0; c0 < DS; c0 += 8) {
       float pv[8];
       if (L::kMma) {
-        const uint4 w = *reinterpret_cast<const uint4*>(row + c0);
+        const uint4 w = prow[c0 / 8];
         pv[0] = bf16_lo(w.x); pv[1] = bf16_hi(w.x); pv[2] = bf16_lo(w.y); pv[3] = bf16_hi(w.y);
         pv[4] = bf16_lo(w.z); pv[5] = bf16_hi(w.z); pv[6] = bf16_lo(w.w); pv[7] = bf16_hi(w.w);
       } else {
-        const float4 w0 = *reinterpret_cast<const float4*>(row + c0);
-        const float4 w1 = *reinterpret_cast<const float4*>(row + c0 + 4);
-        pv[0] = w0.x; pv[1] = w0.y; pv[2] = w0.z; pv[3] = w0.w; pv[4] = w1.x; pv[5] = w1.y; pv[6] = w1.z; pv[7] = w1.w;
+        const uint4 w0 = prow[c0 / 4], w1 = prow[c0 / 4 + 1];
+        pv[0] = __uint_as_float(w0.x); pv[1] = __uint_as_float(w0.y); pv[2] = __uint_as_float(w0.z); pv[3] = __uint_as_float(w0.w);
+        pv[4] = __uint_as_float(w1.x); pv[5] = __uint_as_float(w1.y); pv[6] = __uint_as_float(w1.z); pv[7] = __uint_as_float(w1.w);
       }
 #pragma unroll
       for (int g = 0; g < GV; ++g) {
@@ -392,11 +443,6 @@ bpc_decode_kernel(const DecodeParams p) {
 
   BPC_STAMP(1);
   // ------------------------------------------------------------------ phase 1: scan
-  const int c0 = min(n, rank * chunk), c1 = min(n, c0 + chunk);
-  // In the appending block the last warp codes the new key while the other warps scan; the new key's code is
-  // not in memory yet, so the scan stops one key short and the key is scored separately below.
-  const int nts = appender ? NT - 32 : NT;
-  const int c1s = appender ? c1 - 1 : c1;
   if (tid < nts) {
     uint32_t sg[W32], mk[NP][W32];
 #pragma unroll
@@ -406,25 +452,6 @@ bpc_decode_kernel(const DecodeParams p) {
       for (int pl = 0; pl < NP; ++pl) mk[pl][w] = st->mask[pl][w];
     }
     const int rfull = st->rsum << cs;                       // sum_j |A_j|
-    const uint32_t* cu = reinterpret_cast<const uint32_t*>(p.codes) + (size_t)unit * (size_t)p.n_max * W32;
-    int32_t* dbg = p.dbg_scores != nullptr ? p.dbg_scores + (size_t)unit * p.n_max : nullptr;
-    constexpr int U = W32 <= 4 ? 8 : 4;                     // codes in flight per thread and buffer
-    auto load_code = [&](uint32_t (&h)[W32], int i) {
-      const uint32_t* src = cu + (size_t)i * W32;
-      if (W32 == 2) {
-        const uint2 v = ld_stream_v2(src); h[0] = v.x; h[1] = v.y;
-      } else {
-#pragma unroll
-        for (int w = 0; w < W32; w += 4) {
-          const uint4 v = ld_stream_v4(src + w);
-          h[w] = v.x; h[w + 1] = v.y; h[w + 2] = v.z; h[w + 3] = v.w;
-        }
-      }
-    };
-    auto load_batch = [&](uint32_t (&h)[U][W32], int base) {
-#pragma unroll
-      for (int u = 0; u < U; ++u) load_code(h[u], base + u * nts + tid);
-    };
     auto score_batch = [&](const uint32_t (&h)[U][W32], int base) {
 #pragma unroll
       for (int u = 0; u < U; ++u) {
@@ -434,26 +461,22 @@ bpc_decode_kernel(const DecodeParams p) {
       }
     };
     int i0 = c0;
-    if (dbg == nullptr) {
+    if (pipelined) {
       // Full batches without bounds checks, software-pipelined over two register buffers so that the
       // loads of the next batch are in flight while the current one is scored (a warp's 32 keys share
-      // one score segment).
+      // one score segment).  The first batch was requested before the query hash.
       const int STEP = nts * U;
-      if (i0 + STEP <= c1s) {
-        uint32_t ha[U][W32], hb[U][W32];
-        load_batch(ha, i0);
-        for (;;) {
-          const bool more_b = i0 + 2 * STEP <= c1s;
-          if (more_b) load_batch(hb, i0 + STEP);
-          score_batch(ha, i0);
-          i0 += STEP;
-          if (!more_b) break;
-          const bool more_a = i0 + 2 * STEP <= c1s;
-          if (more_a) load_batch(ha, i0 + STEP);
-          score_batch(hb, i0);
-          i0 += STEP;
-          if (!more_a) break;
-        }
+      for (;;) {
+        const bool more_b = i0 + 2 * STEP <= c1s;
+        if (more_b) load_batch(hb, i0 + STEP);
+        score_batch(ha, i0);
+        i0 += STEP;
+        if (!more_b) break;
+        const bool more_a = i0 + 2 * STEP <= c1s;
+        if (more_a) load_batch(ha, i0 + STEP);
+        score_batch(hb, i0);
+        i0 += STEP;
+        if (!more_a) break;
       }
     }
     // remainder (and the whole range when scores are exported): the same batches with per-key bounds checks,
