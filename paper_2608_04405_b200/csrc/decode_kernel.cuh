@@ -115,6 +115,28 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* wscan,
   return wbase + inc - v;
 }
 
+// the same for two values at once
+template <int NT>
+__device__ __forceinline__ void block_excl_scan2(uint32_t a, uint32_t b, uint32_t* wscan, uint32_t& ea, uint32_t& eb) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t ia = a, ib = b;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t ta = __shfl_up_sync(0xffffffffu, ia, o), tb = __shfl_up_sync(0xffffffffu, ib, o);
+    if (lane >= o) { ia += ta; ib += tb; }
+  }
+  __syncthreads();
+  if (lane == 31) { wscan[warp] = ia; wscan[NT / 32 + warp] = ib; }
+  __syncthreads();
+  uint32_t ba = 0, bb = 0;
+#pragma unroll
+  for (int w = 0; w < NT / 32; ++w) {
+    if (w < warp) { ba += wscan[w]; bb += wscan[NT / 32 + w]; }
+  }
+  ea = ba + ia - a;
+  eb = bb + ib - b;
+}
+
 template <typename T> __device__ __forceinline__ T fast_exp2(T x);
 template <> __device__ __forceinline__ float fast_exp2<float>(float x) { return exp2f(x); }
 template <> __device__ __forceinline__ double fast_exp2<double>(double x) { return exp2(x); }
@@ -589,66 +611,103 @@ bpc_decode_kernel(const DecodeParams p) {
   cluster.sync();                                            // every block's histogram is complete
   BPC_STAMP(8);
   if (appender && tid == 0) p.unit_lens_w[unit] = n;         // every block of the cluster has read the old length
-  // Total histogram through distributed shared memory.  With at most one bin per thread (the common case)
-  // the per-block counts of that bin stay in registers and are reused for the per-block offsets below.
-  const bool one_bin = nbins <= NT;
-  uint32_t myv[BPC_MAX_CLUSTER];
-#pragma unroll
-  for (int r = 0; r < BPC_MAX_CLUSTER; ++r) myv[r] = 0u;
-  if (one_bin) {
-    if (tid < nbins) {
-      uint32_t s = 0;
-#pragma unroll
-      for (int r = 0; r < BPC_MAX_CLUSTER; ++r)
-        if (r < CS) { myv[r] = cluster.map_shared_rank(hist, r)[tid]; s += myv[r]; }
-      tot[tid] = s;
-    }
-  } else {
-    for (int bin = tid; bin < nbins; bin += NT) {
-      uint32_t s = 0;
-      for (int r = 0; r < CS; ++r) s += cluster.map_shared_rank(hist, r)[bin];
-      tot[bin] = s;
-    }
-  }
-  __syncthreads();
-  {
-    const int bpt = (nbins + NT - 1) / NT;                   // bins per thread; thread 0 owns the highest bins
-    const int hi = nbins - tid * bpt;
-    const int lo = max(0, hi - bpt);
-    uint32_t local = 0;
-    for (int bin = hi - 1; bin >= lo; --bin) local += tot[bin];
-    uint32_t total;
-    uint32_t above = block_excl_scan<NT>(local, st->wscan, &total);
-    for (int bin = hi - 1; bin >= lo; --bin) {
-      const uint32_t c = tot[bin];
-      if (above < (uint32_t)k && above + c >= (uint32_t)k) { st->T = bin; st->cnt_gt = (int)above; }
-      above += c;
-    }
-  }
-  __syncthreads();
-  const int T = st->T;
-  BPC_STAMP(9);
-  if (one_bin) {
-    if (tid < nbins && tid >= T) {
+  // Threshold key T (the k-th largest score key) and this block's share of the output.
+  int T;
+  const bool fast_sel = nbins <= NT && hsh == 0;
+  if (fast_sel) {
+    // Common case, one histogram bin per thread: thread t owns bin nbins-1-t, reads that bin from every block of
+    // the cluster (distributed shared memory) and a two-value block scan yields, for every bin, the number of keys
+    // in higher bins (cluster-wide, and in the blocks of lower rank).  The thread whose bin holds the k-th key
+    // then knows everything this block needs: T, how many ties it may take and where its output starts
+    // (ties are granted to blocks in rank order, which is index order).
+    const int bin = nbins - 1 - tid;
+    uint32_t s_all = 0, s_low = 0, mine = 0;
+    if (bin >= 0) {
 #pragma unroll
       for (int r = 0; r < BPC_MAX_CLUSTER; ++r) {
         if (r < CS) {
-          if (tid == T) st->eq[r] = myv[r];
-          else if (myv[r]) atomicAdd(&st->gt[r], myv[r]);
+          const uint32_t v = cluster.map_shared_rank(hist, r)[bin];
+          s_all += v;
+          if (r < rank) s_low += v;
+          if (r == rank) mine = v;
         }
       }
     }
+    uint32_t above_all, above_low;
+    block_excl_scan2<NT>(s_all, s_low, st->wscan, above_all, above_low);
+    if (bin >= 0 && above_all < (uint32_t)k && above_all + s_all >= (uint32_t)k) {
+      const int need = k - (int)above_all;                   // ties to take, cluster-wide (>= 1)
+      const int lower_take = min(need, (int)s_low);          // ties granted to blocks of lower rank
+      st->T = bin;
+      st->cnt_gt = (int)above_all;
+      st->my_take = min(max(need - (int)s_low, 0), (int)mine);
+      st->my_base = (int)above_low + lower_take;
+    }
+    __syncthreads();
+    T = st->T;
+    BPC_STAMP(9);
   } else {
-    for (int bin = T + 1 + tid; bin < nbins; bin += NT) {
-      if (tot[bin] == 0u) continue;
-      for (int r = 0; r < CS; ++r) {
-        const uint32_t v = cluster.map_shared_rank(hist, r)[bin];
-        if (v) atomicAdd(&st->gt[r], v);
+  // Total histogram through distributed shared memory.  With at most one bin per thread (the common case)
+    // the per-block counts of that bin stay in registers and are reused for the per-block offsets below.
+    const bool one_bin = nbins <= NT;
+    uint32_t myv[BPC_MAX_CLUSTER];
+#pragma unroll
+    for (int r = 0; r < BPC_MAX_CLUSTER; ++r) myv[r] = 0u;
+    if (one_bin) {
+      if (tid < nbins) {
+        uint32_t s = 0;
+#pragma unroll
+        for (int r = 0; r < BPC_MAX_CLUSTER; ++r)
+          if (r < CS) { myv[r] = cluster.map_shared_rank(hist, r)[tid]; s += myv[r]; }
+        tot[tid] = s;
+      }
+    } else {
+      for (int bin = tid; bin < nbins; bin += NT) {
+        uint32_t s = 0;
+        for (int r = 0; r < CS; ++r) s += cluster.map_shared_rank(hist, r)[bin];
+        tot[bin] = s;
       }
     }
-    if (tid < CS) st->eq[tid] = cluster.map_shared_rank(hist, tid)[T];
+    __syncthreads();
+    {
+      const int bpt = (nbins + NT - 1) / NT;                   // bins per thread; thread 0 owns the highest bins
+      const int hi = nbins - tid * bpt;
+      const int lo = max(0, hi - bpt);
+      uint32_t local = 0;
+      for (int bin = hi - 1; bin >= lo; --bin) local += tot[bin];
+      uint32_t total;
+      uint32_t above = block_excl_scan<NT>(local, st->wscan, &total);
+      for (int bin = hi - 1; bin >= lo; --bin) {
+        const uint32_t c = tot[bin];
+        if (above < (uint32_t)k && above + c >= (uint32_t)k) { st->T = bin; st->cnt_gt = (int)above; }
+        above += c;
+      }
+    }
+    __syncthreads();
+    T = st->T;
+    BPC_STAMP(9);
+    if (one_bin) {
+      if (tid < nbins && tid >= T) {
+#pragma unroll
+        for (int r = 0; r < BPC_MAX_CLUSTER; ++r) {
+          if (r < CS) {
+            if (tid == T) st->eq[r] = myv[r];
+            else if (myv[r]) atomicAdd(&st->gt[r], myv[r]);
+          }
+        }
+      }
+    } else {
+      for (int bin = T + 1 + tid; bin < nbins; bin += NT) {
+        if (tot[bin] == 0u) continue;
+        for (int r = 0; r < CS; ++r) {
+          const uint32_t v = cluster.map_shared_rank(hist, r)[bin];
+          if (v) atomicAdd(&st->gt[r], v);
+        }
+      }
+      if (tid < CS) st->eq[tid] = cluster.map_shared_rank(hist, tid)[T];
+    }
+    __syncthreads();
   }
-  __syncthreads();
   int T_exact = T;
   if (hsh > 0) {
     // Weighted scores have more distinct values than histogram bins: the search above found the coarse bin
@@ -702,7 +761,7 @@ bpc_decode_kernel(const DecodeParams p) {
     __syncthreads();
     T_exact = st->T;
   }
-  if (tid == 0) {
+  if (!fast_sel && tid == 0) {
     const int need = k - st->cnt_gt;                         // ties to take, cluster-wide (>= 1)
     int tie_base = 0, out_base = 0;
     for (int r = 0; r < CS; ++r) {
