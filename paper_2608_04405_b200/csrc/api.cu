@@ -66,7 +66,13 @@ cudaError_t decode_limits(const bpc_ctx* ctx, int /*unused*/, int* max_cluster, 
                                        : bpc_decode_limits_f32(ctx, nbins, max_cluster, chunk_cap, smem);
 }
 
-int chunk_for(int n_max, int cs) { return (((n_max + cs - 1) / cs) + 63) & ~63; }
+// keys per block the kernel may assign (the larger of its plain and its fused-launch split), rounded to 64
+int chunk_for(int n_max, int cs) {
+  const int plain = (((n_max + cs - 1) / cs) + 63) & ~63;
+  if (cs == 1) return plain;
+  const int fused = ((int)(((long long)n_max * 16 + 16 * cs - 2) / (16 * cs - 1)) + 63) & ~63;
+  return fused > plain ? fused : plain;
+}
 
 // Smallest power-of-two cluster whose blocks can hold n_max scores; then grow it while all clusters of the grid
 // can still be resident at the same time (one wave) and a block keeps at least 1024 keys.

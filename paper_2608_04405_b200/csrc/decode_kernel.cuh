@@ -288,7 +288,10 @@ bpc_decode_kernel(const DecodeParams p) {
                                     : ((long long)n * (long long)p.budget_ppm + 999999LL) / 1000000LL;
   if (kk < 0) kk = 0;
   const int k = (int)(kk < (long long)n ? kk : (long long)n);
-  const int chunk = (((n + CS - 1) / CS) + 63) & ~63;
+  // Keys per block.  In a fused launch the appending block (the last one with keys) scans with one warp less, so
+  // it is given 15/16 of the others' share.
+  const int chunk = (fused && CS > 1) ? ((int)(((long long)n * 16 + 16 * CS - 2) / (16 * CS - 1)) + 63) & ~63
+                                      : (((n + CS - 1) / CS) + 63) & ~63;
   float* out_u = p.out + ((size_t)seq * p.n_kv_heads + kvh) * (size_t)G * BPC_D;
 
   // Both early exits depend only on values every block of the cluster sees identically, so either all

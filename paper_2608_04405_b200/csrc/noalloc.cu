@@ -41,7 +41,13 @@ cudaError_t scratch_for_current_device(int device, void** out) {
   return cudaSuccess;
 }
 
-int chunk_for(int n_max, int cs) { return (((n_max + cs - 1) / cs) + 63) & ~63; }
+// keys per block the kernel may assign (the larger of its plain and its fused-launch split), rounded to 64
+int chunk_for(int n_max, int cs) {
+  const int plain = (((n_max + cs - 1) / cs) + 63) & ~63;
+  if (cs == 1) return plain;
+  const int fused = ((int)(((long long)n_max * 16 + 16 * cs - 2) / (16 * cs - 1)) + 63) & ~63;
+  return fused > plain ? fused : plain;
+}
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
