@@ -25,7 +25,8 @@ Algorithm 1, rank-1 closed form, least-squares optimality of v, greedy step
 optimality and the orthogonal-P special case of Algorithm 2, Gram form vs
 residual form, Hamming identity, bit-plane formula vs integer dot product
 (exhaustive at 8 bits), brute-force sort for top-k, dense softmax at budget n,
-scale invariance of query codes, storage arithmetic printed in the paper.
+scale invariance of query codes, storage arithmetic printed in the paper, safeguard set vs brute force and
+its identity ||k - hP||^2 = ||k||^2 - 2 sum|t_i| + tr(P P^T) with the decision values t_i of Algorithm 2.
 Parity unpinned: none of the functions below (the paper prints no numeric
 worked example; every function has at least one mathematical pin).
 """
@@ -218,18 +219,41 @@ def attend(q_group: np.ndarray, K: np.ndarray, V: np.ndarray, idx: np.ndarray, s
     return w @ Vs
 
 
+# --------------------------------------------------------------------------- Error-Aware Safeguard (Eqs. 8-9)
+def eas_set(errors: np.ndarray, m: int) -> np.ndarray:
+    """Hard-to-hash set S_err: indices of the m largest reconstruction errors ||k - h P||_2 (Eq. 8), ties to the
+    lowest index, returned in ascending index order.  It is built once, at prefill."""
+    errors = np.asarray(errors, dtype=np.float64)
+    order = np.lexsort((np.arange(errors.shape[0]), -errors))
+    return np.sort(order[:max(0, min(m, errors.shape[0]))]).astype(np.int64)
+
+
+def eas_union(hash_idx: np.ndarray, s_err: np.ndarray) -> np.ndarray:
+    """S_attn = S_hash united with S_err (Eq. 9), ascending."""
+    return np.union1d(np.asarray(hash_idx, dtype=np.int64), np.asarray(s_err, dtype=np.int64))
+
+
 # --------------------------------------------------------------------------- one decode step of one unit
-def decode_unit(q_group, K, V, bits, P_h, ppm, count=0, mode=HAMMING, sm_scale=0.0):
+def decode_unit(q_group, K, V, bits, P_h, ppm, count=0, mode=HAMMING, sm_scale=0.0, s_err=None):
     """Query hash -> scores over all cached keys -> top-k -> attention.  K, V, bits hold the n cached rows.
 
-    Returns dict(out [G, D], idx [k], scores [n], s, a).
+    With an error-aware safeguard set s_err (ascending indices), the budget k is split: the first min(|s_err|, k)
+    safeguard keys are always attended and the hash search fills the remaining k - min(|s_err|, k) places
+    (it competes over all keys, so a key may be chosen twice; the union removes it).
+    Returns dict(out [G, D], idx [<= k] (attended keys, ascending), hash_idx, scores [n], s, a).
     """
     _, s, a = query_hash(q_group, P_h, mode)
     sc = hash_scores(bits, s, a)
     k = budget(bits.shape[0], ppm, count)
-    idx = topk(sc, k)
+    if s_err is None:
+        hash_idx = topk(sc, k)
+        idx = hash_idx
+    else:
+        me = min(len(s_err), k)
+        hash_idx = topk(sc, k - me)
+        idx = eas_union(hash_idx, np.asarray(s_err)[:me])
     out = attend(q_group, K, V, idx, sm_scale)
-    return dict(out=out, idx=idx, scores=sc, s=s, a=a)
+    return dict(out=out, idx=idx, hash_idx=hash_idx, scores=sc, s=s, a=a)
 
 
 def ambiguity_threshold_query(q_row: np.ndarray, P_h: np.ndarray, rel: float = 1e-6) -> np.ndarray:

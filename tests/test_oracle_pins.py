@@ -314,3 +314,47 @@ def test_replay_with_adoption_flags_only_real_mismatches():
     bad = bits.copy(); bad[3, 5] ^= 1
     hard, amb = O.replay_encode_with_adoption(K, P, bad)
     assert hard[3, 5] and hard.sum() >= 1 and not hard[:3].any()
+
+
+# ------------------------------------------------------------------ error-aware safeguard
+def test_eas_set_bruteforce_and_union():
+    err = np.array([0.5, 2.0, 2.0, 0.1, 3.0, 2.0])
+    assert list(O.eas_set(err, 1)) == [4]
+    assert list(O.eas_set(err, 3)) == [1, 2, 4]          # ties at 2.0 go to the lowest indices
+    assert list(O.eas_set(err, 10)) == [0, 1, 2, 3, 4, 5]
+    assert list(O.eas_set(err, 0)) == []
+    r = RNG.random(300)
+    for m in (1, 7, 299):
+        want = sorted(sorted(range(300), key=lambda i: (-r[i], i))[:m])
+        assert list(O.eas_set(r, m)) == want
+    assert list(O.eas_union([1, 5, 9], [5, 2])) == [1, 2, 5, 9]
+
+
+def test_reconstruction_error_identity_from_decision_values():
+    # ||k - h P||^2 = ||k||^2 - 2 sum_i |t_i| + trace(P P^T), t_i = decision value of bit i in Algorithm 2:
+    # (the by-product a sweep-based encoder can use instead of forming the residual)
+    n, D, b = 40, 24, 16
+    K = _keys(n, D); P = RNG.standard_normal((b, D)) * 0.4
+    bits, rn = O.encode(K, P)
+    for row in range(n):
+        r = K[row].copy(); tsum = 0.0
+        for i in range(b):
+            t = float(r @ P[i]); tsum += abs(t)
+            r = r - (1.0 if t >= 0 else -1.0) * P[i]
+        rhs = float(K[row] @ K[row]) - 2.0 * tsum + float(np.trace(P @ P.T))
+        assert abs(rn[row] ** 2 - rhs) <= 1e-9 * max(1.0, float(K[row] @ K[row]))
+
+
+def test_decode_unit_with_safeguard_set():
+    G, D, n, b = 2, 16, 200, 64
+    K = _keys(n, D); V = RNG.standard_normal((n, D)); q = RNG.standard_normal((G, D))
+    P, _, _ = O.fit(K, RNG.standard_normal((b, D)))
+    bits, err = O.encode(K, P)
+    s_err = O.eas_set(err, 4)
+    plain = O.decode_unit(q, K, V, bits, P, ppm=100000)                 # k = 20
+    r = O.decode_unit(q, K, V, bits, P, ppm=100000, s_err=s_err)
+    assert len(r["hash_idx"]) == 16 and set(r["hash_idx"]) <= set(plain["idx"])   # top-16 is a prefix of top-20
+    assert set(s_err) <= set(r["idx"]) and 16 <= len(r["idx"]) <= 20
+    assert np.allclose(r["out"], O.attend(q, K, V, r["idx"]), atol=1e-13)
+    tiny = O.decode_unit(q, K, V, bits, P, ppm=0, count=3, s_err=s_err)   # budget below the safeguard size
+    assert list(tiny["idx"]) == list(s_err[:3]) and len(tiny["hash_idx"]) == 0
