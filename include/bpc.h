@@ -71,6 +71,8 @@ typedef struct {
   int32_t hash_sets;            /* batch*n_kv_heads (one projection per unit) or n_kv_heads (shared per KV head) */
   int32_t residual_correction;  /* 1: Algorithm 2 (default). 0: plain sign(k P^T), for comparison only */
   int32_t kv_row_stride;        /* elements between consecutive cache rows; 0 selects head_dim */
+  int32_t eas_ppm;              /* error-aware safeguard: size of the hard-to-hash set as parts per million of the
+                                   keys cached when bpc_build_eas runs (0 = no safeguard; at most 16384 keys per unit) */
 } bpc_config;
 
 typedef struct bpc_ctx bpc_ctx;
@@ -116,6 +118,19 @@ bpc_status bpc_get_projection(bpc_ctx* ctx, float* P_out, float* P_hash_out, flo
 
 /* Algorithm 2 for the first seq_len keys of every unit: codes[unit][0..seq_len). */
 bpc_status bpc_encode_keys(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, void* stream);
+
+/* Error-Aware Safeguard (Section 3.2, Eqs. 8-9).  With cfg.eas_ppm > 0, bpc_encode_keys also records every
+ * key's reconstruction error ||k - h P_h||_2 (squared), and bpc_build_eas, called once after it, keeps per unit the
+ * m = ceil(seq_len * eas_ppm / 1e6) keys with the largest error (ties to the lowest index) as the static set S_err.
+ * From then on a decode step with budget k always attends the first min(m, k) keys of S_err and lets the hash search
+ * fill the other k - min(m, k) places; keys found by both are attended once.  With sel_idx given, entries
+ * [0, k - min(m,k)) are the hash-selected keys (ascending) and the following min(m, k) entries are S_err in ascending
+ * order with -1 in place of keys the hash search already selected.  Keys appended later never join S_err.
+ * Requires residual_correction = 1 and Hamming scores.  bpc_get_eas copies out the squared errors [units][n_max] float, the set
+ * [units][eas_capacity] int32 and its sizes [units] int32 (any pointer may be NULL). */
+bpc_status bpc_build_eas(bpc_ctx* ctx, void* stream);
+bpc_status bpc_get_eas(bpc_ctx* ctx, float* sq_err_out, int32_t* set_out, int32_t* count_out, void* stream);
+int32_t    bpc_eas_capacity(const bpc_config* host_cfg);
 
 /* Cache write of one new (k, v) row per unit at position seq_len, Algorithm 2 on the new key, its
  * code stored beside the others, seq_len += 1 (on the device and in the host shadow).

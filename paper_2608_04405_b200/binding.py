@@ -32,7 +32,7 @@ class bpc_config(ctypes.Structure):
     _fields_ = [("batch", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
                 ("head_dim", ctypes.c_int32), ("code_bits", ctypes.c_int32), ("n_max", ctypes.c_int32),
                 ("kv_dtype", ctypes.c_int32), ("score_mode", ctypes.c_int32), ("sm_scale", ctypes.c_float),
-                ("hash_sets", ctypes.c_int32), ("residual_correction", ctypes.c_int32), ("kv_row_stride", ctypes.c_int32)]
+                ("hash_sets", ctypes.c_int32), ("residual_correction", ctypes.c_int32), ("kv_row_stride", ctypes.c_int32), ("eas_ppm", ctypes.c_int32)]
 
 
 def _load() -> ctypes.CDLL:
@@ -54,6 +54,9 @@ def _load() -> ctypes.CDLL:
         "bpc_set_projection": (i32, [vp, vp, vp]),
         "bpc_get_projection": (i32, [vp, vp, vp, vp, vp]),
         "bpc_encode_keys": (i32, [vp, vp, vp, vp]),
+        "bpc_build_eas": (i32, [vp, vp]),
+        "bpc_get_eas": (i32, [vp, vp, vp, vp, vp]),
+        "bpc_eas_capacity": (i32, [cfgp]),
         "bpc_append": (i32, [vp, vp, vp, vp, vp, vp, vp]),
         "bpc_decode_attn": (i32, [vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]),
         "bpc_append_decode_attn": (i32, [vp, vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]),
@@ -79,7 +82,7 @@ lib = _load()
 EXPORTS = ["bpc_create", "bpc_destroy", "bpc_codes_bytes", "bpc_fit_workspace_bytes", "bpc_fit_codes_offset",
            "bpc_max_context",
            "bpc_set_seq_lens", "bpc_get_seq_lens", "bpc_fit", "bpc_set_projection", "bpc_get_projection",
-           "bpc_encode_keys", "bpc_append", "bpc_decode_attn", "bpc_append_decode_attn", "bpc_decode_attn_static", "bpc_static_scratch_entries",
+           "bpc_encode_keys", "bpc_build_eas", "bpc_get_eas", "bpc_eas_capacity", "bpc_append", "bpc_decode_attn", "bpc_append_decode_attn", "bpc_decode_attn_static", "bpc_static_scratch_entries",
            "bpc_debug_set_buffers", "bpc_debug_set_phase_timer",
            "bpc_set_cluster_size",
            "bpc_get_cluster_size", "bpc_last_device_error", "bpc_last_cuda_error", "bpc_launch_count", "bpc_version"]
@@ -115,10 +118,11 @@ def _check(status: int, what: str) -> None:
 
 def make_config(batch: int, n_q_heads: int, n_kv_heads: int, n_max: int, code_bits: int, dtype: torch.dtype,
                 score_mode: int = BPC_SCORE_HAMMING, sm_scale: float = 0.0, shared_projection: bool = False,
-                residual_correction: bool = True, head_dim: int = 128, kv_row_stride: int = 0) -> bpc_config:
+                residual_correction: bool = True, head_dim: int = 128, kv_row_stride: int = 0,
+                eas_ppm: int = 0) -> bpc_config:
     return bpc_config(batch, n_q_heads, n_kv_heads, head_dim, code_bits, n_max,
                       BPC_BF16 if dtype == torch.bfloat16 else BPC_F32, score_mode, sm_scale,
-                      n_kv_heads if shared_projection else batch * n_kv_heads, 1 if residual_correction else 0, kv_row_stride)
+                      n_kv_heads if shared_projection else batch * n_kv_heads, 1 if residual_correction else 0, kv_row_stride, eas_ppm)
 
 
 class Context:
@@ -197,6 +201,18 @@ class Context:
 
     def encode_keys(self, k_cache: torch.Tensor, codes: torch.Tensor) -> None:
         _check(lib.bpc_encode_keys(self._h, _cache_ptr(k_cache), _ptr(codes), _stream()), "bpc_encode_keys")
+
+    def build_eas(self) -> None:
+        _check(lib.bpc_build_eas(self._h, _stream()), "bpc_build_eas")
+
+    def get_eas(self):
+        c = self.cfg
+        cap = lib.bpc_eas_capacity(ctypes.byref(c))
+        err = torch.empty(self.units, c.n_max, dtype=torch.float32, device="cuda")
+        idx = torch.empty(self.units, max(cap, 1), dtype=torch.int32, device="cuda")
+        cnt = torch.empty(self.units, dtype=torch.int32, device="cuda")
+        _check(lib.bpc_get_eas(self._h, _ptr(err), _ptr(idx), _ptr(cnt), _stream()), "bpc_get_eas")
+        return err, idx, cnt
 
     def append(self, k_new, v_new, k_cache, v_cache, codes) -> None:
         _check(lib.bpc_append(self._h, _ptr(k_new), _ptr(v_new), _cache_ptr(k_cache), _cache_ptr(v_cache), _ptr(codes), _stream()),

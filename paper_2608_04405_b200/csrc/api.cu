@@ -8,6 +8,10 @@ cudaError_t bpc_launch_decode_bf16(bpc_ctx*, const DecodeParams&, cudaStream_t);
 cudaError_t bpc_launch_decode_f32(bpc_ctx*, const DecodeParams&, cudaStream_t);
 cudaError_t bpc_decode_limits_bf16(const bpc_ctx*, int, int*, int*, size_t*);
 cudaError_t bpc_decode_limits_f32(const bpc_ctx*, int, int*, int*, size_t*);
+cudaError_t bpc_launch_decode_bf16_eas(bpc_ctx*, const DecodeParams&, cudaStream_t);
+cudaError_t bpc_launch_decode_f32_eas(bpc_ctx*, const DecodeParams&, cudaStream_t);
+cudaError_t bpc_decode_limits_bf16_eas(const bpc_ctx*, int, int*, int*, size_t*);
+cudaError_t bpc_decode_limits_f32_eas(const bpc_ctx*, int, int*, int*, size_t*);
 cudaError_t bpc_launch_decode_bf16_w7(bpc_ctx*, const DecodeParams&, cudaStream_t);
 cudaError_t bpc_launch_decode_f32_w7(bpc_ctx*, const DecodeParams&, cudaStream_t);
 cudaError_t bpc_decode_limits_bf16_w7(const bpc_ctx*, int, int*, int*, size_t*);
@@ -33,6 +37,9 @@ bpc_status check_cfg(const bpc_config* c) {
   if (c->residual_correction != 0 && c->residual_correction != 1) return BPC_ERR_INVALID_ARG;
   if (!(c->sm_scale >= 0.f)) return BPC_ERR_INVALID_ARG;
   if (c->kv_row_stride != 0 && (c->kv_row_stride < c->head_dim || c->kv_row_stride % 8 != 0)) return BPC_ERR_INVALID_ARG;
+  if (c->eas_ppm < 0 || c->eas_ppm > 1000000) return BPC_ERR_INVALID_ARG;
+  if (c->eas_ppm > 0 && (c->residual_correction == 0 || c->score_mode != BPC_SCORE_HAMMING)) return BPC_ERR_UNSUPPORTED;
+  if (c->eas_ppm > 0 && ((long long)c->n_max * c->eas_ppm + 999999) / 1000000 > 16384) return BPC_ERR_UNSUPPORTED;
   if (c->n_max % 2 != 0) return BPC_ERR_INVALID_ARG;   // keeps every unit's code rows 16-byte aligned at 64 bits
   return BPC_OK;
 }
@@ -62,6 +69,9 @@ cudaError_t decode_limits(const bpc_ctx* ctx, int /*unused*/, int* max_cluster, 
   if (ctx->cfg.score_mode == BPC_SCORE_WEIGHTED7)
     return ctx->cfg.kv_dtype == BPC_BF16 ? bpc_decode_limits_bf16_w7(ctx, nbins, max_cluster, chunk_cap, smem)
                                          : bpc_decode_limits_f32_w7(ctx, nbins, max_cluster, chunk_cap, smem);
+  if (ctx->cfg.eas_ppm > 0)
+    return ctx->cfg.kv_dtype == BPC_BF16 ? bpc_decode_limits_bf16_eas(ctx, nbins, max_cluster, chunk_cap, smem)
+                                         : bpc_decode_limits_f32_eas(ctx, nbins, max_cluster, chunk_cap, smem);
   return ctx->cfg.kv_dtype == BPC_BF16 ? bpc_decode_limits_bf16(ctx, nbins, max_cluster, chunk_cap, smem)
                                        : bpc_decode_limits_f32(ctx, nbins, max_cluster, chunk_cap, smem);
 }
@@ -158,6 +168,14 @@ bpc_status bpc_create(const bpc_config* cfg, bpc_ctx** out) {
   if (e == cudaSuccess) e = cudaMalloc(&ctx->gram, hs * b * b * 4);
   if (e == cudaSuccess) e = cudaMalloc(&ctx->unit_lens, (size_t)ctx->units * 4);
   if (e == cudaSuccess) e = cudaMalloc(&ctx->sel_scratch, (size_t)ctx->units * cfg->n_max * 4);
+  if (cfg->eas_ppm > 0) {
+    ctx->eas_cap = (int)(((long long)cfg->n_max * cfg->eas_ppm + 999999) / 1000000);
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->key_err, (size_t)ctx->units * cfg->n_max * 4);
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->eas_idx, (size_t)ctx->units * ctx->eas_cap * 4);
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->eas_cnt, (size_t)ctx->units * 4);
+    if (e == cudaSuccess) e = cudaMemset(ctx->eas_cnt, 0, (size_t)ctx->units * 4);
+    if (e == cudaSuccess) e = cudaMemset(ctx->key_err, 0, (size_t)ctx->units * cfg->n_max * 4);
+  }
   if (e == cudaSuccess) e = cudaMalloc(&ctx->dev_err, 4);
   if (e == cudaSuccess) e = cudaMemset(ctx->dev_err, 0, 4);
   if (e == cudaSuccess) e = cudaMemset(ctx->unit_lens, 0, (size_t)ctx->units * 4);
@@ -180,6 +198,7 @@ bpc_status bpc_destroy(bpc_ctx* ctx) {
   if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
   cudaFree(ctx->P); cudaFree(ctx->P_h); cudaFree(ctx->P_hf); cudaFree(ctx->gram);
   cudaFree(ctx->unit_lens); cudaFree(ctx->sel_scratch); cudaFree(ctx->dev_err);
+  cudaFree(ctx->key_err); cudaFree(ctx->eas_idx); cudaFree(ctx->eas_cnt);
   delete[] ctx->host_lens;
   delete ctx;
   (void)cudaGetLastError();
@@ -275,6 +294,29 @@ bpc_status bpc_encode_keys(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, v
   return e == cudaSuccess ? BPC_OK : cuda_fail(ctx, e);
 }
 
+int32_t bpc_eas_capacity(const bpc_config* c) {
+  if (check_cfg(c) != BPC_OK || c->eas_ppm <= 0) return 0;
+  return (int32_t)(((long long)c->n_max * c->eas_ppm + 999999) / 1000000);
+}
+
+bpc_status bpc_build_eas(bpc_ctx* ctx, void* stream) {
+  if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
+  if (ctx->cfg.eas_ppm <= 0) return BPC_ERR_UNSUPPORTED;
+  if (!ctx->fitted) return BPC_ERR_NOT_FITTED;
+  cudaError_t e = bpc_launch_build_eas(ctx, (cudaStream_t)stream);
+  return e == cudaSuccess ? BPC_OK : cuda_fail(ctx, e);
+}
+
+bpc_status bpc_get_eas(bpc_ctx* ctx, float* sq_err_out, int32_t* set_out, int32_t* count_out, void* stream) {
+  if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
+  if (ctx->cfg.eas_ppm <= 0) return BPC_ERR_UNSUPPORTED;
+  cudaError_t e = cudaSuccess;
+  if (sq_err_out) e = cudaMemcpyAsync(sq_err_out, ctx->key_err, (size_t)ctx->units * ctx->cfg.n_max * 4, cudaMemcpyDeviceToDevice, (cudaStream_t)stream);
+  if (e == cudaSuccess && set_out) e = cudaMemcpyAsync(set_out, ctx->eas_idx, (size_t)ctx->units * ctx->eas_cap * 4, cudaMemcpyDeviceToDevice, (cudaStream_t)stream);
+  if (e == cudaSuccess && count_out) e = cudaMemcpyAsync(count_out, ctx->eas_cnt, (size_t)ctx->units * 4, cudaMemcpyDeviceToDevice, (cudaStream_t)stream);
+  return e == cudaSuccess ? BPC_OK : cuda_fail(ctx, e);
+}
+
 bpc_status bpc_append(bpc_ctx* ctx, const void* k_new, const void* v_new, void* k_cache, void* v_cache, uint64_t* codes,
                       void* stream) {
   if (ctx == nullptr || k_new == nullptr || v_new == nullptr || k_cache == nullptr || v_cache == nullptr || codes == nullptr)
@@ -311,6 +353,7 @@ static bpc_status decode_common(bpc_ctx* ctx, const void* k_new, const void* v_n
   p.unit_lens = ctx->unit_lens; p.out = out;
   p.k_new = k_new; p.v_new = v_new; p.k_cache_w = k_cache_w; p.v_cache_w = v_cache_w; p.codes_w = codes_w;
   p.unit_lens_w = ctx->unit_lens; p.gram = ctx->gram; p.residual_correction = c.residual_correction;
+  p.eas_idx = ctx->eas_idx; p.eas_cnt = ctx->eas_cnt; p.eas_cap = ctx->eas_cap;
   p.sel = sel_idx != nullptr ? sel_idx : ctx->sel_scratch;
   p.dbg_scores = ctx->dbg_scores; p.dbg_qweights = ctx->dbg_qweights; p.dbg_times = ctx->dbg_times;
   p.err = ctx->dev_err;
@@ -325,6 +368,9 @@ static bpc_status decode_common(bpc_ctx* ctx, const void* k_new, const void* v_n
   if (c.score_mode == BPC_SCORE_WEIGHTED7)
     e = c.kv_dtype == BPC_BF16 ? bpc_launch_decode_bf16_w7(ctx, p, (cudaStream_t)stream)
                                : bpc_launch_decode_f32_w7(ctx, p, (cudaStream_t)stream);
+  else if (c.eas_ppm > 0)
+    e = c.kv_dtype == BPC_BF16 ? bpc_launch_decode_bf16_eas(ctx, p, (cudaStream_t)stream)
+                               : bpc_launch_decode_f32_eas(ctx, p, (cudaStream_t)stream);
   else
     e = c.kv_dtype == BPC_BF16 ? bpc_launch_decode_bf16(ctx, p, (cudaStream_t)stream)
                                : bpc_launch_decode_f32(ctx, p, (cudaStream_t)stream);

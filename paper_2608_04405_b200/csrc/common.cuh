@@ -34,6 +34,10 @@ struct bpc_ctx {
   int32_t* host_lens;       // [batch] host shadow
   int32_t* sel_scratch;     // [units][n_max] int32
   int32_t* dev_err;         // device error word
+  float* key_err;           // [units][n_max] squared reconstruction errors (error-aware safeguard), or null
+  int32_t* eas_idx;         // [units][eas_cap] hard-to-hash set, ascending
+  int32_t* eas_cnt;         // [units] its size (0 until bpc_build_eas)
+  int eas_cap;
   int32_t* dbg_scores;      // caller buffers (may be null)
   int32_t* dbg_qweights;
   unsigned long long* dbg_times;
@@ -60,6 +64,9 @@ struct DecodeParams {
   int32_t* unit_lens_w;
   const float* gram;
   int residual_correction;
+  const int32_t* eas_idx;    // error-aware safeguard set (null when disabled)
+  const int32_t* eas_cnt;
+  int eas_cap;
   float* out;
   int32_t* sel;              // [units][n_max]
   int32_t* dbg_scores;
@@ -94,6 +101,9 @@ cudaError_t bpc_launch_fit(bpc_ctx* ctx, const void* k_cache, const float* v_sta
                            cudaStream_t stream, int* launches);
 size_t bpc_fit_workspace_bytes_impl(const bpc_config* cfg);
 size_t bpc_fit_codes_offset_impl(const bpc_config* cfg);
+
+// ---- error-aware safeguard set construction (prefill.cu)
+cudaError_t bpc_launch_build_eas(bpc_ctx* ctx, cudaStream_t stream);
 
 // ---- tensor-core encode (encode_tc.cu); returns cudaErrorNotSupported when the shape is not covered
 cudaError_t bpc_launch_encode_tc(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStream_t stream);

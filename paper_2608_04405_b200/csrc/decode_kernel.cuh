@@ -32,6 +32,8 @@ constexpr int kSegSlots = 40;       // 16-bit slots per segment (80 B: conflict-
 constexpr int kMaxBins = 2048;      // histogram bins (score keys are 0..nbins-1)
 constexpr int kIdxTile = 1024;      // selected indices staged at a time
 constexpr int kMaxPlanes = 10;
+constexpr int kEasMax = 16384;      // largest error-aware safeguard set per unit
+constexpr int kEasLocal = 1024;     // safeguard keys of one block kept in shared memory (larger slices stay in global)
 
 template <int GP, int MODE> struct PlaneCount {
   static constexpr int value = MODE == 0 ? (GP <= 2 ? 1 : (GP == 4 ? 2 : 3))
@@ -45,8 +47,11 @@ struct SmallState {
   uint32_t eq[BPC_MAX_CLUSTER];
   uint32_t wscan[32];
   double pmax[BPC_MAX_GROUP];
-  int T, cnt_gt, my_take, my_base, rsum, pad[3];
+  int T, cnt_gt, my_take, my_base, rsum, e0, e1, pad;
   uint32_t newcode[8];                   // code of the key appended by this launch
+  uint32_t eas_dup[kEasMax / 32];        // bit t - e0: safeguard key t was also selected by the hash search
+  int32_t eas_s[kEasLocal];              // this block's slice of the safeguard set (when it fits)
+  uint8_t stage_valid[32][4];            // per warp and gather stage: which of the 8 rows are real
 };
 
 template <typename KV> struct IsBf16 { static constexpr bool value = false; };
@@ -229,7 +234,9 @@ struct RowFragF32 {
   }
 };
 
-template <typename KV, int GP, int W32, int MODE>
+// EAS = 1 compiles the error-aware safeguard in (a static hard-to-hash set that is always attended); EAS = 0 is the
+// plain path with none of that code.
+template <typename KV, int GP, int W32, int MODE, int EAS>
 __global__ void __launch_bounds__((DecodeSmem<KV, GP, W32>::NT), 1)
 bpc_decode_kernel(const DecodeParams p) {
   typedef DecodeSmem<KV, GP, W32> L;
@@ -288,6 +295,16 @@ bpc_decode_kernel(const DecodeParams p) {
                                     : ((long long)n * (long long)p.budget_ppm + 999999LL) / 1000000LL;
   if (kk < 0) kk = 0;
   const int k = (int)(kk < (long long)n ? kk : (long long)n);
+  // Error-aware safeguard: the first `me` keys of the unit's static set S_err are always attended, the hash search
+  // fills the remaining kh = k - me places.
+  const int32_t* eas_u = nullptr;
+  int me_rt = 0;
+  if (EAS && p.eas_idx != nullptr) {
+    me_rt = min(min(p.eas_cnt[unit], p.eas_cap), min(k, kEasMax));
+    eas_u = p.eas_idx + (size_t)unit * p.eas_cap;
+  }
+  const int me = EAS ? me_rt : 0;                            // a compile-time zero without the safeguard
+  const int kh = k - me;
   // Keys per block.  In a fused launch the appending block (the last one with keys) scans with one warp less, so
   // it is given 15/16 of the others' share.
   const int chunk = (fused && CS > 1) ? ((int)(((long long)n * 16 + 16 * CS - 2) / (16 * CS - 1)) + 63) & ~63
@@ -383,8 +400,31 @@ bpc_decode_kernel(const DecodeParams p) {
     qf_s[GP * BPC_D + tid] = appender ? to_float(reinterpret_cast<const KV*>(p.k_new)[(size_t)unit * BPC_D + tid]) : 0.f;
   for (int i = tid; i < nbins; i += NT) hist[i] = 0u;
   if (tid < BPC_MAX_CLUSTER) { st->gt[tid] = 0u; st->eq[tid] = 0u; }
-  if (tid == 0) { st->rsum = 0; st->T = 0; st->cnt_gt = 0; }
+  if (tid == 0) { st->rsum = 0; st->T = 0; st->cnt_gt = 0; st->my_take = 0; st->my_base = 0; st->e0 = 0; st->e1 = 0; }
   __syncthreads();
+  if (me > 0) {
+    // safeguard keys inside this block's key range: the set is sorted, so their list positions [e0, e1) are the
+    // numbers of entries below the range's two ends (counted by the whole block in one coalesced sweep)
+    for (int i = tid; i < kEasMax / 32; i += NT) st->eas_dup[i] = 0u;
+    const int lo_key = min(n, rank * chunk), hi_key = min(n, lo_key + chunk);
+    int c_lo = 0, c_hi = 0;
+    for (int i = tid; i < me; i += NT) {
+      const int v = eas_u[i];
+      c_lo += v < lo_key;
+      c_hi += v < hi_key;
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+      c_lo += __shfl_xor_sync(0xffffffffu, c_lo, o);
+      c_hi += __shfl_xor_sync(0xffffffffu, c_hi, o);
+    }
+    if (lane == 0 && (c_lo | c_hi)) { atomicAdd(&st->e0, c_lo); atomicAdd(&st->e1, c_hi); }
+  }
+  __syncthreads();
+  const int e0 = me > 0 ? st->e0 : 0, e1 = me > 0 ? st->e1 : 0;
+  const bool eas_local = (e1 - e0) <= kEasLocal;
+  if (eas_local)
+    for (int i = tid; i < e1 - e0; i += NT) st->eas_s[i] = eas_u[e0 + i];
   {
     constexpr int PARTS = HPARTS, DS = HDS;
     const int j = tid % B, part = tid / B;
@@ -638,8 +678,8 @@ bpc_decode_kernel(const DecodeParams p) {
     }
     uint32_t above_all, above_low;
     block_excl_scan2<NT>(s_all, s_low, st->wscan, above_all, above_low);
-    if (bin >= 0 && above_all < (uint32_t)k && above_all + s_all >= (uint32_t)k) {
-      const int need = k - (int)above_all;                   // ties to take, cluster-wide (>= 1)
+    if (bin >= 0 && above_all < (uint32_t)kh && above_all + s_all >= (uint32_t)kh) {
+      const int need = kh - (int)above_all;                   // ties to take, cluster-wide (>= 1)
       const int lower_take = min(need, (int)s_low);          // ties granted to blocks of lower rank
       st->T = bin;
       st->cnt_gt = (int)above_all;
@@ -682,7 +722,7 @@ bpc_decode_kernel(const DecodeParams p) {
       uint32_t above = block_excl_scan<NT>(local, st->wscan, &total);
       for (int bin = hi - 1; bin >= lo; --bin) {
         const uint32_t c = tot[bin];
-        if (above < (uint32_t)k && above + c >= (uint32_t)k) { st->T = bin; st->cnt_gt = (int)above; }
+        if (above < (uint32_t)kh && above + c >= (uint32_t)kh) { st->T = bin; st->cnt_gt = (int)above; }
         above += c;
       }
     }
@@ -712,7 +752,7 @@ bpc_decode_kernel(const DecodeParams p) {
     __syncthreads();
   }
   int T_exact = T;
-  if (hsh > 0) {
+  if (hsh > 0 && kh > 0) {
     // Weighted scores have more distinct values than histogram bins: the search above found the coarse bin
     // that holds the k-th score.  A second, small histogram over the low bits of the keys inside that bin (again
     // summed across the cluster) yields the exact threshold and corrects the per-block counts.
@@ -744,7 +784,7 @@ bpc_decode_kernel(const DecodeParams p) {
         if (lane + o < 32) incl += v;
       }
       const uint32_t above = incl - f;
-      const uint32_t need_c = (uint32_t)(k - st->cnt_gt);    // keys still to take from the coarse bin (>= 1)
+      const uint32_t need_c = (uint32_t)(kh - st->cnt_gt);    // keys still to take from the coarse bin (>= 1)
       const bool mine = above < need_c && above + f >= need_c;
       const int vstar = __ffs(__ballot_sync(0xffffffffu, mine)) - 1;
       const uint32_t above_star = __shfl_sync(0xffffffffu, above, vstar);
@@ -765,7 +805,7 @@ bpc_decode_kernel(const DecodeParams p) {
     T_exact = st->T;
   }
   if (!fast_sel && tid == 0) {
-    const int need = k - st->cnt_gt;                         // ties to take, cluster-wide (>= 1)
+    const int need = kh - st->cnt_gt;                        // ties to take, cluster-wide (>= 1)
     int tie_base = 0, out_base = 0;
     for (int r = 0; r < CS; ++r) {
       int take = need - tie_base;
@@ -791,7 +831,19 @@ bpc_decode_kernel(const DecodeParams p) {
     constexpr int SPT = 4;                                   // most consecutive segments one thread takes per pass
     const int spt = min(SPT, (nseg + NT - 1) / NT);
     int run_gt = 0, run_eq = 0;
-    for (int s0 = 0; s0 < nseg; s0 += NT * spt) {
+    // a selected key that also belongs to the safeguard set is flagged there, so that it is attended once
+    auto mark_dup = [&](int gi) {
+      if (EAS && me > 0) {
+        int a = 0, b2 = e1 - e0;
+        while (a < b2) {
+          const int mid = (a + b2) >> 1;
+          const int v = eas_local ? st->eas_s[mid] : eas_u[e0 + mid];
+          if (v < gi) a = mid + 1; else b2 = mid;
+        }
+        if (a < e1 - e0 && (eas_local ? st->eas_s[a] : eas_u[e0 + a]) == gi) atomicOr(&st->eas_dup[a >> 5], 1u << (a & 31));
+      }
+    };
+    for (int s0 = 0; s0 < nseg && kh > 0; s0 += NT * spt) {
       uint32_t M[SPT], Mgt[SPT];                             // bit j: key j of the segment is >= T / > T
       int cgt = 0, ceq = 0;
 #pragma unroll
@@ -843,10 +895,12 @@ bpc_decode_kernel(const DecodeParams p) {
           while (rem) {
             const int j = __ffs(rem) - 1;
             rem &= rem - 1;
+            const int gi = c0 + seg * kSegKeys + j;
             if ((Mgt[q] >> j) & 1u) {
-              sel_u[pos++] = c0 + seg * kSegKeys + j;
+              sel_u[pos++] = gi;
+              mark_dup(gi);
             } else {
-              if (eqb < my_take) sel_u[pos++] = c0 + seg * kSegKeys + j;
+              if (eqb < my_take) { sel_u[pos++] = gi; mark_dup(gi); }
               ++eqb;
             }
           }
@@ -856,13 +910,26 @@ bpc_decode_kernel(const DecodeParams p) {
       run_eq += (int)(total >> 16);
     }
   }
+  if (me > 0) {
+    __syncthreads();                                         // all duplicate flags of this block are set
+    for (int t = tid; t < e1 - e0; t += NT) {
+      const bool dup = (st->eas_dup[t >> 5] >> (t & 31)) & 1u;
+      sel_u[kh + e0 + t] = dup ? -1 : (eas_local ? st->eas_s[t] : eas_u[e0 + t]);
+    }
+  }
   BPC_STAMP(3);
   __threadfence();
   cluster.sync();                                            // the unit's index list is complete and visible
   BPC_STAMP(4);
 
   // ------------------------------------------------------------------ phase 3: gathered attention
-  const int lo = (int)(((long long)k * rank) / CS), hi = (int)(((long long)k * (rank + 1)) / CS);
+  // this block attends rows [lo, hi) of the hash list and the safeguard keys that lie in its own key range
+  const int lo = (int)(((long long)kh * rank) / CS), hi = (int)(((long long)kh * (rank + 1)) / CS);
+  const int nh = hi - lo, ne = e1 - e0;                      // rows from the two sources
+  auto row_index = [&](int qrow) -> int {                    // qrow in [0, nh + ne): cache row, or -1 for a duplicate
+    if (!EAS) return sel_u[lo + qrow];
+    return qrow < nh ? sel_u[lo + qrow] : sel_u[kh + e0 + (qrow - nh)];
+  };
   const size_t rstride = (size_t)p.row_stride * sizeof(KV);   // bytes between consecutive cache rows
   const unsigned char* Ku = reinterpret_cast<const unsigned char*>(p.k_cache) + (size_t)unit * (size_t)p.n_max * rstride;
   const unsigned char* Vu = reinterpret_cast<const unsigned char*>(p.v_cache) + (size_t)unit * (size_t)p.n_max * rstride;
@@ -900,15 +967,23 @@ bpc_decode_kernel(const DecodeParams p) {
     // reads are conflict-free), keeps NS-1 blocks in flight and multiplies the oldest one.
     constexpr int WSTG = 8 * 2 * ROWB;                       // bytes of one 8-row stage (K rows, then V rows)
     unsigned char* wst = stg + (size_t)warp * NS * WSTG;
-    const int nblk = (hi - lo + 7) >> 3;
+    const int nrows = nh + ne;
+    const int nblk = (nrows + 7) >> 3;
     const int isv = lane >> 4, ch = lane & 15;
     const unsigned char* srcbase = (isv ? Vu : Ku) + (size_t)ch * 16;
     auto issue = [&](int bi) {
       const int blk = warp + bi * NW;
       if (blk < nblk) {
-        const int rbase = lo + 8 * blk;
+        const int rbase = 8 * blk;
         int myidx = -1;
-        if (lane < 8 && rbase + lane < hi) myidx = min(max(sel_u[rbase + lane], 0), p.n_max - 1);
+        if (lane < 8 && rbase + lane < nrows) {
+          myidx = row_index(rbase + lane);
+          if (myidx >= 0) myidx = min(myidx, p.n_max - 1);
+        }
+        if (EAS) {   // which of the 8 rows are real (not past the end, not a duplicate of a hash-selected key)
+          const uint32_t vm = __ballot_sync(0xffffffffu, myidx >= 0) & 0xffu;
+          if (lane == 0) st->stage_valid[warp][bi % NS] = (uint8_t)vm;
+        }
         unsigned char* dst = wst + (size_t)(bi % NS) * WSTG + (size_t)isv * (8 * ROWB);
 #pragma unroll
         for (int it = 0; it < 8; ++it) {
@@ -930,7 +1005,9 @@ bpc_decode_kernel(const DecodeParams p) {
       if (NS == 2) cp_async_wait<0>(); else cp_async_wait<1>();   // this lane's copies for block bi have landed
       __syncwarp();                                          // ... and every lane's
       issue(bi + NS - 1);                                    // refill the stage consumed in the previous round
-      const int rbase = lo + 8 * (warp + bi * NW);
+      const int rbase_c = 8 * (warp + bi * NW);
+      const uint32_t vmask = EAS ? (uint32_t)st->stage_valid[warp][bi % NS]
+                                 : (rbase_c + 8 <= nrows ? 0xffu : ((1u << (nrows - rbase_c)) - 1u));
       const unsigned char* ks = wst + (size_t)(bi % NS) * WSTG;
       const unsigned char* vs = ks + 8 * ROWB;
       float s[4] = {0.f, 0.f, 0.f, 0.f};
@@ -941,7 +1018,7 @@ bpc_decode_kernel(const DecodeParams p) {
         mma_qk(s, qa0[2 * jj], qa2[2 * jj], b[0], b[1]);
         mma_qk(s, qa0[2 * jj + 1], qa2[2 * jj + 1], b[2], b[3]);
       }
-      const bool v0 = rbase + 2 * t < hi, v1 = rbase + 2 * t + 1 < hi;
+      const bool v0 = (vmask >> (2 * t)) & 1u, v1 = (vmask >> (2 * t + 1)) & 1u;
       const float s0 = v0 ? s[0] * scale2 : -1e30f, s1 = v1 ? s[1] * scale2 : -1e30f;
       float tmax = fmaxf(s0, s1);
       tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
@@ -1032,10 +1109,13 @@ bpc_decode_kernel(const DecodeParams p) {
         }
       }
     };
-    for (int t0 = lo; t0 < hi; t0 += kIdxTile) {
-      const int tn = min(kIdxTile, hi - t0);
+    for (int t0 = 0; t0 < nh + ne; t0 += kIdxTile) {         // virtual rows: hash slice, then own safeguard keys
+      const int tn = min(kIdxTile, nh + ne - t0);
       __syncthreads();
-      for (int i = tid; i < tn; i += NT) idx_s[i] = min(max(sel_u[t0 + i], 0), p.n_max - 1);
+      for (int i = tid; i < tn; i += NT) {
+        const int v = row_index(t0 + i);
+        idx_s[i] = v < 0 ? -1 : min(v, p.n_max - 1);
+      }
       __syncthreads();
       const int ntile = (tn + TR - 1) / TR;
       auto issue = [&](int tile) {
@@ -1045,7 +1125,7 @@ bpc_decode_kernel(const DecodeParams p) {
           for (int c = tid; c < TR * 2 * CPR; c += NT) {
             const int row = c / (2 * CPR), within = c % (2 * CPR);
             const int isv = within / CPR, ch = within % CPR;
-            if (r0 + row < tn) {
+            if (r0 + row < tn && idx_s[r0 + row] >= 0) {
               const size_t off = (size_t)idx_s[r0 + row] * rstride + (size_t)ch * 16;
               cp_async16(dst + (size_t)row * 2 * ROWB + isv * ROWB + ch * 16, (isv ? Vu : Ku) + off);
             }
@@ -1065,7 +1145,7 @@ bpc_decode_kernel(const DecodeParams p) {
           RowFragF32 kf, vf;
           kf.load(src + (size_t)r * 2 * ROWB, hl);
           vf.load(src + (size_t)r * 2 * ROWB + ROWB, hl);
-          process(kf, vf, r0 + r < tn);
+          process(kf, vf, r0 + r < tn && idx_s[r0 + r] >= 0);
         }
       }
       cp_async_wait<0>();

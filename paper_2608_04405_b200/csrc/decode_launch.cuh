@@ -6,9 +6,9 @@ namespace bpcdev {
 
 // The shared-memory ceiling is always raised to the device's opt-in maximum, so contexts with different
 // n_max can share one kernel instance.
-template <typename KV, int GP, int W32, int MODE>
+template <typename KV, int GP, int W32, int MODE, int EAS>
 static cudaError_t configure_kernel(int device) {
-  auto kern = bpc_decode_kernel<KV, GP, W32, MODE>;
+  auto kern = bpc_decode_kernel<KV, GP, W32, MODE, EAS>;
   int optin = 0;
   cudaError_t e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
   if (e != cudaSuccess) return e;
@@ -17,7 +17,7 @@ static cudaError_t configure_kernel(int device) {
   return cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
 }
 
-template <typename KV, int GP, int W32, int MODE>
+template <typename KV, int GP, int W32, int MODE, int EAS>
 static cudaError_t launch_one(bpc_ctx* ctx, const DecodeParams& p_in, cudaStream_t stream) {
   typedef DecodeSmem<KV, GP, W32> L;
   DecodeParams p = p_in;
@@ -28,7 +28,7 @@ static cudaError_t launch_one(bpc_ctx* ctx, const DecodeParams& p_in, cudaStream
   const size_t smem = L(p.chunk_cap, p.nbins, p.stages).total;
   if (smem > (size_t)optin) return cudaErrorInvalidConfiguration;
   if (ctx->decode_smem_set == 0) {                          // function attributes are sticky: set them once
-    e = configure_kernel<KV, GP, W32, MODE>(ctx->device);
+    e = configure_kernel<KV, GP, W32, MODE, EAS>(ctx->device);
     if (e != cudaSuccess) return e;
     ctx->decode_smem_set = 1;
   }
@@ -48,12 +48,12 @@ static cudaError_t launch_one(bpc_ctx* ctx, const DecodeParams& p_in, cudaStream
   at[1].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = at;
   lc.numAttrs = ctx->use_pdl ? 2 : 1;
-  return cudaLaunchKernelEx(&lc, bpc_decode_kernel<KV, GP, W32, MODE>, p);
+  return cudaLaunchKernelEx(&lc, bpc_decode_kernel<KV, GP, W32, MODE, EAS>, p);
 }
 
 // Largest cluster size (power of two) the device can schedule with a full-size block, and the number of
 // score keys one block can hold next to a two-stage gather ring.
-template <typename KV, int GP, int W32, int MODE>
+template <typename KV, int GP, int W32, int MODE, int EAS>
 static cudaError_t limits_one(const bpc_ctx* ctx, int nbins, int* max_cluster, int* chunk_cap, size_t* smem_bytes) {
   typedef DecodeSmem<KV, GP, W32> L;
   int dev = ctx->device, optin = 0;
@@ -70,7 +70,7 @@ static cudaError_t limits_one(const bpc_ctx* ctx, int nbins, int* max_cluster, i
     // max_cluster[0] = largest schedulable cluster size; max_cluster[1 + log2(cs)] = clusters of that size that
     // can be resident at once (a grid with more clusters than that runs in several waves)
     int best = 1;
-    e = configure_kernel<KV, GP, W32, MODE>(dev);
+    e = configure_kernel<KV, GP, W32, MODE, EAS>(dev);
     if (e != cudaSuccess) return e;
     for (int cs = 1, li = 0; cs <= BPC_MAX_CLUSTER; cs *= 2, ++li) {
       cudaLaunchConfig_t lc = {};
@@ -82,7 +82,7 @@ static cudaError_t limits_one(const bpc_ctx* ctx, int nbins, int* max_cluster, i
       at[0].val.clusterDim.x = (unsigned)cs; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
       lc.attrs = at; lc.numAttrs = 1;
       int nclusters = 0;
-      cudaError_t q = cudaOccupancyMaxActiveClusters(&nclusters, bpc_decode_kernel<KV, GP, W32, MODE>, &lc);
+      cudaError_t q = cudaOccupancyMaxActiveClusters(&nclusters, bpc_decode_kernel<KV, GP, W32, MODE, EAS>, &lc);
       if (q != cudaSuccess) { (void)cudaGetLastError(); nclusters = 0; }
       max_cluster[1 + li] = nclusters;
       if (nclusters >= 1) best = cs;
@@ -92,28 +92,28 @@ static cudaError_t limits_one(const bpc_ctx* ctx, int nbins, int* max_cluster, i
   return cudaSuccess;
 }
 
-#define BPC_DISPATCH_W(KV, GP, MODE, FN, ...)                                        \
+#define BPC_DISPATCH_W(KV, GP, MODE, EAS, FN, ...)                                   \
   switch (ctx->cfg.code_bits) {                                                      \
-    case 64:  return FN<KV, GP, 2, MODE>(__VA_ARGS__);                               \
-    case 128: return FN<KV, GP, 4, MODE>(__VA_ARGS__);                               \
-    case 256: return FN<KV, GP, 8, MODE>(__VA_ARGS__);                               \
+    case 64:  return FN<KV, GP, 2, MODE, EAS>(__VA_ARGS__);                          \
+    case 128: return FN<KV, GP, 4, MODE, EAS>(__VA_ARGS__);                          \
+    case 256: return FN<KV, GP, 8, MODE, EAS>(__VA_ARGS__);                          \
     default:  return cudaErrorInvalidValue;                                          \
   }
 
-#define BPC_DISPATCH_G(KV, MODE, FN, ...)                                            \
-  if (ctx->group == 1)      { BPC_DISPATCH_W(KV, 1, MODE, FN, __VA_ARGS__) }         \
-  else if (ctx->group == 2) { BPC_DISPATCH_W(KV, 2, MODE, FN, __VA_ARGS__) }         \
-  else if (ctx->group <= 4) { BPC_DISPATCH_W(KV, 4, MODE, FN, __VA_ARGS__) }         \
-  else                      { BPC_DISPATCH_W(KV, 8, MODE, FN, __VA_ARGS__) }
+#define BPC_DISPATCH_G(KV, MODE, EAS, FN, ...)                                       \
+  if (ctx->group == 1)      { BPC_DISPATCH_W(KV, 1, MODE, EAS, FN, __VA_ARGS__) }    \
+  else if (ctx->group == 2) { BPC_DISPATCH_W(KV, 2, MODE, EAS, FN, __VA_ARGS__) }    \
+  else if (ctx->group <= 4) { BPC_DISPATCH_W(KV, 4, MODE, EAS, FN, __VA_ARGS__) }    \
+  else                      { BPC_DISPATCH_W(KV, 8, MODE, EAS, FN, __VA_ARGS__) }
 
 // One translation unit per (cache dtype, score mode): MODE 0 = Hamming, MODE 1 = sign + 7 magnitude planes.
-template <typename KV, int MODE>
+template <typename KV, int MODE, int EAS>
 static cudaError_t launch_dtype(bpc_ctx* ctx, const DecodeParams& p, cudaStream_t stream) {
-  BPC_DISPATCH_G(KV, MODE, launch_one, ctx, p, stream)
+  BPC_DISPATCH_G(KV, MODE, EAS, launch_one, ctx, p, stream)
 }
-template <typename KV, int MODE>
+template <typename KV, int MODE, int EAS>
 static cudaError_t limits_dtype(const bpc_ctx* ctx, int nbins, int* max_cluster, int* chunk_cap, size_t* smem) {
-  BPC_DISPATCH_G(KV, MODE, limits_one, ctx, nbins, max_cluster, chunk_cap, smem)
+  BPC_DISPATCH_G(KV, MODE, EAS, limits_one, ctx, nbins, max_cluster, chunk_cap, smem)
 }
 
 }  // namespace bpcdev

@@ -84,21 +84,22 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[N]) {
 // On entry t[j] already carries the corrections of all earlier blocks; on exit `word` holds the 32 signs.
 template <int I>
 struct DiagSweep {
-  static __device__ __forceinline__ void run(float (&t)[32], uint32_t& word, const float* g_diag, int ld, int rc) {
+  static __device__ __forceinline__ void run(float (&t)[32], uint32_t& word, float& abs_sum, const float* g_diag, int ld, int rc) {
     const bool pos = t[I] >= 0.f;
     word |= (pos ? 1u : 0u) << I;
+    abs_sum += fabsf(t[I]);
     if (rc) {
       const float u = pos ? 1.f : -1.f;
       const float* gi = g_diag + I * ld;
 #pragma unroll
       for (int j = I + 1; j < 32; ++j) t[j] = fmaf(-u, gi[j], t[j]);
     }
-    DiagSweep<I + 1>::run(t, word, g_diag, ld, rc);
+    DiagSweep<I + 1>::run(t, word, abs_sum, g_diag, ld, rc);
   }
 };
 template <>
 struct DiagSweep<32> {
-  static __device__ __forceinline__ void run(float (&)[32], uint32_t&, const float*, int, int) {}
+  static __device__ __forceinline__ void run(float (&)[32], uint32_t&, float&, const float*, int, int) {}
 };
 
 // byte offset of 16-byte chunk `ch` (0..15) of row `r` inside a [rows x 128 channels] bf16 operand tile:
@@ -111,7 +112,8 @@ template <int NBITS>
 __global__ void __launch_bounds__(kThreads, 1)
 encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16* __restrict__ Ph, const float* __restrict__ gram,
                  const int32_t* __restrict__ unit_lens, uint64_t* __restrict__ codes, int32_t* __restrict__ err,
-                 int n_kv_heads, int n_max, int row_stride, int shared_sets, int residual_correction, int blocks_per_unit) {
+                 int n_kv_heads, int n_max, int row_stride, int shared_sets, int residual_correction, int blocks_per_unit,
+                 float* __restrict__ key_err) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   // the swizzled operand tiles need 1024-byte alignment in the shared address space
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -153,6 +155,9 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = tmem_base_s;
+  float trace_g = 0.f;
+  if (key_err != nullptr)
+    for (int i = 0; i < NBITS; ++i) trace_g += g_s[i * NBITS + i];
 
   const unsigned char* kbase = reinterpret_cast<const unsigned char*>(k_cache) + (size_t)unit * n_max * (size_t)row_stride * 2;
   auto load_tile = [&](int tile, unsigned char* dst) {
@@ -200,6 +205,7 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
     // Column blocks of 32 bits: pull the block out of tensor memory, apply the corrections of all earlier
     // bits (t_j -= u_i G_ij, G rows are broadcast reads from shared memory), then sweep the block itself.
     uint32_t words[NBITS / 32];
+    float abs_sum = 0.f;                                     // sum of |t_i| at decision time (for Eq. 8)
 #pragma unroll
     for (int cb = 0; cb < NBITS / 32; ++cb) {
       float t[32];
@@ -225,7 +231,7 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
         }
       }
       uint32_t word = 0u;
-      DiagSweep<0>::run(t, word, g_s + (size_t)(32 * cb) * NBITS + 32 * cb, NBITS, residual_correction);
+      DiagSweep<0>::run(t, word, abs_sum, g_s + (size_t)(32 * cb) * NBITS + 32 * cb, NBITS, residual_correction);
       words[cb] = word;
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -240,6 +246,20 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
       issue_mma(a_s[(it + 1) & 1]);
     }
     const int key = tile * kTileKeys + tid;
+    if (key_err != nullptr && key < n) {
+      // squared reconstruction error (Eq. 8) from the sweep: ||k - hP||^2 = ||k||^2 - 2 sum|t_i| + trace(G);
+      // the key's channels are still in this tile's operand buffer
+      const unsigned char* arow = a_s[it & 1];
+      float k2 = 0.f;
+#pragma unroll
+      for (int ch = 0; ch < 16; ++ch) {
+        const uint4 w = *reinterpret_cast<const uint4*>(arow + sw128_offset(kTileKeys, tid, ch));
+        const float f0 = bf16_lo(w.x), f1 = bf16_hi(w.x), f2 = bf16_lo(w.y), f3 = bf16_hi(w.y);
+        const float f4 = bf16_lo(w.z), f5 = bf16_hi(w.z), f6 = bf16_lo(w.w), f7 = bf16_hi(w.w);
+        k2 += (f0 * f0 + f1 * f1) + (f2 * f2 + f3 * f3) + (f4 * f4 + f5 * f5) + (f6 * f6 + f7 * f7);
+      }
+      key_err[(size_t)unit * n_max + key] = fmaxf(0.f, k2 - 2.f * abs_sum + trace_g);
+    }
     if (key < n) {
       uint32_t* dst = reinterpret_cast<uint32_t*>(codes + ((size_t)unit * n_max + key) * (NBITS / 64));
       if (NBITS == 64) {
@@ -272,7 +292,7 @@ cudaError_t launch(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStrea
   const dim3 grid(bpu, ctx->units);
   encode_tc_kernel<NBITS><<<grid, kThreads, smem, stream>>>(
       (const __nv_bfloat16*)k_cache, (const __nv_bfloat16*)ctx->P_h, ctx->gram, ctx->unit_lens, codes, ctx->dev_err,
-      c.n_kv_heads, c.n_max, ctx->row_stride, c.hash_sets != ctx->units, c.residual_correction, bpu);
+      c.n_kv_heads, c.n_max, ctx->row_stride, c.hash_sets != ctx->units, c.residual_correction, bpu, ctx->key_err);
   return cudaGetLastError();
 }
 

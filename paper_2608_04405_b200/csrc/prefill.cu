@@ -51,7 +51,7 @@ template <typename KV>
 __global__ void __launch_bounds__(kEncThreads)
 encode_simple_kernel(const KV* __restrict__ k_cache, const float* __restrict__ Phf, const float* __restrict__ gram,
                      const int32_t* __restrict__ unit_lens, uint64_t* __restrict__ codes, int n_kv_heads, int n_max,
-                     int row_stride, int b, int shared_sets, int residual_correction) {
+                     int row_stride, int b, int shared_sets, int residual_correction, float* __restrict__ key_err) {
   extern __shared__ __align__(16) unsigned char smem[];
   float* ps = reinterpret_cast<float*>(smem);                       // [128 rows of P][128]
   float* ts = ps + 128 * BPC_D;                                      // [b][kEncThreads]
@@ -90,9 +90,11 @@ encode_simple_kernel(const KV* __restrict__ k_cache, const float* __restrict__ P
   }
   uint32_t* dst = reinterpret_cast<uint32_t*>(codes + ((size_t)unit * n_max + (live ? key : 0)) * (b / 64));
   uint32_t word = 0;
+  double abs_sum = 0.0;                                              // sum of |t_i| at decision time
   for (int i = 0; i < b; ++i) {
     const float ti = ts[(size_t)i * kEncThreads + threadIdx.x];
     const bool pos = ti >= 0.f;
+    abs_sum += (double)fabsf(ti);
     word |= (pos ? 1u : 0u) << (i & 31);
     if ((i & 31) == 31) {
       if (live) dst[i >> 5] = word;
@@ -103,6 +105,14 @@ encode_simple_kernel(const KV* __restrict__ k_cache, const float* __restrict__ P
       const float* gi = Gset + (size_t)i * b;
       for (int j = i + 1; j < b; ++j) ts[(size_t)j * kEncThreads + threadIdx.x] -= u * __ldg(gi + j);
     }
+  }
+  if (key_err != nullptr && live) {
+    // squared reconstruction error (Eq. 8) from the sweep: ||k - hP||^2 = ||k||^2 - 2 sum|t_i| + trace(G)
+    double k2 = 0.0, trg = 0.0;
+#pragma unroll
+    for (int c = 0; c < BPC_D; ++c) k2 = fma((double)kr[c], (double)kr[c], k2);
+    for (int i = 0; i < b; ++i) trg += (double)__ldg(Gset + (size_t)i * b + i);
+    key_err[(size_t)unit * n_max + key] = (float)fmax(0.0, k2 - 2.0 * abs_sum + trg);
   }
 }
 
@@ -275,6 +285,68 @@ __global__ void fit_reduce_kernel(const float* __restrict__ partials, float* __r
   P[((size_t)unit * b + it) * BPC_D + c] = n > 0 ? (float)(s / (double)n) : 0.f;
 }
 
+// --------------------------------------------------------------------------- error-aware safeguard set
+// One block per unit: the m keys with the largest squared reconstruction error, ties to the lowest index, written
+// in ascending index order.  The errors are non-negative floats, so their bit patterns order like unsigned
+// integers: a 4-pass radix select (8 bits per pass) finds the m-th largest pattern, then one ordered pass compacts.
+constexpr int kEasThreads = 1024;
+
+__global__ void __launch_bounds__(kEasThreads)
+build_eas_kernel(const float* __restrict__ key_err, const int32_t* __restrict__ unit_lens, int32_t* __restrict__ eas_idx,
+                 int32_t* __restrict__ eas_cnt, int n_max, int eas_ppm, int eas_cap) {
+  __shared__ uint32_t hist[256];
+  __shared__ uint32_t wsum[kEasThreads / 32];
+  __shared__ uint32_t s_prefix, s_need, s_run_gt, s_run_eq;
+  const int unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n = min(unit_lens[unit], n_max);
+  int m = (int)(((long long)n * eas_ppm + 999999) / 1000000);
+  m = min(min(m, n), eas_cap);
+  const uint32_t* e = reinterpret_cast<const uint32_t*>(key_err + (size_t)unit * n_max);
+  if (m <= 0) { if (tid == 0) eas_cnt[unit] = 0; return; }
+  if (tid == 0) { s_prefix = 0u; s_need = (uint32_t)m; }
+  __syncthreads();
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    if (tid < 256) hist[tid] = 0u;
+    __syncthreads();
+    const uint32_t prefix = s_prefix, himask = shift == 24 ? 0u : ~((1u << (shift + 8)) - 1u);
+    for (int i = tid; i < n; i += kEasThreads) {
+      const uint32_t v = e[i];
+      if ((v & himask) == prefix) atomicAdd(&hist[(v >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (tid == 0) {                                          // 256 bins: a serial walk from the top is cheap enough
+      uint32_t need = s_need, acc = 0;
+      int d = 255;
+      for (; d > 0; --d) { if (acc + hist[d] >= need) break; acc += hist[d]; }
+      s_need = need - acc;                                   // still to take among values with this digit
+      s_prefix = prefix | ((uint32_t)d << shift);
+    }
+    __syncthreads();
+  }
+  const uint32_t thr = s_prefix, need_eq = s_need;           // take every v > thr and the first need_eq with v == thr
+  if (tid == 0) { s_run_gt = 0u; s_run_eq = 0u; }
+  __syncthreads();
+  int32_t* out = eas_idx + (size_t)unit * eas_cap;
+  for (int i0 = 0; i0 < n; i0 += kEasThreads) {
+    const int i = i0 + tid;
+    const uint32_t v = i < n ? e[i] : 0u;
+    const bool gt = i < n && v > thr, eq = i < n && v == thr;
+    const uint32_t bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
+    if (lane == 0) wsum[warp] = (uint32_t)__popc(bg) | ((uint32_t)__popc(be) << 16);
+    __syncthreads();
+    uint32_t before = 0, total = 0;
+    for (int w = 0; w < kEasThreads / 32; ++w) { if (w < warp) before += wsum[w]; total += wsum[w]; }
+    const uint32_t lt = (1u << lane) - 1u;
+    const uint32_t gt_before = s_run_gt + (before & 0xffffu) + (uint32_t)__popc(bg & lt);
+    const uint32_t eq_before = s_run_eq + (before >> 16) + (uint32_t)__popc(be & lt);
+    if (gt || (eq && eq_before < need_eq)) out[gt_before + min(eq_before, need_eq)] = i;
+    __syncthreads();
+    if (tid == 0) { s_run_gt += total & 0xffffu; s_run_eq += total >> 16; }
+    __syncthreads();
+  }
+  if (tid == 0) eas_cnt[unit] = m;
+}
+
 }  // namespace
 
 // =========================================================================== host launchers
@@ -304,13 +376,13 @@ cudaError_t bpc_launch_encode_simple(bpc_ctx* ctx, const void* k_cache, uint64_t
     if (e != cudaSuccess) return e;
     encode_simple_kernel<__nv_bfloat16><<<grid, kEncThreads, smem, stream>>>(
         (const __nv_bfloat16*)k_cache, ctx->P_hf, ctx->gram, ctx->unit_lens, codes, c.n_kv_heads, c.n_max, ctx->row_stride, b, shared_sets,
-        c.residual_correction);
+        c.residual_correction, ctx->key_err);
   } else {
     e = cudaFuncSetAttribute(encode_simple_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     encode_simple_kernel<float><<<grid, kEncThreads, smem, stream>>>(
         (const float*)k_cache, ctx->P_hf, ctx->gram, ctx->unit_lens, codes, c.n_kv_heads, c.n_max, ctx->row_stride, b, shared_sets,
-        c.residual_correction);
+        c.residual_correction, ctx->key_err);
   }
   ctx->launches += 1;
   return cudaGetLastError();
@@ -378,5 +450,12 @@ cudaError_t bpc_launch_fit(bpc_ctx* ctx, const void* k_cache, const float* v_sta
     fit_reduce_kernel<<<ctx->units, BPC_D, 0, stream>>>(partials, ctx->P, ctx->unit_lens, c.n_max, c.code_bits, it, bpu);
     *launches += 2;
   }
+  return cudaGetLastError();
+}
+
+cudaError_t bpc_launch_build_eas(bpc_ctx* ctx, cudaStream_t stream) {
+  build_eas_kernel<<<ctx->units, kEasThreads, 0, stream>>>(ctx->key_err, ctx->unit_lens, ctx->eas_idx, ctx->eas_cnt,
+                                                           ctx->cfg.n_max, ctx->cfg.eas_ppm, ctx->eas_cap);
+  ctx->launches += 1;
   return cudaGetLastError();
 }

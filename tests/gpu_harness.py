@@ -39,7 +39,7 @@ class Session:
     """A workload on the GPU with its library context, fitted and encoded."""
 
     def __init__(self, spec: WorkloadSpec, gen_device: str = "cpu", salt: int = 0, cluster_size: int = 0,
-                 extra_rows=None, interleaved: bool = False, score_mode: int = 0):
+                 extra_rows=None, interleaved: bool = False, score_mode: int = 0, eas_ppm: int = 0):
         self.spec = spec
         self.w = Workload(spec, device=gen_device, extra_rows=extra_rows, salt=salt)
         dev = "cuda"
@@ -54,7 +54,8 @@ class Session:
         self.v_star = self.w.v_star.to(dev)
         self.cfg = B.make_config(spec.batch, spec.n_q_heads, spec.n_kv_heads, self.w.n_max, spec.code_bits,
                                  spec.torch_dtype, kv_row_stride=2 * spec.head_dim if interleaved else 0,
-                                 score_mode=score_mode)
+                                 score_mode=score_mode, eas_ppm=eas_ppm)
+        self.s_err = None
         self.ctx = B.Context(self.cfg)
         if cluster_size:
             self.ctx.set_cluster_size(cluster_size)
@@ -151,6 +152,38 @@ def check_encode(sess: Session, units, report: dict, max_keys: int = 0, key_slic
             assert np.array_equal(ref, bits)
 
 
+def check_eas(sess: Session, units, report: dict):
+    """bpc_build_eas: squared reconstruction errors (Eq. 8) against the fp64 residual norms, and the hard-to-hash set
+    as a valid top-m of them (keys whose errors differ by less than the fp32 noise of the sweep may swap)."""
+    s = sess.spec
+    sess.ctx.build_eas()
+    torch.cuda.synchronize()
+    err, idx, cnt = sess.ctx.get_eas()
+    torch.cuda.synchronize()
+    sess.s_err = [idx[u, :int(cnt[u])].cpu().numpy().astype(np.int64) for u in range(sess.units)]
+    for u in units:
+        bi, h, n = sess.unit_views(u)
+        K = _np64(sess.k_cache[bi, h, :n])
+        Ph = _np64(sess.Ph[u if sess.cfg.hash_sets == sess.units else h])
+        bits = codes_to_bits(sess.codes[bi, h, :n], s.code_bits)
+        ref = np.linalg.norm(K - (2.0 * bits - 1.0) @ Ph, axis=1) ** 2          # from the library's own codes
+        got = err[u, :n].double().cpu().numpy()
+        scale = (np.linalg.norm(K, axis=1) ** 2).max()
+        assert np.abs(got - ref).max() <= 2e-5 * scale, "squared reconstruction errors differ: %g" % np.abs(got - ref).max()
+        m = -(-n * sess.cfg.eas_ppm // 1000000)
+        mine = sess.s_err[u]
+        assert len(mine) == m and np.all(np.diff(mine) > 0) and (len(mine) == 0 or (mine[0] >= 0 and mine[-1] < n))
+        # exactly the top-m of the library's own error values, ties to the lowest index
+        assert np.array_equal(mine, O.eas_set(got, m)), "hard-to-hash set is not the top-m of the recorded errors"
+        # and a valid top-m of the fp64 errors up to the fp32 noise
+        thr = np.sort(ref)[::-1][m - 1] if m > 0 else np.inf
+        tol = 4e-5 * scale
+        assert np.all(ref[mine] >= thr - tol)
+        rest = np.setdiff1d(np.arange(n), mine)
+        assert np.all(ref[rest] <= thr + tol)
+        report["eas_keys"] = report.get("eas_keys", 0) + m
+
+
 def check_decode(sess: Session, q: torch.Tensor, units, report: dict, budget_ppm=None, budget_count=0, append=None):
     """One decode step through the library, checked stage by stage for the given units.
 
@@ -184,7 +217,12 @@ def check_decode(sess: Session, q: torch.Tensor, units, report: dict, budget_ppm
     # a second call without the parity buffers and without a caller index list must give the same output
     out2 = sess.ctx.decode_attn(q, sess.k_cache, sess.v_cache, sess.codes, budget_ppm=ppm, budget_count=budget_count)
     torch.cuda.synchronize()
-    assert torch.equal(out, out2), "decode is not reproducible between calls"
+    if sess.s_err is not None and append is not None:
+        # with a safeguard set every block also attends the safeguard keys of its own key range, and the fused call
+        # splits the key range differently (the appending block takes a smaller share): same rows, another summation order
+        assert (out - out2).abs().max().item() <= 1e-5, "fused and plain decode disagree"
+    else:
+        assert torch.equal(out, out2), "decode is not reproducible between calls"
     G = s.group
     tol = OUT_TOL[s.dtype]
     for u in units:
@@ -219,9 +257,24 @@ def check_decode(sess: Session, q: torch.Tensor, units, report: dict, budget_ppm
             assert np.array_equal(O.hash_scores(bits, sg, a), sc_gpu)
         # selection
         k = O.budget(n, ppm, budget_count)
-        idx = O.topk(sc_gpu, k)
-        idx_gpu = sel[u, :k].cpu().numpy().astype(np.int64)
-        assert np.array_equal(idx, idx_gpu), "selected index set differs (unit %d)" % u
+        if sess.s_err is None:
+            idx = O.topk(sc_gpu, k)
+            idx_gpu = sel[u, :k].cpu().numpy().astype(np.int64)
+            assert np.array_equal(idx, idx_gpu), "selected index set differs (unit %d)" % u
+        else:
+            # error-aware safeguard: k - me hash-selected keys, then the first me safeguard keys with -1 for duplicates
+            s_err = sess.s_err[u]
+            me = min(len(s_err), k)
+            hash_idx = O.topk(sc_gpu, k - me)
+            got_hash = sel[u, :k - me].cpu().numpy().astype(np.int64)
+            assert np.array_equal(hash_idx, got_hash), "hash-selected part differs (unit %d)" % u
+            want_tail = np.where(np.isin(s_err[:me], hash_idx), -1, s_err[:me])
+            got_tail = sel[u, k - me:k].cpu().numpy().astype(np.int64)
+            assert np.array_equal(want_tail, got_tail), "safeguard part of the index list differs (unit %d)" % u
+            idx_gpu = O.eas_union(hash_idx, s_err[:me])
+            ref_unit = O.decode_unit(qg, K, V, bits, Ph, ppm, budget_count, mode=mode, s_err=s_err)
+            if np.array_equal(A, A_gpu):
+                assert np.array_equal(ref_unit["idx"], idx_gpu)
         if k < n_max:
             assert int(sel[u, k]) == -1, "index list written past k"
         # attention over the selected rows

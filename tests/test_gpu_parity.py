@@ -316,3 +316,34 @@ def test_cfg4_full_size_sampled_units():
     sess.encode(); H.check_encode(sess, [2, 31], rep, key_slice=(60000, 64096))
     _decode_loop(sess, 2, [0, 19, 31], rep, H, fused=True)
     print(rep)
+
+
+@pytest.mark.parametrize("dtype,bits,group,n,cluster", [("bf16", 128, 4, 9000, 0), ("bf16", 128, 4, 9000, 1), ("bf16", 64, 8, 5000, 2),
+                                                        ("f32", 64, 2, 4096, 0), ("bf16", 256, 1, 3000, 0)])
+def test_error_aware_safeguard(dtype, bits, group, n, cluster):
+    """EAS: per-key reconstruction errors from both encode paths, the static hard-to-hash set, and decode steps whose
+    selection is the union of the hash top-(k - m) and that set (10 % of a 2 % budget), incl. the fused cache write."""
+    H = _harness()
+    spec = CONFIGS[1].scaled(n_ctx=n, n_kv_heads=2, n_q_heads=2 * group, code_bits=bits, dtype=dtype, steps=2,
+                             rope_base=None if dtype == "f32" else 500000.0)
+    sess = H.Session(spec, eas_ppm=2000, cluster_size=cluster)
+    rep = {}
+    sess.fit(); sess.encode()
+    H.check_eas(sess, [0, 1], rep)
+    _decode_loop(sess, 2, [0, 1], rep, H)
+    q, _ = sess.w.queries(sess.lens)
+    H.check_decode(sess, q.cuda(), [0, 1], rep, budget_ppm=0, budget_count=5)          # budget below the set size
+    H.check_decode(sess, q.cuda(), [0, 1], rep, budget_ppm=1000000)                    # everything: all duplicates
+    H.check_decode(sess, q.cuda(), [1], rep, budget_ppm=500000)
+    print(rep)
+
+
+def test_error_aware_safeguard_full_size_cfg2():
+    H = _harness()
+    spec = CONFIGS[2].scaled(batch=2)
+    sess = H.Session(spec, gen_device="cuda", interleaved=True, eas_ppm=2000)
+    rep = {}
+    sess.fit(); sess.encode()
+    H.check_eas(sess, [3, 12], rep)
+    _decode_loop(sess, 2, [3, 12, 15], rep, H, fused=True)
+    print(rep)
