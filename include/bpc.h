@@ -192,10 +192,13 @@ size_t     bpc_static_scratch_entries(void);
  * A = sum over the group's heads of sign*magnitude (qweights [units][code_bits] int32). */
 bpc_status bpc_debug_set_buffers(bpc_ctx* ctx, int32_t* scores, int32_t* qweights);
 
-/* Tracing aid.  When set (non-NULL), every thread block of the next bpc_decode_attn calls writes
- * %globaltimer stamps (ns) at its phase boundaries into a row of 16 slots: 0 start, 1 query hash done,
- * 2 scan done, 3 selection done, 4 index list visible, 5 attention done, 6 block merge done, 7 end,
- * 8 histograms complete, 9 threshold known, 10 output offsets known.  stamps [units * cluster_size][16] uint64. */
+/* Tracing aid.  When set (non-NULL), every thread block of the next bpc_decode_attn calls writes time stamps at
+ * its phase boundaries into a row of 16 slots.  Slots 0 and 7 hold %globaltimer (ns) at the block's start and end,
+ * slots 15 and 14 the SM cycle counter at the same two points (which gives the block's ns per cycle); every other
+ * slot holds the cycle counter: 1 query hash done, 2 scan done, 8 histograms complete (cluster barrier passed),
+ * 9 threshold known, 10 output offsets known, 3 selection done, 4 index list visible, 5 attention done, 6 block
+ * merge done; in the block that appends a key also 12 / 11 sign sweep started / finished and 13 its scanning warps
+ * done.  stamps [units * cluster_size][16] uint64. */
 bpc_status bpc_debug_set_phase_timer(bpc_ctx* ctx, uint64_t* stamps);
 
 /* Launch geometry of the decode kernel: thread blocks per cluster (0 = choose automatically).

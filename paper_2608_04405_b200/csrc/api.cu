@@ -80,7 +80,7 @@ cudaError_t decode_limits(const bpc_ctx* ctx, int /*unused*/, int* max_cluster, 
 int chunk_for(int n_max, int cs) {
   const int plain = (((n_max + cs - 1) / cs) + 63) & ~63;
   if (cs == 1) return plain;
-  const int fused = ((int)(((long long)n_max * 16 + 16 * cs - 2) / (16 * cs - 1)) + 63) & ~63;
+  const int fused = bpc_fused_chunk(n_max, cs);
   return fused > plain ? fused : plain;
 }
 

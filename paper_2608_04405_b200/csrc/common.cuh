@@ -14,6 +14,13 @@
 #define BPC_DEVERR_APPEND_CAP  2   // append at n_max
 #define BPC_DEVERR_TIMEOUT     4   // a bounded wait gave up
 
+// In a launch that also appends, the block that codes the new key scans with fewer resources (one warp runs
+// Algorithm 2's sign sweep); it is given (16 - BPC_APPEND_LOSS16)/16 of the other blocks' key share.
+#define BPC_APPEND_LOSS16 2
+__host__ __device__ inline int bpc_fused_chunk(int n, int cs) {
+  return ((int)(((long long)n * 16 + 16 * cs - BPC_APPEND_LOSS16 - 1) / (16 * cs - BPC_APPEND_LOSS16)) + 63) & ~63;
+}
+
 struct bpc_ctx {
   bpc_config cfg;
   int device;

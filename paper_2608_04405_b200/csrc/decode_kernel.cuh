@@ -30,7 +30,7 @@ namespace cg = cooperative_groups;
 constexpr int kSegKeys = 32;        // score keys per shared-memory segment
 constexpr int kSegSlots = 40;       // 16-bit slots per segment (80 B: conflict-free 16-byte reads)
 constexpr int kMaxBins = 2048;      // histogram bins (score keys are 0..nbins-1)
-constexpr int kIdxTile = 1024;      // selected indices staged at a time
+constexpr int kIdxTile = 1024;      // selected indices staged at a time (fp32 path, long lists)
 constexpr int kMaxPlanes = 10;
 constexpr int kEasMax = 16384;      // largest error-aware safeguard set per unit
 constexpr int kEasLocal = 1024;     // safeguard keys of one block kept in shared memory (larger slices stay in global)
@@ -45,7 +45,7 @@ struct SmallState {
   uint32_t mask[kMaxPlanes][8];
   uint32_t gt[BPC_MAX_CLUSTER];
   uint32_t eq[BPC_MAX_CLUSTER];
-  uint32_t wscan[32];
+  uint32_t wscan[64];                    // block scans: two alternating buffers of 2 x 16 warp totals (16-byte aligned)
   double pmax[BPC_MAX_GROUP];
   int T, cnt_gt, my_take, my_base, rsum, e0, e1, pad;
   uint32_t newcode[8];                   // code of the key appended by this launch
@@ -96,25 +96,34 @@ struct DecodeSmem {
 
 __device__ __forceinline__ int score_slot(int i) { return (i >> 5) * kSegSlots + (i & 31); }
 
-// exclusive prefix sum over the NT threads of a block; *total receives the block sum
+// Exclusive prefix sum over the NT threads of a block; *total receives the block sum.  One barrier per call: the warp
+// totals come from a warp reduction and are posted before each warp scans its own lanes, and consecutive calls
+// alternate between two buffers (ph, the number of calls so far, is uniform over the block), so a warp that is early
+// for the next call cannot overwrite totals that a late warp still reads.  wscan holds 2 x 2 x 16 words.
 template <int NT>
-__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* wscan, uint32_t* total) {
+__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* wscan, int& ph, uint32_t* total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t* buf = wscan + (ph & 1) * 32;
+  ++ph;
+  const uint32_t wt = __reduce_add_sync(0xffffffffu, v);
+  if (lane == 0) buf[warp] = wt;
   uint32_t inc = v;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+    const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
     if (lane >= o) inc += t;
   }
-  __syncthreads();                       // wscan may still be read from a previous call
-  if (lane == 31) wscan[warp] = inc;
   __syncthreads();
   uint32_t wbase = 0, tot = 0;
 #pragma unroll
-  for (int w = 0; w < NT / 32; ++w) {
-    uint32_t t = wscan[w];
-    if (w < warp) wbase += t;
-    tot += t;
+  for (int w4 = 0; w4 < NT / 128; ++w4) {
+    const uint4 q = reinterpret_cast<const uint4*>(buf)[w4];
+    const uint32_t e[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (4 * w4 + i < warp) wbase += e[i];
+      tot += e[i];
+    }
   }
   *total = tot;
   return wbase + inc - v;
@@ -122,8 +131,12 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* wscan,
 
 // the same for two values at once
 template <int NT>
-__device__ __forceinline__ void block_excl_scan2(uint32_t a, uint32_t b, uint32_t* wscan, uint32_t& ea, uint32_t& eb) {
+__device__ __forceinline__ void block_excl_scan2(uint32_t a, uint32_t b, uint32_t* wscan, int& ph, uint32_t& ea, uint32_t& eb) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t* buf = wscan + (ph & 1) * 32;
+  ++ph;
+  const uint32_t wa = __reduce_add_sync(0xffffffffu, a), wb = __reduce_add_sync(0xffffffffu, b);
+  if (lane == 0) { buf[warp] = wa; buf[16 + warp] = wb; }
   uint32_t ia = a, ib = b;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -131,12 +144,14 @@ __device__ __forceinline__ void block_excl_scan2(uint32_t a, uint32_t b, uint32_
     if (lane >= o) { ia += ta; ib += tb; }
   }
   __syncthreads();
-  if (lane == 31) { wscan[warp] = ia; wscan[NT / 32 + warp] = ib; }
-  __syncthreads();
   uint32_t ba = 0, bb = 0;
 #pragma unroll
-  for (int w = 0; w < NT / 32; ++w) {
-    if (w < warp) { ba += wscan[w]; bb += wscan[NT / 32 + w]; }
+  for (int w4 = 0; w4 < NT / 128; ++w4) {
+    const uint4 qa = reinterpret_cast<const uint4*>(buf)[w4], qb = reinterpret_cast<const uint4*>(buf + 16)[w4];
+    const uint32_t xa[4] = {qa.x, qa.y, qa.z, qa.w}, xb[4] = {qb.x, qb.y, qb.z, qb.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      if (4 * w4 + i < warp) { ba += xa[i]; bb += xb[i]; }
   }
   ea = ba + ia - a;
   eb = bb + ib - b;
@@ -243,6 +258,8 @@ bpc_decode_kernel(const DecodeParams p) {
   typedef typename L::acc_t acc_t;
   constexpr int NT = L::NT, NW = L::NW, B = L::B;
   constexpr int NP = PlaneCount<GP, MODE>::value;
+  // Hamming scores whose largest key fits one histogram bin per thread: only the one-pass threshold search is compiled
+  constexpr bool kFastOnly = MODE == 0 && L::B * ((1 << NP) - 1) + 1 <= L::NT;
   constexpr int ROWB = L::kRowBytes;
   extern __shared__ __align__(16) unsigned char smem[];
 
@@ -306,9 +323,8 @@ bpc_decode_kernel(const DecodeParams p) {
   const int me = EAS ? me_rt : 0;                            // a compile-time zero without the safeguard
   const int kh = k - me;
   // Keys per block.  In a fused launch the appending block (the last one with keys) scans with one warp less, so
-  // it is given 15/16 of the others' share.
-  const int chunk = (fused && CS > 1) ? ((int)(((long long)n * 16 + 16 * CS - 2) / (16 * CS - 1)) + 63) & ~63
-                                      : (((n + CS - 1) / CS) + 63) & ~63;
+  // it is given a smaller share (bpc_fused_chunk).
+  const int chunk = (fused && CS > 1) ? bpc_fused_chunk(n, CS) : (((n + CS - 1) / CS) + 63) & ~63;
   float* out_u = p.out + ((size_t)seq * p.n_kv_heads + kvh) * (size_t)G * BPC_D;
 
   // Both early exits depend only on values every block of the cluster sees identically, so either all
@@ -337,8 +353,11 @@ bpc_decode_kernel(const DecodeParams p) {
   SmallState* st = reinterpret_cast<SmallState*>(smem + plan.off_small);
   unsigned char* uni = smem + plan.off_union;
   uint16_t* sc = reinterpret_cast<uint16_t*>(uni);
-#define BPC_STAMP(i) do { if (p.dbg_times != nullptr && tid == 0) p.dbg_times[(size_t)blockIdx.x * 16 + (i)] = global_timer_ns(); } while (0)
-  BPC_STAMP(0);
+  // Phase stamps (debug): slots 0 and 7 hold the global timer at block start and end, slots 15 and 14 the SM's cycle
+  // counter at the same two points, every other slot the cycle counter (cheap to read) at that phase boundary.
+#define BPC_STAMP(i) do { if (p.dbg_times != nullptr && tid == 0) p.dbg_times[(size_t)blockIdx.x * 16 + (i)] = (unsigned long long)clock64(); } while (0)
+  if (p.dbg_times != nullptr && tid == 0) p.dbg_times[(size_t)blockIdx.x * 16] = global_timer_ns();
+  BPC_STAMP(15);
   // the block whose key range holds the appended key (index n-1) does the append work in its last warp
   const bool appender = fused && rank == (n - 1) / chunk;
 
@@ -349,8 +368,9 @@ bpc_decode_kernel(const DecodeParams p) {
   if (appender && p.residual_correction != 0) {
     const size_t union_bytes = plan.total - plan.off_union;
     const size_t score_bytes = (size_t)((p.chunk_cap + kSegKeys - 1) / kSegKeys) * kSegSlots * 2;
-    if (score_bytes + (size_t)B * B * 4 <= union_bytes && L::hashpart_bytes() + (size_t)B * B * 4 <= union_bytes) {
-      float* dstg = reinterpret_cast<float*>(uni + union_bytes - (size_t)B * B * 4);
+    constexpr size_t kGramPad = 0;
+    if (score_bytes + (size_t)B * B * 4 + kGramPad <= union_bytes && L::hashpart_bytes() + (size_t)B * B * 4 + kGramPad <= union_bytes) {
+      float* dstg = reinterpret_cast<float*>(uni + union_bytes - (size_t)B * B * 4 - kGramPad);
       const float* Gs = p.gram + (size_t)(p.shared_sets ? kvh : unit) * B * B;
       for (int c = tid; c < B * B / 4; c += NT) cp_async16(dstg + 4 * c, Gs + 4 * c);
       gsm = dstg;
@@ -384,7 +404,7 @@ bpc_decode_kernel(const DecodeParams p) {
     for (int u = 0; u < U; ++u) load_code(h[u], base + u * nts + tid);
   };
   uint32_t ha[U][W32], hb[U][W32];
-  const bool pipelined = tid < nts && dbg == nullptr && c0 + nts * U <= c1s;   // at least one full batch
+  const bool pipelined = tid < nts && c0 + nts * U <= c1s;   // at least one full batch
   if (pipelined) load_batch(ha, c0);
 
   // ------------------------------------------------------------------ phase 0: query hash
@@ -525,12 +545,21 @@ bpc_decode_kernel(const DecodeParams p) {
         atomicAdd(&hist[key >> hsh], 1u);
       }
     };
+    const int STEP = nts * U;
+    if (dbg != nullptr) {                                    // score export (tests): a plain loop, one key at a time
+#pragma unroll 1
+      for (int i = c0 + tid; i < c1s; i += nts) {
+        uint32_t h[W32];
+        load_code(h, i);
+        dbg[i] = ((2 * score_key<W32, NP>(h, sg, mk)) << cs) - rfull;
+      }
+    }
     int i0 = c0;
     if (pipelined) {
       // Full batches without bounds checks, software-pipelined over two register buffers so that the
-      // loads of the next batch are in flight while the current one is scored (a warp's 32 keys share
-      // one score segment).  The first batch was requested before the query hash.
-      const int STEP = nts * U;
+      // loads of the next batch are in flight while the current one is scored (a warp's 32 keys share one
+      // score segment).  The first batch was requested before the query hash.
+#pragma unroll 1
       for (;;) {
         const bool more_b = i0 + 2 * STEP <= c1s;
         if (more_b) load_batch(hb, i0 + STEP);
@@ -544,9 +573,8 @@ bpc_decode_kernel(const DecodeParams p) {
         if (!more_a) break;
       }
     }
-    // remainder (and the whole range when scores are exported): the same batches with per-key bounds checks,
-    // so that the loads of a batch are still in flight together
-    for (; i0 < c1s; i0 += nts * U) {
+    // ragged tail (less than one batch): the same batch with per-key bounds checks, loads in flight together
+    if (i0 < c1s) {
       uint32_t h[U][W32];
 #pragma unroll
       for (int u = 0; u < U; ++u) {
@@ -565,15 +593,14 @@ bpc_decode_kernel(const DecodeParams p) {
           const int key = score_key<W32, NP>(h[u], sg, mk);
           sc[score_slot(i - c0)] = (uint16_t)key;
           atomicAdd(&hist[key >> hsh], 1u);
-          if (dbg != nullptr) dbg[i] = ((2 * key) << cs) - rfull;
         }
       }
     }
-    if (p.dbg_times != nullptr && tid == 0) p.dbg_times[(size_t)blockIdx.x * 16 + 13] = global_timer_ns();
+    if (p.dbg_times != nullptr && tid == 0) p.dbg_times[(size_t)blockIdx.x * 16 + 13] = (unsigned long long)clock64();
   } else {
     // ---- appending warp (Algorithm 2 on the new key, Gram form): cache rows, sign sweep, code words.
     // Lane l holds the decision values of bits l, 32+l, ...; bit i is decided by a shuffle from its owner
-    // lane and every later column is corrected with G[i][.], read from global memory two steps ahead.
+    // lane and every later column is corrected with G[i][.].
     const size_t rstride_e = (size_t)p.row_stride;
     const KV* kn = reinterpret_cast<const KV*>(p.k_new) + (size_t)unit * BPC_D;
     const KV* vn = reinterpret_cast<const KV*>(p.v_new) + (size_t)unit * BPC_D;
@@ -593,44 +620,59 @@ bpc_decode_kernel(const DecodeParams p) {
     const float* Gs = p.gram + (size_t)(p.shared_sets ? kvh : unit) * B * B;
     const bool rc = p.residual_correction != 0;
     uint32_t* code_dst = reinterpret_cast<uint32_t*>(p.codes_w) + ((size_t)unit * p.n_max + (n - 1)) * W32;
-    constexpr int PF = 8;                                    // Gram rows per prefetch group
-#pragma unroll
-    for (int bi = 0; bi < NB; ++bi) {
-      // After step i lane i of the diagonal block is never corrected again (its Gram entries are masked to
-      // zero at fetch time), so at the end its t holds its own decision value and one ballot yields the word.
-      float ga[PF][NB], gb[PF][NB];
-      auto fetch = [&](float (&gq)[PF][NB], int ii) {
-#pragma unroll
-        for (int r = 0; r < PF; ++r)
-#pragma unroll
-          for (int c = bi; c < NB; ++c) {
-            const size_t gi = (size_t)(32 * bi + ii + r) * B + 32 * c + lane;
-            float gv = !rc ? 0.f : (gsm != nullptr ? gsm[gi] : __ldg(Gs + gi));
-            if (c == bi && lane <= ii + r) gv = 0.f;
-            gq[r][c] = gv;
-          }
-      };
-      auto sweep = [&](const float (&gq)[PF][NB], int ii) {
-#pragma unroll
-        for (int r = 0; r < PF; ++r) {
-          const float ti = __shfl_sync(0xffffffffu, t[bi], ii + r);
-          const float u = ti >= 0.f ? 1.f : -1.f;
-#pragma unroll
-          for (int c = bi; c < NB; ++c) t[c] = fmaf(-u, gq[r][c], t[c]);
-        }
-      };
-      fetch(ga, 0);
+    if (p.dbg_times != nullptr && lane == 0) p.dbg_times[(size_t)blockIdx.x * 16 + 12] = (unsigned long long)clock64();
+    {
+      // The b sign decisions are taken eight at a time: every lane collects the eight
+      // decision values of the group and decides them on its own copy (their 8 x 8 Gram block is read at one address
+      // by the whole warp: no cross-lane traffic inside the dependency chain), then the eight signs correct all later
+      // columns, one column per lane and 32-bit word.  Every value sees the same fp32 operations in the same order
+      // as a one-bit-at-a-time sweep.
+      const float* gq = gsm != nullptr ? gsm : Gs;             // Gram matrix: staged in shared memory when it fits
 #pragma unroll 1
-      for (int ii = 0; ii < 32; ii += 2 * PF) {
-        fetch(gb, ii + PF);
-        sweep(ga, ii);
-        if (ii + 2 * PF < 32) fetch(ga, ii + 2 * PF);
-        sweep(gb, ii + PF);
+      for (int bi = 0; bi < NB; ++bi) {
+        uint32_t wbits = 0u;
+        if (!rc) {
+          float tb = t[0];
+#pragma unroll
+          for (int c = 1; c < NB; ++c) tb = bi == c ? t[c] : tb;
+          wbits = __ballot_sync(0xffffffffu, tb >= 0.f);
+        } else {
+#pragma unroll 1
+          for (int sub = 0; sub < 4; ++sub) {
+            float tb = t[0];
+#pragma unroll
+            for (int c = 1; c < NB; ++c) tb = bi == c ? t[c] : tb;
+            float w[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) w[e] = __shfl_sync(0xffffffffu, tb, 8 * sub + e);
+            const int r0 = 32 * bi + 8 * sub;
+            const float* gd = gq + (size_t)r0 * B + r0;         // the group's 8 x 8 diagonal block
+            float nu[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const bool pos = w[e] >= 0.f;
+              wbits |= pos ? (1u << (8 * sub + e)) : 0u;
+              nu[e] = pos ? -1.f : 1.f;
+              const float4 g0 = *reinterpret_cast<const float4*>(gd + (size_t)e * B);
+              const float4 g1 = *reinterpret_cast<const float4*>(gd + (size_t)e * B + 4);
+              const float gr[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+#pragma unroll
+              for (int f = e + 1; f < 8; ++f) w[f] = fmaf(nu[e], gr[f], w[f]);
+            }
+#pragma unroll
+            for (int c = 0; c < NB; ++c) {
+              if (c >= bi) {                                     // decided columns of word bi are corrected too: never read again
+                const float* gc = gq + (size_t)r0 * B + 32 * c + lane;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) t[c] = fmaf(nu[e], gc[(size_t)e * B], t[c]);
+              }
+            }
+          }
+        }
+        if (lane == 0) { st->newcode[bi] = wbits; code_dst[bi] = wbits; }
       }
-      const uint32_t wbits = __ballot_sync(0xffffffffu, t[bi] >= 0.f);
-      if (lane == 0) { st->newcode[bi] = wbits; code_dst[bi] = wbits; }
     }
-    if (p.dbg_times != nullptr && lane == 0) p.dbg_times[(size_t)blockIdx.x * 16 + 11] = global_timer_ns();
+    if (p.dbg_times != nullptr && lane == 0) p.dbg_times[(size_t)blockIdx.x * 16 + 11] = (unsigned long long)clock64();
   }
   if (appender) {
     __syncthreads();                                         // the new code is in shared memory; the scan is done
@@ -651,12 +693,33 @@ bpc_decode_kernel(const DecodeParams p) {
 
   BPC_STAMP(2);
   // ------------------------------------------------------------------ phase 2: threshold and ordered selection
-  cluster.sync();                                            // every block's histogram is complete
+  // With one bin per thread, every block first stores its finished histogram into a slot of every peer's shared memory
+  // (behind the score keys), so that after the barrier all CS histograms are local reads.
+  const bool fast_sel = kFastOnly || (nbins <= NT && hsh == 0);
+  uint32_t* pushed = nullptr;
+  {
+    const size_t union_bytes = plan.total - plan.off_union;
+    size_t push_off = (size_t)((p.chunk_cap + kSegKeys - 1) / kSegKeys) * kSegSlots * 2;
+    if (push_off < L::hashpart_bytes()) push_off = L::hashpart_bytes();   // a peer may still be hashing
+    push_off = (push_off + 15) & ~(size_t)15;
+    if (fast_sel && CS > 1 && push_off + (size_t)CS * nbins * 4 + (size_t)B * B * 4 <= union_bytes)
+      pushed = reinterpret_cast<uint32_t*>(uni + push_off);
+  }
+  if (pushed != nullptr) {
+    __syncthreads();                                         // this block's histogram is complete
+    if (tid < nbins) {
+      const uint32_t v = hist[tid];
+#pragma unroll
+      for (int r = 0; r < BPC_MAX_CLUSTER; ++r)
+        if (r < CS) cluster.map_shared_rank(pushed, r)[rank * nbins + tid] = v;
+    }
+  }
+  cluster.sync();                                            // every block's histogram is complete (and delivered)
   BPC_STAMP(8);
   if (appender && tid == 0) p.unit_lens_w[unit] = n;         // every block of the cluster has read the old length
   // Threshold key T (the k-th largest score key) and this block's share of the output.
   int T;
-  const bool fast_sel = nbins <= NT && hsh == 0;
+  int scan_calls = 0;                                        // block scans so far (selects their buffer)
   if (fast_sel) {
     // Common case, one histogram bin per thread: thread t owns bin nbins-1-t, reads that bin from every block of
     // the cluster (distributed shared memory) and a two-value block scan yields, for every bin, the number of keys
@@ -665,11 +728,20 @@ bpc_decode_kernel(const DecodeParams p) {
     // (ties are granted to blocks in rank order, which is index order).
     const int bin = nbins - 1 - tid;
     uint32_t s_all = 0, s_low = 0, mine = 0;
-    if (bin >= 0) {
-#pragma unroll
-      for (int r = 0; r < BPC_MAX_CLUSTER; ++r) {
-        if (r < CS) {
-          const uint32_t v = cluster.map_shared_rank(hist, r)[bin];
+    {
+      const int bq = max(bin, 0);
+      if (pushed != nullptr) {
+#pragma unroll 1
+        for (int r = 0; r < CS; ++r) {
+          const uint32_t v = bin >= 0 ? pushed[r * nbins + bq] : 0u;
+          s_all += v;
+          if (r < rank) s_low += v;
+          if (r == rank) mine = v;
+        }
+      } else {
+#pragma unroll 1
+        for (int r = 0; r < CS; ++r) {
+          const uint32_t v = bin >= 0 ? cluster.map_shared_rank(hist, r)[bq] : 0u;
           s_all += v;
           if (r < rank) s_low += v;
           if (r == rank) mine = v;
@@ -677,7 +749,7 @@ bpc_decode_kernel(const DecodeParams p) {
       }
     }
     uint32_t above_all, above_low;
-    block_excl_scan2<NT>(s_all, s_low, st->wscan, above_all, above_low);
+    block_excl_scan2<NT>(s_all, s_low, st->wscan, scan_calls, above_all, above_low);
     if (bin >= 0 && above_all < (uint32_t)kh && above_all + s_all >= (uint32_t)kh) {
       const int need = kh - (int)above_all;                   // ties to take, cluster-wide (>= 1)
       const int lower_take = min(need, (int)s_low);          // ties granted to blocks of lower rank
@@ -689,8 +761,8 @@ bpc_decode_kernel(const DecodeParams p) {
     __syncthreads();
     T = st->T;
     BPC_STAMP(9);
-  } else {
-  // Total histogram through distributed shared memory.  With at most one bin per thread (the common case)
+  } else if constexpr (!kFastOnly) {
+    // Total histogram through distributed shared memory.  With at most one bin per thread (the common case)
     // the per-block counts of that bin stay in registers and are reused for the per-block offsets below.
     const bool one_bin = nbins <= NT;
     uint32_t myv[BPC_MAX_CLUSTER];
@@ -719,7 +791,7 @@ bpc_decode_kernel(const DecodeParams p) {
       uint32_t local = 0;
       for (int bin = hi - 1; bin >= lo; --bin) local += tot[bin];
       uint32_t total;
-      uint32_t above = block_excl_scan<NT>(local, st->wscan, &total);
+      uint32_t above = block_excl_scan<NT>(local, st->wscan, scan_calls, &total);
       for (int bin = hi - 1; bin >= lo; --bin) {
         const uint32_t c = tot[bin];
         if (above < (uint32_t)kh && above + c >= (uint32_t)kh) { st->T = bin; st->cnt_gt = (int)above; }
@@ -752,7 +824,7 @@ bpc_decode_kernel(const DecodeParams p) {
     __syncthreads();
   }
   int T_exact = T;
-  if (hsh > 0 && kh > 0) {
+  if (MODE == 1 && hsh > 0 && kh > 0) {
     // Weighted scores have more distinct values than histogram bins: the search above found the coarse bin
     // that holds the k-th score.  A second, small histogram over the low bits of the keys inside that bin (again
     // summed across the cluster) yields the exact threshold and corrects the per-block counts.
@@ -804,7 +876,7 @@ bpc_decode_kernel(const DecodeParams p) {
     __syncthreads();
     T_exact = st->T;
   }
-  if (!fast_sel && tid == 0) {
+  if (!kFastOnly && !fast_sel && tid == 0) {
     const int need = kh - st->cnt_gt;                        // ties to take, cluster-wide (>= 1)
     int tie_base = 0, out_base = 0;
     for (int r = 0; r < CS; ++r) {
@@ -815,7 +887,7 @@ bpc_decode_kernel(const DecodeParams p) {
       tie_base += (int)st->eq[r];
     }
   }
-  __syncthreads();
+  if (!kFastOnly && !fast_sel) __syncthreads();                            // (the fast path published its values before its own barrier)
   int32_t* sel_u = p.sel + (size_t)unit * p.n_max;
   BPC_STAMP(10);
   {
@@ -884,7 +956,7 @@ bpc_decode_kernel(const DecodeParams p) {
         }
       }
       uint32_t total;
-      const uint32_t ex = block_excl_scan<NT>((uint32_t)cgt | ((uint32_t)ceq << 16), st->wscan, &total);
+      const uint32_t ex = block_excl_scan<NT>((uint32_t)cgt | ((uint32_t)ceq << 16), st->wscan, scan_calls, &total);
       if (cgt | ceq) {
         int eqb = run_eq + (int)(ex >> 16);
         int pos = st->my_base + run_gt + (int)(ex & 0xffffu) + min(eqb, my_take);
@@ -910,22 +982,23 @@ bpc_decode_kernel(const DecodeParams p) {
       run_eq += (int)(total >> 16);
     }
   }
+  // this block attends rows [lo, hi) of the hash list and the safeguard keys that lie in its own key range
+  const int lo = (int)(((long long)kh * rank) / CS), hi = (int)(((long long)kh * (rank + 1)) / CS);
+  const int nh = hi - lo, ne = e1 - e0;                      // rows from the two sources
   if (me > 0) {
     __syncthreads();                                         // all duplicate flags of this block are set
     for (int t = tid; t < e1 - e0; t += NT) {
       const bool dup = (st->eas_dup[t >> 5] >> (t & 31)) & 1u;
-      sel_u[kh + e0 + t] = dup ? -1 : (eas_local ? st->eas_s[t] : eas_u[e0 + t]);
+      const int v = dup ? -1 : (eas_local ? st->eas_s[t] : eas_u[e0 + t]);
+      sel_u[kh + e0 + t] = v;
     }
   }
   BPC_STAMP(3);
-  __threadfence();
-  cluster.sync();                                            // the unit's index list is complete and visible
+  cluster.sync();                                            // release/acquire at cluster scope: the unit's index list
+                                                             // (global memory, written by all blocks) is complete and visible
   BPC_STAMP(4);
 
   // ------------------------------------------------------------------ phase 3: gathered attention
-  // this block attends rows [lo, hi) of the hash list and the safeguard keys that lie in its own key range
-  const int lo = (int)(((long long)kh * rank) / CS), hi = (int)(((long long)kh * (rank + 1)) / CS);
-  const int nh = hi - lo, ne = e1 - e0;                      // rows from the two sources
   auto row_index = [&](int qrow) -> int {                    // qrow in [0, nh + ne): cache row, or -1 for a duplicate
     if (!EAS) return sel_u[lo + qrow];
     return qrow < nh ? sel_u[lo + qrow] : sel_u[kh + e0 + (qrow - nh)];
@@ -967,19 +1040,28 @@ bpc_decode_kernel(const DecodeParams p) {
     // reads are conflict-free), keeps NS-1 blocks in flight and multiplies the oldest one.
     constexpr int WSTG = 8 * 2 * ROWB;                       // bytes of one 8-row stage (K rows, then V rows)
     unsigned char* wst = stg + (size_t)warp * NS * WSTG;
-    const int nrows = nh + ne;
+    // the block's rows are split evenly over the warps (contiguous ranges; the last 8-row block of a warp may be short)
+    const int nrows_b = nh + ne;
+    const int r0w = (int)(((long long)nrows_b * warp) / NW), r1w = (int)(((long long)nrows_b * (warp + 1)) / NW);
+    const int nrows = r1w - r0w;
     const int nblk = (nrows + 7) >> 3;
     const int isv = lane >> 4, ch = lane & 15;
     const unsigned char* srcbase = (isv ? Vu : Ku) + (size_t)ch * 16;
+    // a warp's first 64 list entries are fetched once (one coalesced read), later ones block by block
+    int pre0 = -1, pre1 = -1;
+    if (lane < nrows) pre0 = row_index(r0w + lane);
+    if (32 + lane < nrows) pre1 = row_index(r0w + 32 + lane);
     auto issue = [&](int bi) {
-      const int blk = warp + bi * NW;
-      if (blk < nblk) {
-        const int rbase = 8 * blk;
+      if (bi < nblk) {
+        const int rbase = 8 * bi;
         int myidx = -1;
-        if (lane < 8 && rbase + lane < nrows) {
-          myidx = row_index(rbase + lane);
-          if (myidx >= 0) myidx = min(myidx, p.n_max - 1);
+        if (bi < 8) {                                        // warp-uniform
+          const int v = __shfl_sync(0xffffffffu, bi < 4 ? pre0 : pre1, (rbase & 31) + (lane & 7));
+          if (lane < 8) myidx = v;
+        } else if (lane < 8 && rbase + lane < nrows) {
+          myidx = row_index(r0w + rbase + lane);
         }
+        if (myidx >= 0) myidx = min(myidx, p.n_max - 1);
         if (EAS) {   // which of the 8 rows are real (not past the end, not a duplicate of a hash-selected key)
           const uint32_t vm = __ballot_sync(0xffffffffu, myidx >= 0) & 0xffu;
           if (lane == 0) st->stage_valid[warp][bi % NS] = (uint8_t)vm;
@@ -1000,12 +1082,11 @@ bpc_decode_kernel(const DecodeParams p) {
       }
       cp_async_commit();
     };
-    for (int tt = 0; tt < NS - 1; ++tt) issue(tt);
-    for (int bi = 0; warp + bi * NW < nblk; ++bi) {
-      if (NS == 2) cp_async_wait<0>(); else cp_async_wait<1>();   // this lane's copies for block bi have landed
+    for (int tt = 0; tt < NS; ++tt) issue(tt);              // every stage of the ring starts in flight
+    for (int bi = 0; bi < nblk; ++bi) {
+      if (NS == 2) cp_async_wait<1>(); else cp_async_wait<2>();   // this lane's copies for block bi have landed
       __syncwarp();                                          // ... and every lane's
-      issue(bi + NS - 1);                                    // refill the stage consumed in the previous round
-      const int rbase_c = 8 * (warp + bi * NW);
+      const int rbase_c = 8 * bi;
       const uint32_t vmask = EAS ? (uint32_t)st->stage_valid[warp][bi % NS]
                                  : (rbase_c + 8 <= nrows ? 0xffu : ((1u << (nrows - rbase_c)) - 1u));
       const unsigned char* ks = wst + (size_t)(bi % NS) * WSTG;
@@ -1047,7 +1128,8 @@ bpc_decode_kernel(const DecodeParams p) {
         mma_pv(o[4 * jj + 2], pa0, pa1, b[2]);
         mma_pv(o[4 * jj + 3], pa0, pa1, b[3]);
       }
-      __syncwarp();
+      __syncwarp();                                          // every lane is done with this stage:
+      issue(bi + NS);                                        // refill it
     }
     cp_async_wait<0>();
     // lanes of one head (same g) hold partial sums of l over their keys
@@ -1218,7 +1300,8 @@ bpc_decode_kernel(const DecodeParams p) {
     }
   }
   cluster.sync();                                            // keep shared memory alive until all peers have read it
-  BPC_STAMP(7);
+  BPC_STAMP(14);
+  if (p.dbg_times != nullptr && tid == 0) p.dbg_times[(size_t)blockIdx.x * 16 + 7] = global_timer_ns();
 #undef BPC_STAMP
 }
 

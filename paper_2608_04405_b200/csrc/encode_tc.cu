@@ -234,6 +234,21 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
       DiagSweep<0>::run(t, word, abs_sum, g_s + (size_t)(32 * cb) * NBITS + 32 * cb, NBITS, residual_correction);
       words[cb] = word;
     }
+    // squared reconstruction error (Eq. 8) from the sweep: ||k - hP||^2 = ||k||^2 - 2 sum|t_i| + trace(G).  The key's
+    // channels are read from this tile's operand buffer before the barrier below: after it, other threads refill
+    // that buffer with the tile after next.
+    const int key = tile * kTileKeys + tid;
+    float k2 = 0.f;
+    if (key_err != nullptr && key < n) {
+      const unsigned char* arow = a_s[it & 1];
+#pragma unroll
+      for (int ch = 0; ch < 16; ++ch) {
+        const uint4 w = *reinterpret_cast<const uint4*>(arow + sw128_offset(kTileKeys, tid, ch));
+        const float f0 = bf16_lo(w.x), f1 = bf16_hi(w.x), f2 = bf16_lo(w.y), f3 = bf16_hi(w.y);
+        const float f4 = bf16_lo(w.z), f5 = bf16_hi(w.z), f6 = bf16_lo(w.w), f7 = bf16_hi(w.w);
+        k2 += (f0 * f0 + f1 * f1) + (f2 * f2 + f3 * f3) + (f4 * f4 + f5 * f5) + (f6 * f6 + f7 * f7);
+      }
+    }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     if (next < ntiles) {
       cp_async_wait_all();
@@ -245,21 +260,7 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       issue_mma(a_s[(it + 1) & 1]);
     }
-    const int key = tile * kTileKeys + tid;
-    if (key_err != nullptr && key < n) {
-      // squared reconstruction error (Eq. 8) from the sweep: ||k - hP||^2 = ||k||^2 - 2 sum|t_i| + trace(G);
-      // the key's channels are still in this tile's operand buffer
-      const unsigned char* arow = a_s[it & 1];
-      float k2 = 0.f;
-#pragma unroll
-      for (int ch = 0; ch < 16; ++ch) {
-        const uint4 w = *reinterpret_cast<const uint4*>(arow + sw128_offset(kTileKeys, tid, ch));
-        const float f0 = bf16_lo(w.x), f1 = bf16_hi(w.x), f2 = bf16_lo(w.y), f3 = bf16_hi(w.y);
-        const float f4 = bf16_lo(w.z), f5 = bf16_hi(w.z), f6 = bf16_lo(w.w), f7 = bf16_hi(w.w);
-        k2 += (f0 * f0 + f1 * f1) + (f2 * f2 + f3 * f3) + (f4 * f4 + f5 * f5) + (f6 * f6 + f7 * f7);
-      }
-      key_err[(size_t)unit * n_max + key] = fmaxf(0.f, k2 - 2.f * abs_sum + trace_g);
-    }
+    if (key_err != nullptr && key < n) key_err[(size_t)unit * n_max + key] = fmaxf(0.f, k2 - 2.f * abs_sum + trace_g);
     if (key < n) {
       uint32_t* dst = reinterpret_cast<uint32_t*>(codes + ((size_t)unit * n_max + key) * (NBITS / 64));
       if (NBITS == 64) {

@@ -45,7 +45,7 @@ cudaError_t scratch_for_current_device(int device, void** out) {
 int chunk_for(int n_max, int cs) {
   const int plain = (((n_max + cs - 1) / cs) + 63) & ~63;
   if (cs == 1) return plain;
-  const int fused = ((int)(((long long)n_max * 16 + 16 * cs - 2) / (16 * cs - 1)) + 63) & ~63;
+  const int fused = bpc_fused_chunk(n_max, cs);
   return fused > plain ? fused : plain;
 }
 
