@@ -122,9 +122,10 @@ class ClockSampler:
 class Layer:
     """One attention layer replica: caches, codes, context, per-step inputs (all resident on the device)."""
 
-    def __init__(self, spec, salt, extra_rows, B, fit_ws, interleaved):
+    def __init__(self, spec, salt, extra_rows, B, fit_ws, interleaved, budget_count=0):
         w = Workload(spec, device="cuda", extra_rows=extra_rows, salt=salt)
         self.w = w
+        self.budget_count = budget_count    # > 0: a fixed number of selected keys instead of the spec's fraction
         if interleaved:     # one buffer, K and V rows of a token adjacent (row stride 2*head_dim)
             self.kv_buf, kc, vc = B.interleaved_kv(spec.batch, spec.n_kv_heads, w.n_max, spec.head_dim, spec.torch_dtype)
             kc.copy_(w.k_cache)
@@ -155,7 +156,7 @@ class Layer:
     def step(self):
         """One decode step: cache write of the new (k, v) + decode, as the single fused launch."""
         self.ctx.append_decode_attn(self.k_new, self.v_new, self.k_cache, self.v_cache, self.codes, self.q,
-                                    budget_ppm=self.w.spec.budget_ppm, out=self.out)
+                                    budget_ppm=self.w.spec.budget_ppm, budget_count=self.budget_count, out=self.out)
 
     def make_weighted_twin(self, B):
         """A second context on the same caches, codes and projection that scores with Algorithm 3's sign + seven
@@ -453,6 +454,66 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ----------------------------------------------------------------------------- paper-scale sweep (second workload)
+SWEEP_CASES = [  # (context, batch): 64-bit codes, fixed budgets, 32/8 heads, bf16, as in the paper's latency-vs-context study
+    (32768, 1), (32768, 16), (131072, 1), (131072, 8), (262144, 1), (262144, 4), (1048576, 1),
+]
+
+
+def run_sweep(args):
+    """Decode-step latency of one layer over contexts and batch sizes with 64-bit codes and fixed budgets of 1024 and
+    2048 keys (the paper's own operating points: single-word codes, 1K/2K budgets, latency flat in the context length).
+    One JSON line; every case is timed like the main workload (CUDA graph of K fused steps over enough layer replicas that
+    a step's bytes exceed L2).  Contexts above the kernel's limit (cluster size 16 x keys per block) are reported as
+    unsupported."""
+    from paper_2608_04405_b200 import binding as B
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    K, W = args.steps, max(args.warmup, 3)
+    rows = []
+    fit_ws = [None]
+    for n_ctx, batch in SWEEP_CASES:
+        spec = CONFIGS[1].scaled(name="sweep_ctx%d_b%d" % (n_ctx, batch), wid=100 + len(rows), batch=batch, n_ctx=n_ctx,
+                                 code_bits=64, steps=K, needles=8)
+        units = batch * spec.n_kv_heads
+        for budget in (1024, 2048):
+            step_bytes = units * (n_ctx * 8 + 2 * budget * spec.head_dim * 2)
+            L = max(2, min(32, -(-(2 * 126 * 2**20) // step_bytes)))
+            extra = ((K + W) // L + 2) * 2 + 64
+            try:
+                layers = [Layer(spec, salt=i, extra_rows=extra, B=B, fit_ws=fit_ws, interleaved=True, budget_count=budget)
+                          for i in range(L)]
+            except Exception as e:                                   # e.g. context beyond the kernel's limit
+                rows.append({"context": n_ctx, "batch": batch, "budget": budget, "unsupported": str(e)[:120]})
+                layers = None
+                torch.cuda.empty_cache()
+                continue
+            for s in range(W):
+                layers[s % L].step()
+            torch.cuda.synchronize()
+            per = [(W + L - 1 - i) // L for i in range(L)]
+            for ly, c in zip(layers, per):
+                ly.ctx.set_seq_lens([n + c for n in ly.lens0])
+            g = _graph_of(lambda: [layers[(W + s) % L].step() for s in range(K)])
+            for ly, c in zip(layers, per):
+                ly.ctx.set_seq_lens([n + c for n in ly.lens0])
+            g.replay()
+            torch.cuda.synchronize()
+            for ly, c in zip(layers, per):
+                ly.ctx.set_seq_lens([n + c for n in ly.lens0])
+            ms = _time_graph(g, lambda: None) / K
+            err = max(ly.ctx.last_device_error() for ly in layers)
+            rows.append({"context": n_ctx, "batch": batch, "budget": budget, "us_per_step": round(ms * 1e3, 2),
+                         "cluster_size": layers[0].ctx.get_cluster_size(), "layer_replicas": L,
+                         "algorithmic_GBps": round(step_bytes / ms / 1e6, 1), "device_error_word": err})
+            layers = None
+            g = None
+            torch.cuda.empty_cache()
+    print(json.dumps({"metric": "decode_step_latency_sweep", "unit": "us_per_step", "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": "paper-scale sweep: 64-bit codes, budgets 1024/2048, 32/8 heads, bf16 K|V interleaved",
+                                 "cold_l2": "layer replicas visited round-robin, bytes per step x replicas > 2 x L2"},
+                      "steps": K, "warmup": W, "cases": rows}))
+
+
 # ----------------------------------------------------------------------------- CPU checker arm
 def _oracle_unit_setup(spec, seed_salt=0):
     """One unit of the workload prepared for the checker: keys, values, projection, codes (prefill, untimed)."""
@@ -530,11 +591,14 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--separate-kv", action="store_true", help="separate K and V arrays instead of interleaved rows")
     ap.add_argument("--profile", action="store_true", help="warm-up plus K eager steps only (for ncu captures)")
+    ap.add_argument("--sweep", action="store_true", help="second workload: latency over contexts and batch sizes, 64-bit codes, 1K/2K budgets")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.sweep:
+        run_sweep(args)
     else:
         run_ours(args)
 

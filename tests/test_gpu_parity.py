@@ -318,6 +318,27 @@ def test_cfg4_full_size_sampled_units():
     print(rep)
 
 
+@pytest.mark.parametrize("n_ctx,batch", [(262144, 1), (32768, 16)])
+def test_sweep_shapes_single_word_codes_fixed_budgets(n_ctx, batch):
+    """The second bench workload's shapes (Section 4 "Setup" / latency-vs-context study: 64-bit codes, budgets of 1024
+    and 2048 keys) at full size in the launch geometry the sweep times: long context at batch 1 (cluster size 8) and
+    short context at batch 16 (cluster size 1); sampled units, plain and fused steps."""
+    H = _harness()
+    spec = CONFIGS[1].scaled(name="sweep", wid=40 + batch, batch=batch, n_ctx=n_ctx, code_bits=64, steps=2)
+    sess = H.Session(spec, gen_device="cuda", interleaved=True)
+    rep = {}
+    sess.fit()
+    sess.encode(); H.check_encode(sess, [2], rep, max_keys=4096)
+    units = [0, sess.units - 1]
+    for budget in (1024, 2048):
+        q, _ = sess.w.queries(sess.lens)
+        H.check_decode(sess, q.cuda(), units, rep, budget_count=budget)
+    k_new, v_new = sess.w.new_kv(sess.lens)
+    q, _ = sess.w.queries(sess.lens)
+    H.check_decode(sess, q.cuda(), units, rep, budget_count=2048, append=(k_new.cuda(), v_new.cuda()))
+    print(rep)
+
+
 @pytest.mark.parametrize("dtype,bits,group,n,cluster", [("bf16", 128, 4, 9000, 0), ("bf16", 128, 4, 9000, 1), ("bf16", 64, 8, 5000, 2),
                                                         ("f32", 64, 2, 4096, 0), ("bf16", 256, 1, 3000, 0)])
 def test_error_aware_safeguard(dtype, bits, group, n, cluster):
