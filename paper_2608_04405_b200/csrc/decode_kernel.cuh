@@ -49,7 +49,6 @@ struct SmallState {
   double pmax[BPC_MAX_GROUP];
   int T, cnt_gt, my_take, my_base, rsum, e0, e1, pad;
   uint32_t newcode[8];                   // code of the key appended by this launch
-  uint32_t eas_dup[kEasMax / 32];        // bit t - e0: safeguard key t was also selected by the hash search
   int32_t eas_s[kEasLocal];              // this block's slice of the safeguard set (when it fits)
   uint8_t stage_valid[32][4];            // per warp and gather stage: which of the 8 rows are real
 };
@@ -423,11 +422,20 @@ bpc_decode_kernel(const DecodeParams p) {
   for (int i = tid; i < nbins; i += NT) hist[i] = 0u;
   if (tid < BPC_MAX_CLUSTER) { st->gt[tid] = 0u; st->eq[tid] = 0u; }
   if (tid == 0) { st->rsum = 0; st->T = 0; st->cnt_gt = 0; st->my_take = 0; st->my_base = 0; st->e0 = 0; st->e1 = 0; }
+  // Safeguard keys inside this block's key range: the set is sorted, so their list positions [e0, e1) are the numbers
+  // of entries below the range's two ends.  A set of at most kEasLocal keys is copied to shared memory asynchronously
+  // now and searched after the hash (nothing needs e0, e1 before the selection); a larger one stays in global
+  // memory and is counted by the whole block right away.
+  const bool eas_local = EAS && me > 0 && me <= kEasLocal;
+  if (eas_local) {
+    for (int i = tid; i < me; i += NT) {
+      const unsigned d = (unsigned)__cvta_generic_to_shared(&st->eas_s[i]);
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d), "l"(eas_u + i) : "memory");
+    }
+    cp_async_commit();
+  }
   __syncthreads();
-  if (me > 0) {
-    // safeguard keys inside this block's key range: the set is sorted, so their list positions [e0, e1) are the
-    // numbers of entries below the range's two ends (counted by the whole block in one coalesced sweep)
-    for (int i = tid; i < kEasMax / 32; i += NT) st->eas_dup[i] = 0u;
+  if (EAS && me > kEasLocal) {
     const int lo_key = min(n, rank * chunk), hi_key = min(n, lo_key + chunk);
     int c_lo = 0, c_hi = 0;
     for (int i = tid; i < me; i += NT) {
@@ -442,11 +450,6 @@ bpc_decode_kernel(const DecodeParams p) {
     }
     if (lane == 0 && (c_lo | c_hi)) { atomicAdd(&st->e0, c_lo); atomicAdd(&st->e1, c_hi); }
   }
-  __syncthreads();
-  const int e0 = me > 0 ? st->e0 : 0, e1 = me > 0 ? st->e1 : 0;
-  const bool eas_local = (e1 - e0) <= kEasLocal;
-  if (eas_local)
-    for (int i = tid; i < e1 - e0; i += NT) st->eas_s[i] = eas_u[e0 + i];
   {
     constexpr int PARTS = HPARTS, DS = HDS;
     const int j = tid % B, part = tid / B;
@@ -527,6 +530,16 @@ bpc_decode_kernel(const DecodeParams p) {
   }
   cp_async_wait<0>();                                        // Gram staging (appending block only) has landed
   __syncthreads();
+  if (eas_local && (tid == 0 || tid == 32)) {                // lower bounds of the block's two range ends in the set
+    const int lo_key = min(n, rank * chunk);
+    const int bound = tid == 0 ? lo_key : min(n, lo_key + chunk);
+    int a = 0, b2 = me;
+    while (a < b2) {
+      const int mid = (a + b2) >> 1;
+      if (st->eas_s[mid] < bound) a = mid + 1; else b2 = mid;
+    }
+    if (tid == 0) st->e0 = a; else st->e1 = a;              // read after the cluster barrier that ends the scan
+  }
 
   BPC_STAMP(1);
   // ------------------------------------------------------------------ phase 1: scan
@@ -718,6 +731,7 @@ bpc_decode_kernel(const DecodeParams p) {
   }
   cluster.sync();                                            // every block's histogram is complete (and delivered)
   BPC_STAMP(8);
+  const int e0 = (EAS && me > 0) ? st->e0 : 0, e1 = (EAS && me > 0) ? st->e1 : 0;
   if (appender && tid == 0) p.unit_lens_w[unit] = n;         // every block of the cluster has read the old length
   // Threshold key T (the k-th largest score key) and this block's share of the output.
   int T;
@@ -905,18 +919,9 @@ bpc_decode_kernel(const DecodeParams p) {
     constexpr int SPT = 4;                                   // most consecutive segments one thread takes per pass
     const int spt = min(SPT, (nseg + NT - 1) / NT);
     int run_gt = 0, run_eq = 0;
-    // a selected key that also belongs to the safeguard set is flagged there, so that it is attended once
-    auto mark_dup = [&](int gi) {
-      if (EAS && me > 0) {
-        int a = 0, b2 = e1 - e0;
-        while (a < b2) {
-          const int mid = (a + b2) >> 1;
-          const int v = eas_local ? st->eas_s[mid] : eas_u[e0 + mid];
-          if (v < gi) a = mid + 1; else b2 = mid;
-        }
-        if (a < e1 - e0 && (eas_local ? st->eas_s[a] : eas_u[e0 + a]) == gi) atomicOr(&st->eas_dup[a >> 5], 1u << (a & 31));
-      }
-    };
+    // With the safeguard, every thread also leaves the mask of the keys it selected in the padding of each of its
+    // segments (slots 32, 33), where the safeguard keys of this block look themselves up afterwards: a key chosen
+    // by both sources is attended once.
     for (int s0 = 0; s0 < nseg && kh > 0; s0 += NT * spt) {
       uint32_t M[SPT], Mgt[SPT];                             // bit j: key j of the segment is >= T / > T
       int cgt = 0, ceq = 0;
@@ -959,6 +964,9 @@ bpc_decode_kernel(const DecodeParams p) {
       }
       uint32_t total;
       const uint32_t ex = block_excl_scan<NT>((uint32_t)cgt | ((uint32_t)ceq << 16), st->wscan, scan_calls, &total);
+      uint32_t TK[SPT];                                      // bit j: key j of the segment was selected
+#pragma unroll
+      for (int q = 0; q < SPT; ++q) TK[q] = 0u;
       if (cgt | ceq) {
         int eqb = run_eq + (int)(ex >> 16);
         int pos = st->my_base + run_gt + (int)(ex & 0xffffu) + min(eqb, my_take);
@@ -970,14 +978,20 @@ bpc_decode_kernel(const DecodeParams p) {
             const int j = __ffs(rem) - 1;
             rem &= rem - 1;
             const int gi = c0 + seg * kSegKeys + j;
-            if ((Mgt[q] >> j) & 1u) {
+            bool takes = true;
+            if (!((Mgt[q] >> j) & 1u)) { takes = eqb < my_take; ++eqb; }
+            if (takes) {
               sel_u[pos++] = gi;
-              mark_dup(gi);
-            } else {
-              if (eqb < my_take) { sel_u[pos++] = gi; mark_dup(gi); }
-              ++eqb;
+              if (EAS) TK[q] |= 1u << j;
             }
           }
+        }
+      }
+      if (EAS && me > 0) {
+#pragma unroll
+        for (int q = 0; q < SPT; ++q) {
+          const int seg = s0 + tid * spt + q;
+          if (q < spt && seg < nseg) *reinterpret_cast<uint32_t*>(sc + (size_t)seg * kSegSlots + kSegKeys) = TK[q];
         }
       }
       run_gt += (int)(total & 0xffffu);
@@ -988,11 +1002,12 @@ bpc_decode_kernel(const DecodeParams p) {
   const int lo = (int)(((long long)kh * rank) / CS), hi = (int)(((long long)kh * (rank + 1)) / CS);
   const int nh = hi - lo, ne = e1 - e0;                      // rows from the two sources
   if (me > 0) {
-    __syncthreads();                                         // all duplicate flags of this block are set
+    __syncthreads();                                         // the selection masks of this block are written
     for (int t = tid; t < e1 - e0; t += NT) {
-      const bool dup = (st->eas_dup[t >> 5] >> (t & 31)) & 1u;
-      const int v = dup ? -1 : (eas_local ? st->eas_s[t] : eas_u[e0 + t]);
-      sel_u[kh + e0 + t] = v;
+      const int v = eas_local ? st->eas_s[e0 + t] : eas_u[e0 + t];
+      const int rel = v - c0;                                // the key's position in this block's range
+      const bool dup = kh > 0 && ((*reinterpret_cast<const uint32_t*>(sc + (size_t)(rel >> 5) * kSegSlots + kSegKeys) >> (rel & 31)) & 1u);
+      sel_u[kh + e0 + t] = dup ? -1 : v;
     }
   }
   BPC_STAMP(3);
