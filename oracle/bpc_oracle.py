@@ -62,11 +62,15 @@ def sign_pm1(t: np.ndarray) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------- Algorithm 1
-def fit(K: np.ndarray, v_star: np.ndarray):
+def fit(K: np.ndarray, v_star: np.ndarray, power_iters: int = 0):
     """Algorithm 1: greedy binary principal components.
 
     K [N, D], v_star [b, D] (the Gaussian draws, passed in).  Returns
     P [b, D], H [N, b] in {-1,+1}, and the residual Frobenius norms after 0..b iterations.
+
+    power_iters = n > 0 takes the binary component from the power iteration the section "Binary Principal
+    Components Finding" starts from, u = sign((R R^T)^n R v*^T); n = 0 is Algorithm 1 as printed, u = sign(R v*^T).
+    The vector is rescaled between multiplications (a positive factor: the signs are those of the formula).
     """
     R = np.array(K, dtype=np.float64)
     N = R.shape[0]
@@ -75,7 +79,13 @@ def fit(K: np.ndarray, v_star: np.ndarray):
     H = np.zeros((N, b))
     trace = [np.linalg.norm(R)]
     for i in range(b):
-        u = sign_pm1(R @ np.asarray(v_star[i], dtype=np.float64))   # u <- sign(R v*^T)
+        w = R @ np.asarray(v_star[i], dtype=np.float64)              # R v*^T
+        for _ in range(power_iters):                                 # (R R^T)^n applied one factor at a time
+            nw = np.linalg.norm(w)
+            if nw > 0.0:
+                w = w / nw
+            w = R @ (R.T @ w)
+        u = sign_pm1(w)                                              # u <- sign(...)
         v = (u @ R) / N                                              # v <- u R / N
         R = R - np.outer(u, v)                                       # R <- R - u^T v
         H[:, i] = u

@@ -358,3 +358,57 @@ def test_decode_unit_with_safeguard_set():
     assert np.allclose(r["out"], O.attend(q, K, V, r["idx"]), atol=1e-13)
     tiny = O.decode_unit(q, K, V, bits, P, ppm=0, count=3, s_err=s_err)   # budget below the safeguard size
     assert list(tiny["idx"]) == list(s_err[:3]) and len(tiny["hash_idx"]) == 0
+
+
+def test_fit_power_iteration_finds_the_sign_of_the_top_singular_vector():
+    """Section "Binary Principal Components Finding": u = sign((R R^T)^n R v*^T) tends to the sign pattern of R's largest
+    left singular vector as n grows (library SVD as the outside reference), even from a start that is nearly
+    orthogonal to the top right singular vector, where the printed n = 0 rule picks up other directions."""
+    rng = np.random.default_rng(77)
+    N, D = 400, 16
+    a = rng.standard_normal(N); a /= np.linalg.norm(a)
+    bvec = rng.standard_normal(D); bvec /= np.linalg.norm(bvec)
+    K = 40.0 * np.outer(a, bvec) + 0.5 * rng.standard_normal((N, D))
+    U, S, Vt = np.linalg.svd(K, full_matrices=False)
+    assert S[0] > 3 * S[1]
+    top = np.sign(U[:, 0])
+    # a start direction with only a small component along the top right singular vector
+    g = rng.standard_normal(D)
+    g -= (g @ Vt[0]) * Vt[0]
+    v0 = (g / np.linalg.norm(g) + 0.02 * Vt[0])[None, :]
+    _, H0, _ = O.fit(K, v0, power_iters=0)
+    _, H8, _ = O.fit(K, v0, power_iters=8)
+    agree0 = max(np.mean(H0[:, 0] == top), np.mean(H0[:, 0] == -top))
+    agree8 = max(np.mean(H8[:, 0] == top), np.mean(H8[:, 0] == -top))
+    assert agree8 == 1.0
+    assert agree0 < 0.9
+    # and the first binary component then removes more of the matrix
+    _, _, tr0 = O.fit(K, v0, power_iters=0)
+    _, _, tr8 = O.fit(K, v0, power_iters=8)
+    assert tr8[1] < tr0[1]
+
+
+def test_fit_power_iteration_zero_is_algorithm_1_and_residual_gram_downdate():
+    """n = 0 reproduces Algorithm 1 exactly; and one greedy step changes the residual's Gram matrix by a rank-one term,
+    (R - u^T v)^T (R - u^T v) = R^T R - N v^T v (because u R = N v and u u^T = N), the closed form that lets
+    (R R^T)^n R v*^T = R (R^T R)^n v*^T be evaluated without extra passes over R."""
+    rng = np.random.default_rng(5)
+    K = rng.standard_normal((300, 12)) * np.linspace(0.2, 3.0, 12)
+    vs = rng.standard_normal((6, 12))
+    Pa, Ha, _ = O.fit(K, vs)
+    Pb, Hb, _ = O.fit(K, vs, power_iters=0)
+    assert np.array_equal(Pa, Pb) and np.array_equal(Ha, Hb)
+    R = K.copy()
+    N = R.shape[0]
+    C = R.T @ R
+    for i in range(3):
+        z = np.linalg.matrix_power(C, 2) @ vs[i]
+        u = O.sign_pm1(R @ z)
+        w = R @ vs[i]
+        for _ in range(2):
+            w = R @ (R.T @ w)
+        assert np.array_equal(u, O.sign_pm1(w))                     # R (R^T R)^n v = (R R^T)^n R v
+        v = (u @ R) / N
+        R = R - np.outer(u, v)
+        C = C - N * np.outer(v, v)
+        assert np.allclose(C, R.T @ R, rtol=1e-10, atol=1e-9)
