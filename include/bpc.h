@@ -73,6 +73,7 @@ typedef struct {
   int32_t kv_row_stride;        /* elements between consecutive cache rows; 0 selects head_dim */
   int32_t eas_ppm;              /* error-aware safeguard: size of the hard-to-hash set as parts per million of the
                                    keys cached when bpc_build_eas runs (0 = no safeguard; at most 16384 keys per unit) */
+  int32_t fit_power_iters;      /* bpc_fit: n in u = sign((R R^T)^n R v*^T), 0..8; 0 is Algorithm 1 as printed */
 } bpc_config;
 
 typedef struct bpc_ctx bpc_ctx;
@@ -104,7 +105,10 @@ bpc_status bpc_get_seq_lens(bpc_ctx* ctx, int32_t* host_lens_out);
  * float are the Gaussian directions the algorithm samples (supplied by the caller so that a run is
  * reproducible).  workspace must hold bpc_fit_workspace_bytes(cfg).  Requires hash_sets ==
  * batch*n_kv_heads.  Leaves P, P rounded to the cache precision (the hash function proper) and
- * its Gram matrix in the context. */
+ * its Gram matrix in the context.  With cfg.fit_power_iters = n > 0 the binary component comes from the power
+ * iteration the same section starts from, u = sign((R R^T)^n R v*^T) = sign(R (R^T R)^n v*^T): the head_dim x head_dim
+ * matrix R^T R is formed once (one extra pass over the keys) and then follows the residual by the rank-one change
+ * -N v^T v per iteration, so the passes over R stay one per bit. */
 bpc_status bpc_fit(bpc_ctx* ctx, const void* k_cache, const float* v_star,
                    void* workspace, size_t workspace_bytes, void* stream);
 

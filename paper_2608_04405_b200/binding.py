@@ -32,7 +32,8 @@ class bpc_config(ctypes.Structure):
     _fields_ = [("batch", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
                 ("head_dim", ctypes.c_int32), ("code_bits", ctypes.c_int32), ("n_max", ctypes.c_int32),
                 ("kv_dtype", ctypes.c_int32), ("score_mode", ctypes.c_int32), ("sm_scale", ctypes.c_float),
-                ("hash_sets", ctypes.c_int32), ("residual_correction", ctypes.c_int32), ("kv_row_stride", ctypes.c_int32), ("eas_ppm", ctypes.c_int32)]
+                ("hash_sets", ctypes.c_int32), ("residual_correction", ctypes.c_int32), ("kv_row_stride", ctypes.c_int32), ("eas_ppm", ctypes.c_int32),
+                ("fit_power_iters", ctypes.c_int32)]
 
 
 def _load() -> ctypes.CDLL:
@@ -119,10 +120,10 @@ def _check(status: int, what: str) -> None:
 def make_config(batch: int, n_q_heads: int, n_kv_heads: int, n_max: int, code_bits: int, dtype: torch.dtype,
                 score_mode: int = BPC_SCORE_HAMMING, sm_scale: float = 0.0, shared_projection: bool = False,
                 residual_correction: bool = True, head_dim: int = 128, kv_row_stride: int = 0,
-                eas_ppm: int = 0) -> bpc_config:
+                eas_ppm: int = 0, fit_power_iters: int = 0) -> bpc_config:
     return bpc_config(batch, n_q_heads, n_kv_heads, head_dim, code_bits, n_max,
                       BPC_BF16 if dtype == torch.bfloat16 else BPC_F32, score_mode, sm_scale,
-                      n_kv_heads if shared_projection else batch * n_kv_heads, 1 if residual_correction else 0, kv_row_stride, eas_ppm)
+                      n_kv_heads if shared_projection else batch * n_kv_heads, 1 if residual_correction else 0, kv_row_stride, eas_ppm, fit_power_iters)
 
 
 class Context:

@@ -38,6 +38,7 @@ bpc_status check_cfg(const bpc_config* c) {
   if (!(c->sm_scale >= 0.f)) return BPC_ERR_INVALID_ARG;
   if (c->kv_row_stride != 0 && (c->kv_row_stride < c->head_dim || c->kv_row_stride % 8 != 0)) return BPC_ERR_INVALID_ARG;
   if (c->eas_ppm < 0 || c->eas_ppm > 1000000) return BPC_ERR_INVALID_ARG;
+  if (c->fit_power_iters < 0 || c->fit_power_iters > 8) return BPC_ERR_INVALID_ARG;
   if (c->eas_ppm > 0 && (c->residual_correction == 0 || c->score_mode != BPC_SCORE_HAMMING)) return BPC_ERR_UNSUPPORTED;
   if (c->eas_ppm > 0 && ((long long)c->n_max * c->eas_ppm + 999999) / 1000000 > 16384) return BPC_ERR_UNSUPPORTED;
   if (c->n_max % 2 != 0) return BPC_ERR_INVALID_ARG;   // keeps every unit's code rows 16-byte aligned at 64 bits

@@ -227,13 +227,16 @@ template <typename KV>
 __global__ void __launch_bounds__(kFitThreads)
 fit_pass_kernel(const KV* __restrict__ k_cache, float* __restrict__ R, uint8_t* __restrict__ usign,
                 uint32_t* __restrict__ hfit, const float* __restrict__ v_star, const float* __restrict__ P, float* __restrict__ partials,
-                const int32_t* __restrict__ unit_lens, int n_max, int row_stride, int b, int it, int blocks_per_unit) {
+                const int32_t* __restrict__ unit_lens, int n_max, int row_stride, int b, int it, int blocks_per_unit,
+                const float* __restrict__ dir) {
   const int unit = blockIdx.y;
   const int n = min(unit_lens[unit], n_max);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int row0 = blockIdx.x * kFitRowsPerBlock;
   __shared__ float red[kFitThreads / 32][BPC_D];
-  const float4 vs = reinterpret_cast<const float4*>(v_star + ((size_t)unit * b + it) * BPC_D)[lane];
+  // direction of the projection: the caller's draw v*_i, or (power-iteration fit) (R^T R)^n v*_i prepared per unit
+  const float4 vs = dir != nullptr ? reinterpret_cast<const float4*>(dir + (size_t)unit * BPC_D)[lane]
+                                   : reinterpret_cast<const float4*>(v_star + ((size_t)unit * b + it) * BPC_D)[lane];
   float4 vp = make_float4(0.f, 0.f, 0.f, 0.f);
   if (it > 0) vp = reinterpret_cast<const float4*>(P + ((size_t)unit * b + (it - 1)) * BPC_D)[lane];
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -283,6 +286,111 @@ __global__ void fit_reduce_kernel(const float* __restrict__ partials, float* __r
   double s = 0.0;
   for (int k = 0; k < nblk; ++k) s += (double)partials[((size_t)unit * blocks_per_unit + k) * BPC_D + c];
   P[((size_t)unit * b + it) * BPC_D + c] = n > 0 ? (float)(s / (double)n) : 0.f;
+}
+
+// --------------------------------------------------------------------------- power-iteration fit
+// u = sign((R R^T)^n R v*^T) = sign(R z) with z = (R^T R)^n v*^T.  C = R^T R (D x D, fp64) is formed once from the keys
+// and then follows the residual through C <- C - N v^T v (u R = N v and u u^T = N make the cross terms collapse), so
+// a power-iteration fit costs one extra pass over the keys and a D x D product per bit.
+constexpr int kGramRows = 8192;          // key rows per block of the initial Gram pass
+
+// One block per (row slab, unit): its 256 threads own 8 x 8 tiles of the D x D partial sum.  Rows are staged 32 at a
+// time in shared memory; a tile of 32 rows is summed in fp32 and added to fp64 accumulators.
+template <typename KV>
+__global__ void __launch_bounds__(256, 1)
+fit_gram0_kernel(const KV* __restrict__ k_cache, double* __restrict__ cpart, const int32_t* __restrict__ unit_lens,
+                 int n_max, int row_stride, int slabs_per_unit) {
+  const int unit = blockIdx.y, tid = threadIdx.x;
+  const int n = min(unit_lens[unit], n_max);
+  const int row0 = blockIdx.x * kGramRows, row_end = min(n, row0 + kGramRows);
+  __shared__ float tile[32][BPC_D + 4];
+  const int i0 = (tid >> 4) * 8, j0 = (tid & 15) * 8;
+  double acc[8][8];
+#pragma unroll
+  for (int a = 0; a < 8; ++a)
+#pragma unroll
+    for (int c = 0; c < 8; ++c) acc[a][c] = 0.0;
+  for (int r0 = row0; r0 < row_end; r0 += 32) {
+    __syncthreads();
+    for (int e = tid; e < 32 * BPC_D; e += 256) {
+      const int r = e >> 7, c = e & 127;
+      tile[r][c] = (r0 + r < row_end) ? to_float(k_cache[((size_t)unit * n_max + r0 + r) * row_stride + c]) : 0.f;
+    }
+    __syncthreads();
+    float part[8][8];
+#pragma unroll
+    for (int a = 0; a < 8; ++a)
+#pragma unroll
+      for (int c = 0; c < 8; ++c) part[a][c] = 0.f;
+#pragma unroll 4
+    for (int r = 0; r < 32; ++r) {
+      float xa[8], xb[8];
+#pragma unroll
+      for (int a = 0; a < 8; ++a) { xa[a] = tile[r][i0 + a]; xb[a] = tile[r][j0 + a]; }
+#pragma unroll
+      for (int a = 0; a < 8; ++a)
+#pragma unroll
+        for (int c = 0; c < 8; ++c) part[a][c] = fmaf(xa[a], xb[c], part[a][c]);
+    }
+#pragma unroll
+    for (int a = 0; a < 8; ++a)
+#pragma unroll
+      for (int c = 0; c < 8; ++c) acc[a][c] += (double)part[a][c];
+  }
+  double* dst = cpart + ((size_t)unit * slabs_per_unit + blockIdx.x) * BPC_D * BPC_D;
+#pragma unroll
+  for (int a = 0; a < 8; ++a)
+#pragma unroll
+    for (int c = 0; c < 8; ++c) dst[(size_t)(i0 + a) * BPC_D + j0 + c] = acc[a][c];
+}
+
+// C[unit] = sum of the slabs' partial sums, in slab order
+__global__ void fit_gram0_reduce_kernel(const double* __restrict__ cpart, double* __restrict__ C,
+                                        const int32_t* __restrict__ unit_lens, int n_max, int slabs_per_unit) {
+  const int unit = blockIdx.y, e = blockIdx.x * blockDim.x + threadIdx.x;
+  const int n = min(unit_lens[unit], n_max);
+  const int nslab = (n + kGramRows - 1) / kGramRows;
+  double s = 0.0;
+  for (int k = 0; k < nslab; ++k) s += cpart[((size_t)unit * slabs_per_unit + k) * BPC_D * BPC_D + e];
+  C[(size_t)unit * BPC_D * BPC_D + e] = s;
+}
+
+// One block of D threads per unit, before the pass of bit `it`: apply the previous bit's downdate C -= N v v^T (v = row
+// it-1 of P), then z = C^n v*_it with a rescale between the products, written as the pass's direction (fp32).
+__global__ void __launch_bounds__(BPC_D)
+fit_direction_kernel(double* __restrict__ C, const float* __restrict__ P, const float* __restrict__ v_star,
+                     float* __restrict__ dir, const int32_t* __restrict__ unit_lens, int n_max, int b, int it, int power_iters) {
+  const int unit = blockIdx.x, j = threadIdx.x;
+  const int n = min(unit_lens[unit], n_max);
+  double* Cu = C + (size_t)unit * BPC_D * BPC_D;
+  __shared__ double z[BPC_D];
+  __shared__ double red[BPC_D / 32];
+  __shared__ float vprev[BPC_D];
+  if (it > 0) {
+    vprev[j] = P[((size_t)unit * b + (it - 1)) * BPC_D + j];
+    __syncthreads();
+    const double nv = (double)n * (double)vprev[j];
+    for (int c = 0; c < BPC_D; ++c) Cu[(size_t)c * BPC_D + j] -= nv * (double)vprev[c];   // column j (C is symmetric)
+  }
+  z[j] = (double)v_star[((size_t)unit * b + it) * BPC_D + j];
+  __syncthreads();
+  for (int k = 0; k < power_iters; ++k) {
+    double s = 0.0;
+    for (int c = 0; c < BPC_D; ++c) s += Cu[(size_t)c * BPC_D + j] * z[c];                // (C z)_j, reading column j
+    double q = s * s;
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+    __syncthreads();                                        // everyone has read z
+    if ((j & 31) == 0) red[j >> 5] = q;
+    __syncthreads();
+    double nrm = 0.0;
+#pragma unroll
+    for (int w = 0; w < BPC_D / 32; ++w) nrm += red[w];
+    nrm = sqrt(nrm);
+    z[j] = nrm > 0.0 ? s / nrm : s;
+    __syncthreads();
+  }
+  dir[(size_t)unit * BPC_D + j] = (float)z[j];
 }
 
 // --------------------------------------------------------------------------- error-aware safeguard set
@@ -416,11 +524,19 @@ cudaError_t bpc_launch_append(bpc_ctx* ctx, const void* k_new, const void* v_new
 
 static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
+// extra workspace of the power-iteration fit, placed after the fitted codes: C, the slabs' partial sums, the directions
+static size_t fit_power_bytes(const bpc_config* c) {
+  if (c->fit_power_iters <= 0) return 0;
+  const size_t units = (size_t)c->batch * c->n_kv_heads;
+  const size_t slabs = ((size_t)c->n_max + kGramRows - 1) / kGramRows;
+  return align256(units * BPC_D * BPC_D * 8) + align256(units * slabs * BPC_D * BPC_D * 8) + align256(units * BPC_D * 4);
+}
+
 size_t bpc_fit_workspace_bytes_impl(const bpc_config* c) {
   const size_t units = (size_t)c->batch * c->n_kv_heads;
   const size_t bpu = ((size_t)c->n_max + kFitRowsPerBlock - 1) / kFitRowsPerBlock;
   return align256(units * c->n_max * BPC_D * 4) + align256(units * c->n_max) + align256(units * bpu * BPC_D * 4) +
-         align256(units * c->n_max * (c->code_bits / 8));
+         align256(units * c->n_max * (c->code_bits / 8)) + fit_power_bytes(c);
 }
 
 size_t bpc_fit_codes_offset_impl(const bpc_config* c) {
@@ -440,13 +556,34 @@ cudaError_t bpc_launch_fit(bpc_ctx* ctx, const void* k_cache, const float* v_sta
   float* partials = (float*)(usign + align256(units * c.n_max));
   uint32_t* hfit = (uint32_t*)(ws + bpc_fit_codes_offset_impl(&c));
   const dim3 grid(bpu, ctx->units);
+  const int npow = c.fit_power_iters;
+  double* Cm = nullptr;
+  float* dir = nullptr;
+  if (npow > 0) {
+    const int slabs = (c.n_max + kGramRows - 1) / kGramRows;
+    unsigned char* pw = (unsigned char*)hfit + align256(units * c.n_max * (c.code_bits / 8));
+    Cm = (double*)pw;
+    double* cpart = (double*)(pw + align256(units * BPC_D * BPC_D * 8));
+    dir = (float*)(pw + align256(units * BPC_D * BPC_D * 8) + align256(units * (size_t)slabs * BPC_D * BPC_D * 8));
+    const dim3 g0(slabs, ctx->units);
+    if (c.kv_dtype == BPC_BF16)
+      fit_gram0_kernel<__nv_bfloat16><<<g0, 256, 0, stream>>>((const __nv_bfloat16*)k_cache, cpart, ctx->unit_lens, c.n_max, ctx->row_stride, slabs);
+    else
+      fit_gram0_kernel<float><<<g0, 256, 0, stream>>>((const float*)k_cache, cpart, ctx->unit_lens, c.n_max, ctx->row_stride, slabs);
+    fit_gram0_reduce_kernel<<<dim3(BPC_D * BPC_D / 256, ctx->units), 256, 0, stream>>>(cpart, Cm, ctx->unit_lens, c.n_max, slabs);
+    *launches += 2;
+  }
   for (int it = 0; it < c.code_bits; ++it) {
+    if (npow > 0) {
+      fit_direction_kernel<<<ctx->units, BPC_D, 0, stream>>>(Cm, ctx->P, v_star, dir, ctx->unit_lens, c.n_max, c.code_bits, it, npow);
+      *launches += 1;
+    }
     if (c.kv_dtype == BPC_BF16)
       fit_pass_kernel<__nv_bfloat16><<<grid, kFitThreads, 0, stream>>>((const __nv_bfloat16*)k_cache, R, usign, hfit, v_star, ctx->P,
-                                                                        partials, ctx->unit_lens, c.n_max, ctx->row_stride, c.code_bits, it, bpu);
+                                                                        partials, ctx->unit_lens, c.n_max, ctx->row_stride, c.code_bits, it, bpu, dir);
     else
       fit_pass_kernel<float><<<grid, kFitThreads, 0, stream>>>((const float*)k_cache, R, usign, hfit, v_star, ctx->P, partials,
-                                                               ctx->unit_lens, c.n_max, ctx->row_stride, c.code_bits, it, bpu);
+                                                               ctx->unit_lens, c.n_max, ctx->row_stride, c.code_bits, it, bpu, dir);
     fit_reduce_kernel<<<ctx->units, BPC_D, 0, stream>>>(partials, ctx->P, ctx->unit_lens, c.n_max, c.code_bits, it, bpu);
     *launches += 2;
   }

@@ -39,7 +39,7 @@ class Session:
     """A workload on the GPU with its library context, fitted and encoded."""
 
     def __init__(self, spec: WorkloadSpec, gen_device: str = "cpu", salt: int = 0, cluster_size: int = 0,
-                 extra_rows=None, interleaved: bool = False, score_mode: int = 0, eas_ppm: int = 0):
+                 extra_rows=None, interleaved: bool = False, score_mode: int = 0, eas_ppm: int = 0, fit_power_iters: int = 0):
         self.spec = spec
         self.w = Workload(spec, device=gen_device, extra_rows=extra_rows, salt=salt)
         dev = "cuda"
@@ -54,7 +54,7 @@ class Session:
         self.v_star = self.w.v_star.to(dev)
         self.cfg = B.make_config(spec.batch, spec.n_q_heads, spec.n_kv_heads, self.w.n_max, spec.code_bits,
                                  spec.torch_dtype, kv_row_stride=2 * spec.head_dim if interleaved else 0,
-                                 score_mode=score_mode, eas_ppm=eas_ppm)
+                                 score_mode=score_mode, eas_ppm=eas_ppm, fit_power_iters=fit_power_iters)
         self.s_err = None
         self.ctx = B.Context(self.cfg)
         if cluster_size:
@@ -103,12 +103,17 @@ def check_fit(sess: Session, units, report: dict):
         R = K.copy()
         amb = hard = 0
         Pref = np.zeros_like(gpuP)
+        npow = int(sess.cfg.fit_power_iters)
         for i in range(s.code_bits):
-            t = R @ vs[i]
+            z = vs[i].copy()                                 # direction: v*, or (R^T R)^n v* for the power-iteration fit
+            for _ in range(npow):
+                z = R.T @ (R @ z)
+                z = z / max(np.linalg.norm(z), 1e-300)
+            t = R @ z
             mine = t >= 0
             theirs = gpuH[:, i].astype(bool)
             diff = mine != theirs
-            tau = 1e-5 * np.linalg.norm(R, axis=1) * np.linalg.norm(vs[i])
+            tau = 1e-5 * np.linalg.norm(R, axis=1) * np.linalg.norm(z)
             hard += int(np.count_nonzero(diff & (np.abs(t) >= tau)))
             amb += int(np.count_nonzero(diff & (np.abs(t) < tau)))
             uu = np.where(theirs, 1.0, -1.0)
@@ -128,7 +133,7 @@ def check_fit(sess: Session, units, report: dict):
         report["fit_max_rel_err"] = max(report.get("fit_max_rel_err", 0.0), float(rel.max()))
         # pure-checker fit from scratch agrees wherever no sign was ambiguous
         if amb == 0:
-            P0, _, _ = O.fit(K, vs)
+            P0, _, _ = O.fit(K, vs, power_iters=npow)
             rel0 = np.linalg.norm(gpuP - P0, axis=1) / np.maximum(np.linalg.norm(P0, axis=1), 1e-30)
             assert rel0.max() <= 2e-5
 

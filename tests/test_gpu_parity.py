@@ -143,6 +143,35 @@ def test_shared_projection_per_kv_head():
     H.check_decode(sess, q.cuda(), [0, 3], rep)
 
 
+def test_offline_projection_calibration_on_aggregated_keys():
+    """Offline Projection Calibration (Section 3.2): Algorithm 1 runs once, ahead of serving, on keys aggregated over
+    several sequences (here with two power iterations), one projection per KV head; the serving context takes that
+    projection through bpc_set_projection and shares it among all its sequences."""
+    H = _harness()
+    from paper_2608_04405_b200 import binding as B
+    spec = CONFIGS[1].scaled(name="serve", wid=71, batch=3, n_ctx=1500, n_kv_heads=2, n_q_heads=8, steps=1)
+    serve = H.Session(spec)
+    # calibration context: one "sequence" per KV head holding the keys of all serving sequences of that head
+    n_agg = spec.batch * spec.n_ctx
+    cal_spec = spec.scaled(name="calib", wid=72, batch=1, n_ctx=n_agg)
+    cal = H.Session(cal_spec, fit_power_iters=2)
+    for h in range(spec.n_kv_heads):
+        cal.k_cache[0, h, :n_agg] = torch.cat([serve.k_cache[b, h, :spec.n_ctx] for b in range(spec.batch)], dim=0)
+    rep = {}
+    cal.fit(); H.check_fit(cal, [0, 1], rep)
+    cfg = B.make_config(spec.batch, spec.n_q_heads, spec.n_kv_heads, serve.w.n_max, spec.code_bits, spec.torch_dtype,
+                        shared_projection=True)
+    ctx2 = B.Context(cfg)
+    ctx2.set_seq_lens(serve.lens)
+    ctx2.set_projection(cal.P.contiguous())
+    serve.ctx, serve.cfg = ctx2, cfg
+    serve.P, serve.Ph, serve.gram = ctx2.get_projection()
+    serve.encode(); H.check_encode(serve, [0, 3, 5], rep)
+    q, _ = serve.w.queries(serve.lens)
+    H.check_decode(serve, q.cuda(), [0, 5], rep)
+    print(rep)
+
+
 def test_fused_append_decode_tiny_and_boundary_lengths():
     """Fused cache write at lengths where the new key opens a new chunk / a new 32-key segment, and from n = 0."""
     H = _harness()
@@ -315,6 +344,23 @@ def test_cfg4_full_size_sampled_units():
     sess.fit(); H.check_fit(sess, [17], rep)
     sess.encode(); H.check_encode(sess, [2, 31], rep, key_slice=(60000, 64096))
     _decode_loop(sess, 2, [0, 19, 31], rep, H, fused=True)
+    print(rep)
+
+
+@pytest.mark.parametrize("dtype,bits,n,power", [("bf16", 128, 20000, 2), ("f32", 64, 9000, 1), ("bf16", 64, 70000, 4)])
+def test_fit_with_power_iterations(dtype, bits, n, power):
+    """bpc_fit with cfg.fit_power_iters = n: the binary component of every bit is sign((R R^T)^n R v*^T) (section "Binary
+    Principal Components Finding"); replayed by the checker with the library's signs adopted inside the fp32 ambiguity
+    band, then the usual encode and decode checks on the projection it produced."""
+    H = _harness()
+    spec = CONFIGS[1].scaled(name="powerfit", wid=60 + power, batch=2, n_q_heads=8, n_kv_heads=2, n_ctx=n, dtype=dtype,
+                             code_bits=bits, steps=2)
+    sess = H.Session(spec, gen_device="cuda", fit_power_iters=power)
+    rep = {}
+    sess.fit(); H.check_fit(sess, [0, 3], rep)
+    sess.encode(); H.check_encode(sess, [1], rep, max_keys=4096)
+    q, _ = sess.w.queries(sess.lens)
+    H.check_decode(sess, q.cuda(), [0, 3], rep)
     print(rep)
 
 
