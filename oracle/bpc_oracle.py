@@ -229,6 +229,37 @@ def attend(q_group: np.ndarray, K: np.ndarray, V: np.ndarray, idx: np.ndarray, s
     return w @ Vs
 
 
+# --------------------------------------------------------------------------- quality yard-sticks
+def exact_topk(q_head: np.ndarray, K: np.ndarray, k: int) -> np.ndarray:
+    """The TOPK (Oracle) baseline of the appendix "Baseline Methods": the k keys with the largest exact attention
+    scores q . k_i for ONE query head (full precision), ties to the lowest index, returned in ascending index order."""
+    scores = np.asarray(K, dtype=np.float64) @ np.asarray(q_head, dtype=np.float64)
+    k = max(0, min(int(k), scores.shape[0]))
+    order = np.lexsort((np.arange(scores.shape[0]), -scores))
+    return np.sort(order[:k]).astype(np.int64)
+
+
+def dense_attend(q_group: np.ndarray, K: np.ndarray, V: np.ndarray, sm_scale: float = 0.0) -> np.ndarray:
+    """Full softmax attention over every cached key (the reference the sparse output is compared with)."""
+    return attend(q_group, K, V, np.arange(np.asarray(K).shape[0]), sm_scale)
+
+
+def selection_recall(selected: np.ndarray, reference: np.ndarray) -> float:
+    """Fraction of the reference set that the selection contains."""
+    reference = np.asarray(reference)
+    if reference.size == 0:
+        return 1.0
+    return float(np.isin(reference, np.asarray(selected)).mean())
+
+
+def cosine_similarity(a: np.ndarray, b: np.ndarray) -> float:
+    """cos(a, b) of two vectors (appendix table "cosine similarity between sparse and full attention outputs")."""
+    a = np.asarray(a, dtype=np.float64).ravel()
+    b = np.asarray(b, dtype=np.float64).ravel()
+    den = np.linalg.norm(a) * np.linalg.norm(b)
+    return float(a @ b / den) if den > 0.0 else 0.0
+
+
 # --------------------------------------------------------------------------- Error-Aware Safeguard (Eqs. 8-9)
 def eas_set(errors: np.ndarray, m: int) -> np.ndarray:
     """Hard-to-hash set S_err: indices of the m largest reconstruction errors ||k - h P||_2 (Eq. 8), ties to the

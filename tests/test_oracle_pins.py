@@ -412,3 +412,30 @@ def test_fit_power_iteration_zero_is_algorithm_1_and_residual_gram_downdate():
         R = R - np.outer(u, v)
         C = C - N * np.outer(v, v)
         assert np.allclose(C, R.T @ R, rtol=1e-10, atol=1e-9)
+
+
+def test_quality_yardsticks_against_brute_force_and_closed_forms():
+    """TOPK (Oracle) baseline and the output-similarity measure (appendix "Baseline Methods" and the cosine table):
+    exact_topk against a brute-force rank count, dense attention against attention over the full index set and the
+    uniform-logit closed form, recall and cosine on hand-made cases."""
+    rng = np.random.default_rng(11)
+    K = rng.standard_normal((57, 6)); K[9] = K[3]; K[20] = K[3]          # exact ties
+    q = rng.standard_normal(6)
+    k = 10
+    got = O.exact_topk(q, K, k)
+    s = K @ q
+    # brute force: key i is selected iff fewer than k keys beat it (larger score, or equal score and lower index)
+    beats = [(np.sum(s > s[i]) + np.sum((s == s[i]) & (np.arange(57) < i))) < k for i in range(57)]
+    assert np.array_equal(got, np.nonzero(beats)[0])
+    assert O.exact_topk(q, K, 0).size == 0 and np.array_equal(O.exact_topk(q, K, 99), np.arange(57))
+    # dense attention: all-zero query -> uniform weights -> the mean of V
+    V = rng.standard_normal((57, 6))
+    out = O.dense_attend(np.zeros((2, 6)), K, V)
+    assert np.allclose(out, np.tile(V.mean(0), (2, 1)))
+    qg = rng.standard_normal((3, 6))
+    assert np.allclose(O.dense_attend(qg, K, V), O.attend(qg, K, V, np.arange(57)))
+    # selecting every key makes sparse = dense; recall and cosine on small cases
+    assert O.selection_recall([1, 2, 3, 4], [2, 4, 6, 8]) == 0.5
+    assert O.selection_recall([], []) == 1.0
+    assert abs(O.cosine_similarity([1, 0], [1, 1]) - 2 ** -0.5) < 1e-15
+    assert O.cosine_similarity([1, 2, 3], [-2, -4, -6]) == -1.0
