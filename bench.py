@@ -531,6 +531,69 @@ def run_sweep(args):
                       "steps": K, "warmup": W, "cases": rows}))
 
 
+# ----------------------------------------------------------------------------- quality yard-sticks
+def run_quality(args):
+    """Selection quality on the synthetic workload for code lengths 64, 128 and 256: recall of the hash selection with
+    respect to the exact-score top-k of every query head (the paper's TOPK (Oracle) baseline), cosine similarity between
+    the sparse output and dense attention (the paper's output-similarity table), and recall of the planted needles.
+    All three selections and both outputs come from the library (bpc_exact_topk, bpc_decode_attn with the workload's
+    budget and with a budget of all keys); torch only intersects index sets and takes the cosine of the outputs."""
+    from paper_2608_04405_b200 import binding as B
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    spec0 = CONFIGS[args.workload]
+    rows = []
+    for bits in (64, 128, 256):
+        spec = spec0.scaled(code_bits=bits)
+        w = Workload(spec, device="cuda", extra_rows=64)
+        cfg = B.make_config(spec.batch, spec.n_q_heads, spec.n_kv_heads, w.n_max, bits, spec.torch_dtype)
+        ctx = B.Context(cfg)
+        ctx.set_seq_lens(w.seq_lens)
+        codes = ctx.alloc_codes()
+        ws = torch.empty(ctx.fit_workspace_bytes(), dtype=torch.uint8, device="cuda")
+        ctx.fit(w.k_cache, w.v_star, ws)
+        del ws
+        ctx.encode_keys(w.k_cache, codes)
+        q, needles = w.queries(w.seq_lens)
+        units = spec.batch * spec.n_kv_heads
+        dense = ctx.decode_attn(q, w.k_cache, w.v_cache, codes, budget_ppm=1000000)
+        _, tsel, tcnt = ctx.exact_topk(q, w.k_cache, budget_ppm=spec.budget_ppm)
+        G = spec.group
+        P, _, _ = ctx.get_projection()
+        for mode_name, mode in (("hamming", B.BPC_SCORE_HAMMING), ("weighted7", B.BPC_SCORE_WEIGHTED7)):
+            mctx = ctx
+            if mode != B.BPC_SCORE_HAMMING:     # Algorithm 3's sign + seven magnitude planes, same projection and codes
+                try:
+                    mctx = B.Context(B.make_config(spec.batch, spec.n_q_heads, spec.n_kv_heads, w.n_max, bits, spec.torch_dtype,
+                                                   score_mode=mode))
+                except Exception as e:          # scores beyond 16 bits for this code length and group size
+                    rows.append({"code_bits": bits, "score_mode": mode_name, "unsupported": str(e)[:100]})
+                    continue
+                mctx.set_projection(P)
+                mctx.set_seq_lens(w.seq_lens)
+            hsel = torch.full((units, w.n_max), -1, dtype=torch.int32, device="cuda")
+            sparse = mctx.decode_attn(q, w.k_cache, w.v_cache, codes, budget_ppm=spec.budget_ppm, sel_idx=hsel)
+            torch.cuda.synchronize()
+            rec, nrec = [], []
+            for bi in range(spec.batch):
+                for hq in range(spec.n_q_heads):
+                    u = bi * spec.n_kv_heads + hq // G
+                    head = bi * spec.n_q_heads + hq
+                    k = int(tcnt[head])
+                    mine = hsel[u, :k]
+                    rec.append(float(torch.isin(tsel[head, :k], mine).float().mean()))
+                    nrec.append(float(torch.isin(needles[bi, hq], mine).float().mean()))
+            cos = torch.nn.functional.cosine_similarity(sparse.reshape(-1, spec.head_dim), dense.reshape(-1, spec.head_dim), dim=1)
+            rows.append({"code_bits": bits, "score_mode": mode_name, "recall_vs_exact_topk": sum(rec) / len(rec),
+                         "cosine_sparse_vs_dense": float(cos.mean()), "cosine_min": float(cos.min()),
+                         "needle_recall": sum(nrec) / len(nrec), "device_error_word": mctx.last_device_error()})
+        del ctx, mctx, codes, w, hsel, tsel, sparse, dense
+        torch.cuda.empty_cache()
+    print(json.dumps({"metric": "selection_quality", "data": "synthetic", "dtype": "bf16",
+                      "config": {"workload": spec0.name, "budget_ppm": spec0.budget_ppm, "code_bits": [64, 128, 256],
+                                 "note": "32-bit codes are not supported by this library"},
+                      "cases": rows}))
+
+
 # ----------------------------------------------------------------------------- CPU checker arm
 def _oracle_unit_setup(spec, seed_salt=0):
     """One unit of the workload prepared for the checker: keys, values, projection, codes (prefill, untimed)."""
@@ -609,6 +672,7 @@ def main():
     ap.add_argument("--separate-kv", action="store_true", help="separate K and V arrays instead of interleaved rows")
     ap.add_argument("--profile", action="store_true", help="warm-up plus K eager steps only (for ncu captures)")
     ap.add_argument("--sweep", action="store_true", help="second workload: latency over contexts and batch sizes, 64-bit codes, 1K/2K budgets")
+    ap.add_argument("--quality", action="store_true", help="selection quality yard-sticks (recall vs exact top-k, cosine vs dense) for 64/128/256-bit codes")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -616,6 +680,8 @@ def main():
         run_reference(args)
     elif args.sweep:
         run_sweep(args)
+    elif args.quality:
+        run_quality(args)
     else:
         run_ours(args)
 

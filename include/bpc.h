@@ -191,6 +191,16 @@ bpc_status bpc_decode_attn_static(const bpc_config* host_cfg, const void* q, con
                                   int32_t budget_ppm, int32_t budget_count, float* out, void* stream);
 size_t     bpc_static_scratch_entries(void);
 
+/* Quality yard-stick: the exact-score selector (appendix "Baseline Methods", TOPK (Oracle)).  For every query head,
+ * scores[(seq * n_q_heads + head)][i] = q_head . k_i over the cached keys (fp32) and the k keys with the largest
+ * scores (k from the budget as in bpc_decode_attn; ties to the lowest index) in ascending index order in
+ * sel_out[(seq * n_q_heads + head)][0..k), with k in count_out[seq * n_q_heads + head].  scores (float) and sel_out
+ * (int32) are device arrays [batch * n_q_heads][n_max], count_out int32 [batch * n_q_heads]; q and k_cache as for
+ * bpc_decode_attn.  An evaluation aid: it reads every key row.  The other yard-stick, dense attention over all cached
+ * keys, is bpc_decode_attn with budget_ppm = 1000000. */
+bpc_status bpc_exact_topk(bpc_ctx* ctx, const void* q, const void* k_cache, int32_t budget_ppm, int32_t budget_count,
+                          float* scores, int32_t* sel_out, int32_t* count_out, void* stream);
+
 /* Parity aids.  When set (non-NULL), the next bpc_decode_attn calls also write the integer hash
  * score of every cached key (scores [units][n_max] int32) and the collapsed integer query weights
  * A = sum over the group's heads of sign*magnitude (qweights [units][code_bits] int32). */

@@ -58,6 +58,7 @@ def _load() -> ctypes.CDLL:
         "bpc_build_eas": (i32, [vp, vp]),
         "bpc_get_eas": (i32, [vp, vp, vp, vp, vp]),
         "bpc_eas_capacity": (i32, [cfgp]),
+        "bpc_exact_topk": (i32, [vp, vp, vp, i32, i32, vp, vp, vp, vp]),
         "bpc_append": (i32, [vp, vp, vp, vp, vp, vp, vp]),
         "bpc_decode_attn": (i32, [vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]),
         "bpc_append_decode_attn": (i32, [vp, vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]),
@@ -83,7 +84,7 @@ lib = _load()
 EXPORTS = ["bpc_create", "bpc_destroy", "bpc_codes_bytes", "bpc_fit_workspace_bytes", "bpc_fit_codes_offset",
            "bpc_max_context",
            "bpc_set_seq_lens", "bpc_get_seq_lens", "bpc_fit", "bpc_set_projection", "bpc_get_projection",
-           "bpc_encode_keys", "bpc_build_eas", "bpc_get_eas", "bpc_eas_capacity", "bpc_append", "bpc_decode_attn", "bpc_append_decode_attn", "bpc_decode_attn_static", "bpc_static_scratch_entries",
+           "bpc_encode_keys", "bpc_build_eas", "bpc_get_eas", "bpc_eas_capacity", "bpc_exact_topk", "bpc_append", "bpc_decode_attn", "bpc_append_decode_attn", "bpc_decode_attn_static", "bpc_static_scratch_entries",
            "bpc_debug_set_buffers", "bpc_debug_set_phase_timer",
            "bpc_set_cluster_size",
            "bpc_get_cluster_size", "bpc_last_device_error", "bpc_last_cuda_error", "bpc_launch_count", "bpc_version"]
@@ -205,6 +206,18 @@ class Context:
 
     def build_eas(self) -> None:
         _check(lib.bpc_build_eas(self._h, _stream()), "bpc_build_eas")
+
+    def exact_topk(self, q, k_cache, budget_ppm: int = 20000, budget_count: int = 0):
+        """Quality yard-stick: exact scores of every cached key for every query head and the per-head top-k.
+        Returns (scores [batch*n_q_heads, n_max] float32, sel [batch*n_q_heads, n_max] int32, count [batch*n_q_heads] int32)."""
+        c = self.cfg
+        heads = c.batch * c.n_q_heads
+        scores = torch.zeros(heads, c.n_max, dtype=torch.float32, device=q.device)
+        sel = torch.full((heads, c.n_max), -1, dtype=torch.int32, device=q.device)
+        cnt = torch.zeros(heads, dtype=torch.int32, device=q.device)
+        _check(lib.bpc_exact_topk(self._h, _ptr(q), _cache_ptr(k_cache), budget_ppm, budget_count, _ptr(scores), _ptr(sel),
+                                  _ptr(cnt), _stream()), "bpc_exact_topk")
+        return scores, sel, cnt
 
     def get_eas(self):
         c = self.cfg

@@ -308,6 +308,16 @@ bpc_status bpc_build_eas(bpc_ctx* ctx, void* stream) {
   return e == cudaSuccess ? BPC_OK : cuda_fail(ctx, e);
 }
 
+bpc_status bpc_exact_topk(bpc_ctx* ctx, const void* q, const void* k_cache, int32_t budget_ppm, int32_t budget_count,
+                          float* scores, int32_t* sel_out, int32_t* count_out, void* stream) {
+  if (ctx == nullptr || q == nullptr || k_cache == nullptr || scores == nullptr || sel_out == nullptr || count_out == nullptr)
+    return BPC_ERR_INVALID_ARG;
+  if (budget_count < 0 || (budget_count == 0 && (budget_ppm < 0 || budget_ppm > 1000000))) return BPC_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k_cache)) & 15u) return BPC_ERR_INVALID_ARG;
+  cudaError_t e = bpc_launch_exact_topk(ctx, q, k_cache, budget_ppm, budget_count, scores, sel_out, count_out, (cudaStream_t)stream);
+  return e == cudaSuccess ? BPC_OK : cuda_fail(ctx, e);
+}
+
 bpc_status bpc_get_eas(bpc_ctx* ctx, float* sq_err_out, int32_t* set_out, int32_t* count_out, void* stream) {
   if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
   if (ctx->cfg.eas_ppm <= 0) return BPC_ERR_UNSUPPORTED;

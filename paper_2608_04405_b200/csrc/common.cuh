@@ -111,6 +111,8 @@ size_t bpc_fit_codes_offset_impl(const bpc_config* cfg);
 
 // ---- error-aware safeguard set construction (prefill.cu)
 cudaError_t bpc_launch_build_eas(bpc_ctx* ctx, cudaStream_t stream);
+cudaError_t bpc_launch_exact_topk(bpc_ctx* ctx, const void* q, const void* k_cache, int budget_ppm, int budget_count,
+                                  float* scores, int32_t* sel, int32_t* sel_cnt, cudaStream_t stream);
 
 // ---- tensor-core encode (encode_tc.cu); returns cudaErrorNotSupported when the shape is not covered
 cudaError_t bpc_launch_encode_tc(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStream_t stream);

@@ -306,3 +306,50 @@ def check_append(sess: Session, k_new: torch.Tensor, v_new: torch.Tensor, units,
         n = n1 - 1
         assert torch.equal(sess.k_cache[bi, h, n], k_new[bi, h]) and torch.equal(sess.v_cache[bi, h, n], v_new[bi, h])
         check_encode(sess, [u], report, key_slice=(n, n + 1))
+
+
+def check_yardsticks(sess: Session, q: torch.Tensor, units, report: dict, budget_ppm=None):
+    """Quality yard-sticks through the library: bpc_exact_topk (per-head exact scores and top-k) and dense attention
+    (the decode call with a budget of all keys), against the checker; then recall of the hash selection with respect to
+    the exact top-k and the cosine similarity of sparse and dense outputs, computed on both sides."""
+    s = sess.spec
+    ppm = s.budget_ppm if budget_ppm is None else budget_ppm
+    G = s.group
+    scores, sel, cnt = sess.ctx.exact_topk(q, sess.k_cache, budget_ppm=ppm)
+    dense = sess.ctx.decode_attn(q, sess.k_cache, sess.v_cache, sess.codes, budget_ppm=1000000)
+    hsel = torch.full((sess.units, sess.w.n_max), -1, dtype=torch.int32, device="cuda")
+    sparse = sess.ctx.decode_attn(q, sess.k_cache, sess.v_cache, sess.codes, budget_ppm=ppm, sel_idx=hsel)
+    torch.cuda.synchronize()
+    tol_out = 2e-3 if s.dtype == "bf16" else 1e-5
+    rec_gpu, rec_ref, cos_all = [], [], []
+    for u in units:
+        bi, h, n = sess.unit_views(u)
+        K = _np64(sess.k_cache[bi, h, :n]); V = _np64(sess.v_cache[bi, h, :n])
+        qg = _np64(q[bi, h * G:(h + 1) * G])
+        k = O.budget(n, ppm)
+        hash_idx = hsel[u, :k].cpu().numpy().astype(np.int64)
+        d_ref = O.dense_attend(qg, K, V)
+        d_gpu = _np64(dense[bi, h * G:(h + 1) * G])
+        assert np.abs(d_gpu - d_ref).max() <= tol_out * max(1.0, np.abs(d_ref).max()), "dense attention differs"
+        s_gpu = _np64(sparse[bi, h * G:(h + 1) * G])
+        for g in range(G):
+            head = bi * s.n_q_heads + h * G + g
+            sc64 = K @ qg[g]
+            got_sc = _np64(scores[head, :n])
+            assert np.abs(got_sc - sc64).max() <= 2e-5 * np.linalg.norm(qg[g]) * np.linalg.norm(K, axis=1).max(), "exact scores differ"
+            assert int(cnt[head]) == k
+            got = sel[head, :k].cpu().numpy().astype(np.int64)
+            assert np.all(np.diff(got) > 0), "exact top-k list is not ascending"
+            ref = O.exact_topk(qg[g], K, k)
+            # keys on which the two selections disagree must sit at the k-th score within fp32 rounding
+            kth = np.sort(sc64)[n - k]
+            band = 4e-5 * np.linalg.norm(qg[g]) * np.linalg.norm(K, axis=1).max()
+            diff = np.setxor1d(got, ref)
+            assert np.all(np.abs(sc64[diff] - kth) <= band), "exact top-k differs outside the rounding band"
+            rec_gpu.append(O.selection_recall(hash_idx, got)); rec_ref.append(O.selection_recall(hash_idx, ref))
+            cos_all.append(O.cosine_similarity(s_gpu[g], d_gpu[g]))
+            cref = O.cosine_similarity(O.attend(qg[g:g + 1], K, V, hash_idx)[0], d_ref[g])
+            assert abs(cos_all[-1] - cref) <= 5e-3, "cosine of sparse vs dense output differs (%g vs %g)" % (cos_all[-1], cref)
+        assert abs(np.mean(rec_gpu[-G:]) - np.mean(rec_ref[-G:])) <= 2.0 / max(k, 1)
+    report["recall_vs_exact_topk"] = float(np.mean(rec_gpu))
+    report["cosine_sparse_vs_dense"] = float(np.mean(cos_all))

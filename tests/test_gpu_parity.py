@@ -364,6 +364,22 @@ def test_fit_with_power_iterations(dtype, bits, n, power):
     print(rep)
 
 
+@pytest.mark.parametrize("dtype,bits,group,n", [("bf16", 128, 4, 9000), ("f32", 64, 2, 5000), ("bf16", 256, 8, 6000)])
+def test_quality_yardsticks(dtype, bits, group, n):
+    """The TOPK (Oracle) selector and dense attention (appendix "Baseline Methods"; cosine-similarity table), and the two
+    numbers built on them: recall of the hash selection against the exact top-k, cosine of sparse against dense output."""
+    H = _harness()
+    spec = CONFIGS[1].scaled(name="yard", wid=80 + group, batch=2, n_kv_heads=2, n_q_heads=2 * group, n_ctx=n, dtype=dtype,
+                             code_bits=bits, steps=1)
+    sess = H.Session(spec, gen_device="cuda")
+    rep = {}
+    sess.fit(); sess.encode()
+    q, _ = sess.w.queries(sess.lens)
+    H.check_yardsticks(sess, q.cuda(), [0, 3], rep)
+    H.check_yardsticks(sess, q.cuda(), [1], rep, budget_ppm=100000)
+    print(rep)
+
+
 @pytest.mark.parametrize("n_ctx,batch", [(262144, 1), (32768, 16)])
 def test_sweep_shapes_single_word_codes_fixed_budgets(n_ctx, batch):
     """The second bench workload's shapes (Section 4 "Setup" / latency-vs-context study: 64-bit codes, budgets of 1024
