@@ -42,6 +42,7 @@ bpc_status check_cfg(const bpc_config* c) {
   if (c->eas_ppm > 0 && (c->residual_correction == 0 || c->score_mode != BPC_SCORE_HAMMING)) return BPC_ERR_UNSUPPORTED;
   if (c->eas_ppm > 0 && ((long long)c->n_max * c->eas_ppm + 999999) / 1000000 > 16384) return BPC_ERR_UNSUPPORTED;
   if (c->n_max % 2 != 0) return BPC_ERR_INVALID_ARG;   // keeps every unit's code rows 16-byte aligned at 64 bits
+  if (c->n_max > (1 << 26)) return BPC_ERR_UNSUPPORTED; // far above what a cluster's shared memory holds; keeps index math in 32 bits
   return BPC_OK;
 }
 

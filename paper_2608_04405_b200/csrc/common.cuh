@@ -18,7 +18,9 @@
 // Algorithm 2's sign sweep); it is given (16 - BPC_APPEND_LOSS16)/16 of the other blocks' key share.
 #define BPC_APPEND_LOSS16 2
 __host__ __device__ inline int bpc_fused_chunk(int n, int cs) {
-  return ((int)(((long long)n * 16 + 16 * cs - BPC_APPEND_LOSS16 - 1) / (16 * cs - BPC_APPEND_LOSS16)) + 63) & ~63;
+  // n <= 2^26 (bpc_create rejects larger n_max), so 32-bit arithmetic is exact here; a 64-bit division by a run-time
+  // divisor would cost every thread of the kernel some hundred instructions
+  return ((int)(((unsigned)n * 16u + 16u * (unsigned)cs - (unsigned)BPC_APPEND_LOSS16 - 1u) / (16u * (unsigned)cs - (unsigned)BPC_APPEND_LOSS16)) + 63) & ~63;
 }
 
 struct bpc_ctx {

@@ -82,8 +82,8 @@ struct DecodeSmem {
     off_qf = off_tot + nb;                                           // float[GP+1][128]
     off_pd = off_qf + (size_t)GV * BPC_D * 4;                        // double[GP+1][B]
     off_idx = off_pd + (size_t)GV * B * 8;                           // int32[kIdxTile]
-    off_cta = off_idx + kIdxTile * 4;                                // acc_t[GP][130]
-    off_small = a16(off_cta + (size_t)GP * (BPC_D + 2) * sizeof(acc_t));
+    off_cta = off_idx + kIdxTile * 4;                                // merge inbox: acc_t[GP * (128 + 2 * 16) + 16]
+    off_small = a16(off_cta + ((size_t)GP * (BPC_D + 2 * BPC_MAX_CLUSTER) + BPC_MAX_CLUSTER) * sizeof(acc_t));
     off_union = a16(off_small + sizeof(SmallState));
     size_t u = (size_t)((chunk_cap + kSegKeys - 1) / kSegKeys) * kSegSlots * 2;   // score keys
     if (u < part_bytes()) u = part_bytes();                                      // block-level merge
@@ -348,9 +348,9 @@ bpc_decode_kernel(const DecodeParams p) {
   float* qf_s = reinterpret_cast<float*>(smem + plan.off_qf);
   double* pd = reinterpret_cast<double*>(smem + plan.off_pd);
   int32_t* idx_s = reinterpret_cast<int32_t*>(smem + plan.off_idx);
-  acc_t* cta_acc = reinterpret_cast<acc_t*>(smem + plan.off_cta);      // [GP][128], then m[GP], l[GP]
-  acc_t* cta_m = cta_acc + GP * BPC_D;
-  acc_t* cta_l = cta_m + GP;
+  // Inbox of the cluster-level merge: row r holds block r's partial sums for the outputs this block owns, then its
+  // running maxima and denominators of all heads (peers store them here before the last cluster barrier).
+  acc_t* inbox = reinterpret_cast<acc_t*>(smem + plan.off_cta);
   SmallState* st = reinterpret_cast<SmallState*>(smem + plan.off_small);
   unsigned char* uni = smem + plan.off_union;
   uint16_t* sc = reinterpret_cast<uint16_t*>(uni);
@@ -999,7 +999,7 @@ bpc_decode_kernel(const DecodeParams p) {
     }
   }
   // this block attends rows [lo, hi) of the hash list and the safeguard keys that lie in its own key range
-  const int lo = (int)(((long long)kh * rank) / CS), hi = (int)(((long long)kh * (rank + 1)) / CS);
+  const int lo = (int)(((unsigned)kh * (unsigned)rank) / (unsigned)CS), hi = (int)(((unsigned)kh * (unsigned)(rank + 1)) / (unsigned)CS);   // kh * 16 < 2^31
   const int nh = hi - lo, ne = e1 - e0;                      // rows from the two sources
   if (me > 0) {
     __syncthreads();                                         // the selection masks of this block are written
@@ -1277,6 +1277,11 @@ bpc_decode_kernel(const DecodeParams p) {
   }
   BPC_STAMP(5);
   __syncthreads();
+  // Block-level merge of the warps' partials; every result goes straight to the block of the cluster that owns that
+  // output (outputs are split evenly over the ranks), its maximum and denominator to every block.
+  const int nout = G * BPC_D;
+  const int per = (nout + CS - 1) / CS;                      // outputs owned by one rank
+  const int istride = per + 2 * GP;                          // one inbox row
   for (int o = tid; o < GP * BPC_D; o += NT) {
     const int g = o >> 7, d = o & 127;
     acc_t mm = (acc_t)-1e30;
@@ -1291,32 +1296,41 @@ bpc_decode_kernel(const DecodeParams p) {
       num = fma(src[d], wt, num);
       den = fma(src[BPC_D + 1], wt, den);
     }
-    cta_acc[o] = num;
-    if (d == 0) { cta_m[g] = mm; cta_l[g] = den; }
+    if (o < nout) {
+      const int owner = o / per;
+      cluster.map_shared_rank(inbox, owner)[rank * istride + (o - owner * per)] = num;
+    }
+    if (d == 0 && g < G) {
+#pragma unroll 1
+      for (int r = 0; r < CS; ++r) {
+        acc_t* row = cluster.map_shared_rank(inbox, r) + rank * istride + per;
+        row[g] = mm;
+        row[GP + g] = den;
+      }
+    }
   }
   BPC_STAMP(6);
-  cluster.sync();                                            // every block's partial result is published
+  cluster.sync();                                            // every block's partial results have been delivered
   {
-    const int nout = G * BPC_D;
-    const int per = (nout + CS - 1) / CS;
+    // cluster-level merge of the outputs this block owns, from its own shared memory; nothing remote is read after
+    // the barrier, so a block may exit as soon as it has written its outputs
     const int o_end = min(nout, (rank + 1) * per);
     for (int o = rank * per + tid; o < o_end; o += NT) {
-      const int g = o >> 7;
+      const int g = o >> 7, j = o - rank * per;
       acc_t mm = (acc_t)-1e30;
       for (int r = 0; r < CS; ++r) {
-        const acc_t v = cluster.map_shared_rank(cta_m, r)[g];
+        const acc_t v = inbox[r * istride + per + g];
         mm = v > mm ? v : mm;
       }
       acc_t num = 0, den = 0;
       for (int r = 0; r < CS; ++r) {
-        const acc_t wt = fast_exp2<acc_t>(cluster.map_shared_rank(cta_m, r)[g] - mm);
-        num = fma(cluster.map_shared_rank(cta_acc, r)[o], wt, num);
-        den = fma(cluster.map_shared_rank(cta_l, r)[g], wt, den);
+        const acc_t wt = fast_exp2<acc_t>(inbox[r * istride + per + g] - mm);
+        num = fma(inbox[r * istride + j], wt, num);
+        den = fma(inbox[r * istride + per + GP + g], wt, den);
       }
       out_u[o] = (float)(num / den);
     }
   }
-  cluster.sync();                                            // keep shared memory alive until all peers have read it
   BPC_STAMP(14);
   if (p.dbg_times != nullptr && tid == 0) p.dbg_times[(size_t)blockIdx.x * 16 + 7] = global_timer_ns();
 #undef BPC_STAMP
