@@ -215,60 +215,148 @@ append_kernel(const KV* __restrict__ k_new, const KV* __restrict__ v_new, KV* __
 }
 
 // --------------------------------------------------------------------------- Algorithm 1 (fit)
-// The residual R (fp32) lives in the workspace.  Iteration i is one pass over R:
-//   R_row -= u_{i-1}(row) * v_{i-1}   (skipped at i = 0, where R_row = K_row)
-//   t = R_row . v*_i ; u_i(row) = sign(t) ; partial[c] += u_i(row) * R_row[c]
-// followed by a small deterministic reduction v_i = sum(partials) / N.  One warp handles one row at a
-// time (4 channels per lane, coalesced 512-byte rows).
+// The residual is never stored.  With the signs u_j of the earlier bits kept as packed code words (the codes H that
+// Algorithm 1 itself produces) and P_j = v_j, a row's residual is R_row = K_row - sum_j u_j v_j, hence
+//   t = R_row . d        = K_row . d - sum_{j<i} u_j (v_j . d)          (d = the direction of bit i)
+//   u_i R = u_i K - sum_{j<i} (u_i . u_j) v_j                            (u_i . u_j = 2 * agreements - N, an integer)
+// Iteration i therefore reads the key row and its code words (272 bytes per row instead of 1 KB of fp32 residual read and
+// written back), writes one bit, and leaves per block a partial sum of +-K rows and the per-bit agreement counts; a
+// small kernel before the pass prepares d and the b inner products v_j . d, a small one after it forms v_i.
 constexpr int kFitThreads = 256;
 constexpr int kFitRowsPerBlock = 1024;
 
-template <typename KV>
+// before the pass of bit `it`: dir[unit] = direction (the caller's draw, unless the power-iteration kernel already
+// wrote one), dots[unit][j] = v_j . dir for j < it and 0 for the other bits
+__global__ void __launch_bounds__(BPC_D)
+fit_prep_kernel(const float* __restrict__ P, const float* __restrict__ v_star, float* __restrict__ dir, float* __restrict__ dots,
+                int b, int it, int have_dir) {
+  const int unit = blockIdx.x, tid = threadIdx.x;
+  __shared__ float d_s[BPC_D];
+  float dv = have_dir ? dir[(size_t)unit * BPC_D + tid] : v_star[((size_t)unit * b + it) * BPC_D + tid];
+  d_s[tid] = dv;
+  if (!have_dir) dir[(size_t)unit * BPC_D + tid] = dv;
+  __syncthreads();
+  for (int j = tid; j < b; j += BPC_D) {
+    double acc = 0.0;
+    if (j < it) {
+      const float* pj = P + ((size_t)unit * b + j) * BPC_D;
+      for (int c = 0; c < BPC_D; ++c) acc += (double)pj[c] * (double)d_s[c];
+    }
+    dots[(size_t)unit * b + j] = (float)acc;
+  }
+}
+
+// Eight lanes share a row (16 channels and b/8 earlier bits each), so a warp works on four rows at once.
+template <typename KV, int JPL>          // JPL = b / 8 bits per lane
 __global__ void __launch_bounds__(kFitThreads)
-fit_pass_kernel(const KV* __restrict__ k_cache, float* __restrict__ R, uint8_t* __restrict__ usign,
-                uint32_t* __restrict__ hfit, const float* __restrict__ v_star, const float* __restrict__ P, float* __restrict__ partials,
-                const int32_t* __restrict__ unit_lens, int n_max, int row_stride, int b, int it, int blocks_per_unit,
-                const float* __restrict__ dir) {
+fit_pass_kernel(const KV* __restrict__ k_cache, uint32_t* __restrict__ hfit, const float* __restrict__ dir,
+                const float* __restrict__ dots, float* __restrict__ partials, int32_t* __restrict__ agree,
+                const int32_t* __restrict__ unit_lens, int n_max, int row_stride, int it, int blocks_per_unit) {
+  constexpr int b = JPL * 8, WORDS = b / 32;
+  constexpr int CPLN = 16;                                    // channels per lane
   const int unit = blockIdx.y;
   const int n = min(unit_lens[unit], n_max);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int sub = lane & 7, grp = lane >> 3;                  // lane within the row's group, row within the warp's four
   const int row0 = blockIdx.x * kFitRowsPerBlock;
   __shared__ float red[kFitThreads / 32][BPC_D];
-  // direction of the projection: the caller's draw v*_i, or (power-iteration fit) (R^T R)^n v*_i prepared per unit
-  const float4 vs = dir != nullptr ? reinterpret_cast<const float4*>(dir + (size_t)unit * BPC_D)[lane]
-                                   : reinterpret_cast<const float4*>(v_star + ((size_t)unit * b + it) * BPC_D)[lane];
-  float4 vp = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (it > 0) vp = reinterpret_cast<const float4*>(P + ((size_t)unit * b + (it - 1)) * BPC_D)[lane];
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  const int row_end = min(n, row0 + kFitRowsPerBlock);
-  for (int r = row0 + warp; r < row_end; r += kFitThreads / 32) {
-    const size_t ro = ((size_t)unit * n_max + r) * BPC_D;
-    float4 x;
-    if (it == 0) {
-      const KV* kr = k_cache + ((size_t)unit * n_max + r) * row_stride + 4 * lane;
-      x = make_float4(to_float(kr[0]), to_float(kr[1]), to_float(kr[2]), to_float(kr[3]));
-    } else {
-      x = reinterpret_cast<const float4*>(R + ro)[lane];
-      const float u = usign[(size_t)unit * n_max + r] ? 1.f : -1.f;
-      x.x = fmaf(-u, vp.x, x.x); x.y = fmaf(-u, vp.y, x.y); x.z = fmaf(-u, vp.z, x.z); x.w = fmaf(-u, vp.w, x.w);
-    }
-    reinterpret_cast<float4*>(R + ro)[lane] = x;
-    float t = x.x * vs.x;
-    t = fmaf(x.y, vs.y, t); t = fmaf(x.z, vs.z, t); t = fmaf(x.w, vs.w, t);
+  __shared__ int32_t redc[kFitThreads / 32][b];
+  float dv[CPLN];
 #pragma unroll
-    for (int o = 16; o >= 1; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-    const bool pos = t >= 0.f;
-    if (lane == 0) {
-      usign[(size_t)unit * n_max + r] = pos ? 1 : 0;
-      // diagnostic copy of the fitted codes H (Algorithm 1's by-product), packed like the cache codes
-      uint32_t* hw = hfit + ((size_t)unit * n_max + r) * (b / 32) + (it >> 5);
-      const uint32_t prev = (it & 31) ? *hw : 0u;
-      *hw = prev | ((pos ? 1u : 0u) << (it & 31));
+  for (int c = 0; c < CPLN; ++c) dv[c] = dir[(size_t)unit * BPC_D + sub * CPLN + c];
+  // sum_j u_j (v_j . d) over a lane's bits is looked up four bits at a time: lut[sub][nibble][pattern] = sum over the
+  // nibble's bits of +-(v_j . d) (the inner products of bits >= it are zero, so later bits add nothing)
+  constexpr int NIB = JPL / 4;
+  __shared__ float lut[8][NIB][16];
+  for (int e = tid; e < 8 * NIB * 16; e += kFitThreads) {
+    const int m = e & 15, nb = (e >> 4) % NIB, sb = e / (16 * NIB);
+    float v = 0.f;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float d = dots[(size_t)unit * b + sb * JPL + 4 * nb + q];
+      v += ((m >> q) & 1) ? d : -d;
     }
-    if (pos) { acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w; }
-    else     { acc.x -= x.x; acc.y -= x.y; acc.z -= x.z; acc.w -= x.w; }
+    lut[sb][nb][m] = v;
   }
-  red[warp][4 * lane] = acc.x; red[warp][4 * lane + 1] = acc.y; red[warp][4 * lane + 2] = acc.z; red[warp][4 * lane + 3] = acc.w;
+  __syncthreads();
+  const int my_word = (sub * JPL) >> 5, my_shift = (sub * JPL) & 31;
+  float acc[CPLN];
+#pragma unroll
+  for (int c = 0; c < CPLN; ++c) acc[c] = 0.f;
+  // agreements with the earlier bits are counted in six bit-sliced counter planes (at most 32 rows per lane group)
+  uint32_t pl[6] = {0u, 0u, 0u, 0u, 0u, 0u};
+  const int row_end = min(n, row0 + kFitRowsPerBlock);
+  constexpr int ROWS_PER_ITER = (kFitThreads / 32) * 4;
+  for (int rb = row0; rb < row_end; rb += ROWS_PER_ITER) {   // uniform trip count: the shuffles below need whole warps
+    const int r = rb + warp * 4 + grp;
+    const bool live = r < row_end;
+    const int rr = live ? r : row0;
+    const KV* kr = k_cache + ((size_t)unit * n_max + rr) * row_stride + sub * CPLN;
+    float x[CPLN];
+    if (sizeof(KV) == 2) {
+      const uint4 w0 = reinterpret_cast<const uint4*>(kr)[0], w1 = reinterpret_cast<const uint4*>(kr)[1];
+      const uint32_t ww[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+      for (int c = 0; c < 8; ++c) { x[2 * c] = __uint_as_float(ww[c] << 16); x[2 * c + 1] = __uint_as_float(ww[c] & 0xffff0000u); }
+    } else {
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {
+        const float4 f = reinterpret_cast<const float4*>(kr)[v];
+        x[4 * v] = f.x; x[4 * v + 1] = f.y; x[4 * v + 2] = f.z; x[4 * v + 3] = f.w;
+      }
+    }
+    uint32_t* hw = hfit + ((size_t)unit * n_max + rr) * WORDS;
+    const uint32_t mine = it > 0 ? (hw[my_word] >> my_shift) : 0u;                     // this lane's JPL earlier bits
+    float tk = 0.f;
+#pragma unroll
+    for (int c = 0; c < CPLN; ++c) tk = fmaf(x[c], dv[c], tk);
+    float tc = 0.f;
+#pragma unroll
+    for (int nb = 0; nb < NIB; ++nb) tc += lut[sub][nb][(mine >> (4 * nb)) & 15u];
+    double t = (double)tk - (double)tc;
+#pragma unroll
+    for (int o = 4; o >= 1; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    const bool pos = t >= 0.0;
+    if (live) {
+      if (sub == 0) {
+        uint32_t* w = hw + (it >> 5);
+        const uint32_t prev = (it & 31) ? *w : 0u;
+        *w = prev | ((pos ? 1u : 0u) << (it & 31));
+      }
+      const float sg = pos ? 1.f : -1.f;
+#pragma unroll
+      for (int c = 0; c < CPLN; ++c) acc[c] = fmaf(sg, x[c], acc[c]);
+      uint32_t carry = pos ? mine : ~mine;                                              // bit e: u_j agrees with u_i
+#pragma unroll
+      for (int k = 0; k < 6; ++k) {
+        const uint32_t nc = pl[k] & carry;
+        pl[k] ^= carry;
+        carry = nc;
+      }
+    }
+  }
+  // the four row groups of a warp hold partial sums for the same channels and bits
+#pragma unroll
+  for (int c = 0; c < CPLN; ++c) {
+    acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], 8);
+    acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], 16);
+  }
+  int cnt[JPL];
+#pragma unroll
+  for (int e = 0; e < JPL; ++e) {
+    int c = 0;
+#pragma unroll
+    for (int k = 0; k < 6; ++k) c += (int)((pl[k] >> e) & 1u) << k;
+    c += __shfl_xor_sync(0xffffffffu, c, 8);
+    c += __shfl_xor_sync(0xffffffffu, c, 16);
+    cnt[e] = c;
+  }
+  if (grp == 0) {
+#pragma unroll
+    for (int c = 0; c < CPLN; ++c) red[warp][sub * CPLN + c] = acc[c];
+#pragma unroll
+    for (int e = 0; e < JPL; ++e) redc[warp][sub * JPL + e] = cnt[e];
+  }
   __syncthreads();
   if (tid < BPC_D) {
     float s = 0.f;
@@ -276,16 +364,42 @@ fit_pass_kernel(const KV* __restrict__ k_cache, float* __restrict__ R, uint8_t* 
     for (int w = 0; w < kFitThreads / 32; ++w) s += red[w][tid];
     partials[((size_t)unit * blocks_per_unit + blockIdx.x) * BPC_D + tid] = s;
   }
+  for (int j = tid; j < b; j += kFitThreads) {
+    int c = 0;
+#pragma unroll
+    for (int w = 0; w < kFitThreads / 32; ++w) c += redc[w][j];
+    agree[((size_t)unit * blocks_per_unit + blockIdx.x) * b + j] = c;
+  }
 }
 
-__global__ void fit_reduce_kernel(const float* __restrict__ partials, float* __restrict__ P,
-                                  const int32_t* __restrict__ unit_lens, int n_max, int b, int it, int blocks_per_unit) {
-  const int unit = blockIdx.x, c = threadIdx.x;
+// v_i = (sum of the blocks' +-K partial sums - sum_{j<i} (2 * agreements_j - N) v_j) / N.  Four thread groups split
+// the blocks and the earlier bits; every sum is formed in a fixed order (group partials added 0..3).
+constexpr int kRedGroups = 4;
+__global__ void __launch_bounds__(BPC_D * kRedGroups)
+fit_reduce_kernel(const float* __restrict__ partials, const int32_t* __restrict__ agree, float* __restrict__ P,
+                  const int32_t* __restrict__ unit_lens, int n_max, int b, int it, int blocks_per_unit) {
+  const int unit = blockIdx.x, c = threadIdx.x & (BPC_D - 1), q = threadIdx.x / BPC_D;
   const int n = min(unit_lens[unit], n_max);
   const int nblk = (n + kFitRowsPerBlock - 1) / kFitRowsPerBlock;
+  __shared__ double corr[256];                               // u_i . u_j for j < it
+  __shared__ double part[kRedGroups][BPC_D];
+  for (int j = threadIdx.x; j < it; j += BPC_D * kRedGroups) {
+    long long a = 0;
+    for (int k = 0; k < nblk; ++k) a += agree[((size_t)unit * blocks_per_unit + k) * b + j];
+    corr[j] = (double)(2 * a - (long long)n);
+  }
+  __syncthreads();
   double s = 0.0;
-  for (int k = 0; k < nblk; ++k) s += (double)partials[((size_t)unit * blocks_per_unit + k) * BPC_D + c];
-  P[((size_t)unit * b + it) * BPC_D + c] = n > 0 ? (float)(s / (double)n) : 0.f;
+  for (int k = q; k < nblk; k += kRedGroups) s += (double)partials[((size_t)unit * blocks_per_unit + k) * BPC_D + c];
+  for (int j = q; j < it; j += kRedGroups) s -= corr[j] * (double)P[((size_t)unit * b + j) * BPC_D + c];
+  part[q][c] = s;
+  __syncthreads();
+  if (q == 0) {
+    double t = 0.0;
+#pragma unroll
+    for (int g = 0; g < kRedGroups; ++g) t += part[g][c];
+    P[((size_t)unit * b + it) * BPC_D + c] = n > 0 ? (float)(t / (double)n) : 0.f;
+  }
 }
 
 // --------------------------------------------------------------------------- power-iteration fit
@@ -532,18 +646,30 @@ static size_t fit_power_bytes(const bpc_config* c) {
   return align256(units * BPC_D * BPC_D * 8) + align256(units * slabs * BPC_D * BPC_D * 8) + align256(units * BPC_D * 4);
 }
 
-size_t bpc_fit_workspace_bytes_impl(const bpc_config* c) {
+// workspace layout: fitted codes H | per-block partial sums | per-block agreement counts | direction | inner products
+// | (power-iteration fit) C, its slab partial sums
+static size_t fit_off_partials(const bpc_config* c) {
+  const size_t units = (size_t)c->batch * c->n_kv_heads;
+  return align256(units * c->n_max * (c->code_bits / 8));
+}
+static size_t fit_off_agree(const bpc_config* c) {
   const size_t units = (size_t)c->batch * c->n_kv_heads;
   const size_t bpu = ((size_t)c->n_max + kFitRowsPerBlock - 1) / kFitRowsPerBlock;
-  return align256(units * c->n_max * BPC_D * 4) + align256(units * c->n_max) + align256(units * bpu * BPC_D * 4) +
-         align256(units * c->n_max * (c->code_bits / 8)) + fit_power_bytes(c);
+  return fit_off_partials(c) + align256(units * bpu * BPC_D * 4);
+}
+static size_t fit_off_dir(const bpc_config* c) {
+  const size_t units = (size_t)c->batch * c->n_kv_heads;
+  const size_t bpu = ((size_t)c->n_max + kFitRowsPerBlock - 1) / kFitRowsPerBlock;
+  return fit_off_agree(c) + align256(units * bpu * c->code_bits * 4);
+}
+static size_t fit_off_power(const bpc_config* c) {
+  const size_t units = (size_t)c->batch * c->n_kv_heads;
+  return fit_off_dir(c) + align256(units * BPC_D * 4) + align256(units * c->code_bits * 4);
 }
 
-size_t bpc_fit_codes_offset_impl(const bpc_config* c) {
-  const size_t units = (size_t)c->batch * c->n_kv_heads;
-  const size_t bpu = ((size_t)c->n_max + kFitRowsPerBlock - 1) / kFitRowsPerBlock;
-  return align256(units * c->n_max * BPC_D * 4) + align256(units * c->n_max) + align256(units * bpu * BPC_D * 4);
-}
+size_t bpc_fit_workspace_bytes_impl(const bpc_config* c) { return fit_off_power(c) + fit_power_bytes(c); }
+
+size_t bpc_fit_codes_offset_impl(const bpc_config* c) { (void)c; return 0; }
 
 cudaError_t bpc_launch_fit(bpc_ctx* ctx, const void* k_cache, const float* v_star, void* workspace,
                            cudaStream_t stream, int* launches) {
@@ -551,20 +677,19 @@ cudaError_t bpc_launch_fit(bpc_ctx* ctx, const void* k_cache, const float* v_sta
   const size_t units = (size_t)ctx->units;
   const int bpu = (c.n_max + kFitRowsPerBlock - 1) / kFitRowsPerBlock;
   unsigned char* ws = (unsigned char*)workspace;
-  float* R = (float*)ws;
-  uint8_t* usign = ws + align256(units * c.n_max * BPC_D * 4);
-  float* partials = (float*)(usign + align256(units * c.n_max));
-  uint32_t* hfit = (uint32_t*)(ws + bpc_fit_codes_offset_impl(&c));
+  uint32_t* hfit = (uint32_t*)ws;
+  float* partials = (float*)(ws + fit_off_partials(&c));
+  int32_t* agree = (int32_t*)(ws + fit_off_agree(&c));
+  float* dir = (float*)(ws + fit_off_dir(&c));
+  float* dots = (float*)(ws + fit_off_dir(&c) + align256(units * BPC_D * 4));
   const dim3 grid(bpu, ctx->units);
   const int npow = c.fit_power_iters;
   double* Cm = nullptr;
-  float* dir = nullptr;
   if (npow > 0) {
     const int slabs = (c.n_max + kGramRows - 1) / kGramRows;
-    unsigned char* pw = (unsigned char*)hfit + align256(units * c.n_max * (c.code_bits / 8));
+    unsigned char* pw = ws + fit_off_power(&c);
     Cm = (double*)pw;
     double* cpart = (double*)(pw + align256(units * BPC_D * BPC_D * 8));
-    dir = (float*)(pw + align256(units * BPC_D * BPC_D * 8) + align256(units * (size_t)slabs * BPC_D * BPC_D * 8));
     const dim3 g0(slabs, ctx->units);
     if (c.kv_dtype == BPC_BF16)
       fit_gram0_kernel<__nv_bfloat16><<<g0, 256, 0, stream>>>((const __nv_bfloat16*)k_cache, cpart, ctx->unit_lens, c.n_max, ctx->row_stride, slabs);
@@ -578,14 +703,18 @@ cudaError_t bpc_launch_fit(bpc_ctx* ctx, const void* k_cache, const float* v_sta
       fit_direction_kernel<<<ctx->units, BPC_D, 0, stream>>>(Cm, ctx->P, v_star, dir, ctx->unit_lens, c.n_max, c.code_bits, it, npow);
       *launches += 1;
     }
-    if (c.kv_dtype == BPC_BF16)
-      fit_pass_kernel<__nv_bfloat16><<<grid, kFitThreads, 0, stream>>>((const __nv_bfloat16*)k_cache, R, usign, hfit, v_star, ctx->P,
-                                                                        partials, ctx->unit_lens, c.n_max, ctx->row_stride, c.code_bits, it, bpu, dir);
-    else
-      fit_pass_kernel<float><<<grid, kFitThreads, 0, stream>>>((const float*)k_cache, R, usign, hfit, v_star, ctx->P, partials,
-                                                               ctx->unit_lens, c.n_max, ctx->row_stride, c.code_bits, it, bpu, dir);
-    fit_reduce_kernel<<<ctx->units, BPC_D, 0, stream>>>(partials, ctx->P, ctx->unit_lens, c.n_max, c.code_bits, it, bpu);
-    *launches += 2;
+    fit_prep_kernel<<<ctx->units, BPC_D, 0, stream>>>(ctx->P, v_star, dir, dots, c.code_bits, it, npow > 0 ? 1 : 0);
+#define BPC_FIT_PASS(KV, JPL)                                                                                          \
+    fit_pass_kernel<KV, JPL><<<grid, kFitThreads, 0, stream>>>((const KV*)k_cache, hfit, dir, dots, partials, agree,   \
+                                                                ctx->unit_lens, c.n_max, ctx->row_stride, it, bpu)
+    if (c.kv_dtype == BPC_BF16) {
+      if (c.code_bits == 64) BPC_FIT_PASS(__nv_bfloat16, 8); else if (c.code_bits == 128) BPC_FIT_PASS(__nv_bfloat16, 16); else BPC_FIT_PASS(__nv_bfloat16, 32);
+    } else {
+      if (c.code_bits == 64) BPC_FIT_PASS(float, 8); else if (c.code_bits == 128) BPC_FIT_PASS(float, 16); else BPC_FIT_PASS(float, 32);
+    }
+#undef BPC_FIT_PASS
+    fit_reduce_kernel<<<ctx->units, BPC_D * kRedGroups, 0, stream>>>(partials, agree, ctx->P, ctx->unit_lens, c.n_max, c.code_bits, it, bpu);
+    *launches += 3;
   }
   return cudaGetLastError();
 }
