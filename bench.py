@@ -473,7 +473,7 @@ def run_ours(args):
 
 # ----------------------------------------------------------------------------- paper-scale sweep (second workload)
 SWEEP_CASES = [  # (context, batch): 64-bit codes, fixed budgets, 32/8 heads, bf16, as in the paper's latency-vs-context study
-    (32768, 1), (32768, 16), (131072, 1), (131072, 8), (262144, 1), (262144, 4), (1048576, 1),
+    (32768, 1), (32768, 16), (131072, 1), (131072, 8), (262144, 1), (262144, 4), (1048576, 1), (2097152, 1),
 ]
 
 
@@ -520,7 +520,7 @@ def run_sweep(args):
             ms = _time_graph(g, lambda: None) / K
             err = max(ly.ctx.last_device_error() for ly in layers)
             rows.append({"context": n_ctx, "batch": batch, "budget": budget, "us_per_step": round(ms * 1e3, 2),
-                         "cluster_size": layers[0].ctx.get_cluster_size(), "layer_replicas": L,
+                         "cluster_size": layers[0].ctx.get_cluster_size(), "streaming": layers[0].ctx.uses_streaming(), "layer_replicas": L,
                          "algorithmic_GBps": round(step_bytes / ms / 1e6, 1), "device_error_word": err})
             layers = None
             g = None

@@ -84,8 +84,10 @@ bpc_status bpc_create(const bpc_config* host_cfg, bpc_ctx** host_out);
 bpc_status bpc_destroy(bpc_ctx* ctx);
 
 /* Sizes the caller needs: bytes of the code array, bytes of the workspace bpc_fit needs, the largest
- * n_max this build supports for cfg (scores of one unit are kept in the shared memory of one thread
- * block cluster), and the most keys a decode step can select per unit (= n_max). */
+ * n_max this build supports for cfg, and the most keys a decode step can select per unit (= n_max).  Normally the
+ * scores of one unit are kept in the shared memory of one thread block cluster (up to about 1.3 M keys per unit);
+ * longer units are served, for Hamming scores without the safeguard, by a streaming selection that stores no scores
+ * and reads the codes twice (n_max up to 2^26); the weighted score mode and the safeguard keep the cluster limit. */
 size_t  bpc_codes_bytes(const bpc_config* host_cfg);
 size_t  bpc_fit_workspace_bytes(const bpc_config* host_cfg);
 /* Byte offset inside the fit workspace at which bpc_fit leaves the codes H that Algorithm 1 itself
@@ -219,6 +221,8 @@ bpc_status bpc_debug_set_phase_timer(bpc_ctx* ctx, uint64_t* stamps);
  * Returns BPC_ERR_UNSUPPORTED if n_max does not fit that many blocks. */
 bpc_status bpc_set_cluster_size(bpc_ctx* ctx, int32_t cluster_size);
 int32_t    bpc_get_cluster_size(bpc_ctx* ctx);
+/* 1 when this context's decode calls use the streaming selection (units longer than a cluster's shared memory holds). */
+int32_t    bpc_uses_streaming(bpc_ctx* ctx);
 
 /* Diagnostics: device error word (synchronises the stream), last CUDA error code seen by the
  * context, number of kernels this context has launched so far. */

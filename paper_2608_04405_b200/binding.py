@@ -68,6 +68,7 @@ def _load() -> ctypes.CDLL:
         "bpc_debug_set_phase_timer": (i32, [vp, vp]),
         "bpc_set_cluster_size": (i32, [vp, i32]),
         "bpc_get_cluster_size": (i32, [vp]),
+        "bpc_uses_streaming": (i32, [vp]),
         "bpc_last_device_error": (i32, [vp, ctypes.POINTER(i32), vp]),
         "bpc_last_cuda_error": (i32, [vp]),
         "bpc_launch_count": (i64, [vp]),
@@ -87,7 +88,7 @@ EXPORTS = ["bpc_create", "bpc_destroy", "bpc_codes_bytes", "bpc_fit_workspace_by
            "bpc_encode_keys", "bpc_build_eas", "bpc_get_eas", "bpc_eas_capacity", "bpc_exact_topk", "bpc_append", "bpc_decode_attn", "bpc_append_decode_attn", "bpc_decode_attn_static", "bpc_static_scratch_entries",
            "bpc_debug_set_buffers", "bpc_debug_set_phase_timer",
            "bpc_set_cluster_size",
-           "bpc_get_cluster_size", "bpc_last_device_error", "bpc_last_cuda_error", "bpc_launch_count", "bpc_version"]
+           "bpc_get_cluster_size", "bpc_uses_streaming", "bpc_last_device_error", "bpc_last_cuda_error", "bpc_launch_count", "bpc_version"]
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -259,6 +260,9 @@ class Context:
     def debug_set_phase_timer(self, stamps: Optional[torch.Tensor]) -> None:
         self._stamps = stamps
         _check(lib.bpc_debug_set_phase_timer(self._h, _ptr(stamps)), "bpc_debug_set_phase_timer")
+
+    def uses_streaming(self) -> bool:
+        return bool(lib.bpc_uses_streaming(self._h))
 
     def last_device_error(self) -> int:
         v = ctypes.c_int32(0)

@@ -12,6 +12,8 @@ cudaError_t bpc_launch_decode_bf16_eas(bpc_ctx*, const DecodeParams&, cudaStream
 cudaError_t bpc_launch_decode_f32_eas(bpc_ctx*, const DecodeParams&, cudaStream_t);
 cudaError_t bpc_decode_limits_bf16_eas(const bpc_ctx*, int, int*, int*, size_t*);
 cudaError_t bpc_decode_limits_f32_eas(const bpc_ctx*, int, int*, int*, size_t*);
+cudaError_t bpc_launch_decode_bf16_stream(bpc_ctx*, const DecodeParams&, cudaStream_t);
+cudaError_t bpc_launch_decode_f32_stream(bpc_ctx*, const DecodeParams&, cudaStream_t);
 cudaError_t bpc_launch_decode_bf16_w7(bpc_ctx*, const DecodeParams&, cudaStream_t);
 cudaError_t bpc_launch_decode_f32_w7(bpc_ctx*, const DecodeParams&, cudaStream_t);
 cudaError_t bpc_decode_limits_bf16_w7(const bpc_ctx*, int, int*, int*, size_t*);
@@ -109,6 +111,21 @@ cudaError_t bpc_plan_decode_geometry(bpc_ctx* ctx) {
   for (int i = 0; i < 5; ++i) ctx->max_active[i] = mc[1 + i];
   ctx->chunk_cap_limit = cap;
   ctx->cluster_size = choose_cluster(ctx, cap, ctx->max_cluster);
+  ctx->streaming = false;
+  const char* force = getenv("BPC_FORCE_STREAMING");        // diagnostic switch: two-pass selection at any size
+  const bool forced = force != nullptr && force[0] == '1';
+  if ((ctx->cluster_size == 0 || forced) && ctx->cfg.score_mode == BPC_SCORE_HAMMING && ctx->cfg.eas_ppm == 0) {
+    // Units too long for the largest cluster's shared memory: no score is stored, the codes are read twice.  The
+    // largest cluster size that still runs all units in one wave is used (at least the largest schedulable one).
+    int cs = forced && ctx->cluster_size > 0 ? ctx->cluster_size : ctx->max_cluster;
+    if (!(forced && ctx->cluster_size > 0)) {
+      int li = 0;
+      for (int c = 1; c < ctx->max_cluster; c *= 2) ++li;
+      while (cs > 1 && ctx->units > ctx->max_active[li]) { cs /= 2; --li; }
+    }
+    ctx->cluster_size = cs;
+    ctx->streaming = true;
+  }
   return cudaSuccess;
 }
 
@@ -140,6 +157,7 @@ int64_t bpc_max_context(const bpc_config* c) {
   tmp.group = c->n_q_heads / c->n_kv_heads;
   if (cudaGetDevice(&tmp.device) != cudaSuccess) return 0;
   if (bpc_plan_decode_geometry(&tmp) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+  if (c->score_mode == BPC_SCORE_HAMMING && c->eas_ppm == 0) return (int64_t)1 << 26;   // streaming selection: no per-unit limit
   return (int64_t)tmp.max_cluster * tmp.chunk_cap_limit;
 }
 
@@ -210,14 +228,16 @@ bpc_status bpc_destroy(bpc_ctx* ctx) {
 bpc_status bpc_set_cluster_size(bpc_ctx* ctx, int32_t cs) {
   if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
   const int cap = ctx->chunk_cap_limit, mc = ctx->max_cluster;
+  if (cs == 0 && ctx->streaming) return BPC_OK;            // keeps the size chosen at creation
   if (cs == 0) cs = choose_cluster(ctx, cap, mc);
   if (cs < 1 || cs > mc || (cs & (cs - 1)) != 0) return BPC_ERR_UNSUPPORTED;
-  if (chunk_for(ctx->cfg.n_max, cs) > cap) return BPC_ERR_UNSUPPORTED;
+  if (!ctx->streaming && chunk_for(ctx->cfg.n_max, cs) > cap) return BPC_ERR_UNSUPPORTED;
   ctx->cluster_size = cs;
   return BPC_OK;
 }
 
 int32_t bpc_get_cluster_size(bpc_ctx* ctx) { return ctx ? ctx->cluster_size : 0; }
+int32_t bpc_uses_streaming(bpc_ctx* ctx) { return (ctx && ctx->streaming) ? 1 : 0; }
 
 bpc_status bpc_set_seq_lens(bpc_ctx* ctx, const int32_t* host_lens, void* stream) {
   if (ctx == nullptr || host_lens == nullptr) return BPC_ERR_INVALID_ARG;
@@ -373,11 +393,14 @@ static bpc_status decode_common(bpc_ctx* ctx, const void* k_new, const void* v_n
   p.shared_sets = c.hash_sets != ctx->units;
   p.budget_ppm = budget_ppm; p.budget_count = budget_count; p.sm_scale_d = ctx->sm_scale_d;
   const int chunk = chunk_for(c.n_max, ctx->cluster_size);
-  if (chunk > cap) return BPC_ERR_UNSUPPORTED;
-  p.chunk_cap = chunk;                                    // shared memory is sized for the largest possible unit
+  if (!ctx->streaming && chunk > cap) return BPC_ERR_UNSUPPORTED;
+  p.chunk_cap = ctx->streaming ? 0 : chunk;               // shared memory is sized for the largest possible unit
   p.nbins = hist_bins(ctx);
   p.hist_shift = hist_shift(ctx);
-  if (c.score_mode == BPC_SCORE_WEIGHTED7)
+  if (ctx->streaming)
+    e = c.kv_dtype == BPC_BF16 ? bpc_launch_decode_bf16_stream(ctx, p, (cudaStream_t)stream)
+                               : bpc_launch_decode_f32_stream(ctx, p, (cudaStream_t)stream);
+  else if (c.score_mode == BPC_SCORE_WEIGHTED7)
     e = c.kv_dtype == BPC_BF16 ? bpc_launch_decode_bf16_w7(ctx, p, (cudaStream_t)stream)
                                : bpc_launch_decode_f32_w7(ctx, p, (cudaStream_t)stream);
   else if (c.eas_ppm > 0)

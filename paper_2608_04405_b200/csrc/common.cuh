@@ -35,6 +35,7 @@ struct bpc_ctx {
   int sm_count;
   bool fitted;
   bool use_pdl;             // launch the decode kernel with programmatic stream serialization
+  bool streaming;           // the scores of a full unit do not fit the largest cluster: two-pass (streaming) selection
   float* P;                 // [hash_sets][b][D] float
   void*  P_h;               // [hash_sets][b][D] cache dtype (the hash function)
   float* P_hf;              // P_h as float values

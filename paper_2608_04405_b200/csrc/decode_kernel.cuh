@@ -45,6 +45,7 @@ struct SmallState {
   uint32_t mask[kMaxPlanes][8];
   uint32_t gt[BPC_MAX_CLUSTER];
   uint32_t eq[BPC_MAX_CLUSTER];
+  uint32_t wgt[32], weq[32];             // streaming selection: per-warp numbers of keys above / at the threshold
   uint32_t wscan[64];                    // block scans: two alternating buffers of 2 x 16 warp totals (16-byte aligned)
   double pmax[BPC_MAX_GROUP];
   int T, cnt_gt, my_take, my_base, rsum, e0, e1, pad;
@@ -248,11 +249,15 @@ struct RowFragF32 {
   }
 };
 
-// EAS = 1 compiles the error-aware safeguard in (a static hard-to-hash set that is always attended); EAS = 0 is the
-// plain path with none of that code.
-template <typename KV, int GP, int W32, int MODE, int EAS>
+// VAR selects what is compiled in besides the plain path (VAR = 0): 1 = the error-aware safeguard (a static
+// hard-to-hash set that is always attended); 2 = the streaming selection for units whose scores do not fit the
+// cluster's shared memory (no score is stored: the scan keeps one histogram per warp over that warp's contiguous key
+// range, and after the threshold is known every warp reads its codes a second time and emits its selection in order).
+template <typename KV, int GP, int W32, int MODE, int VAR>
 __global__ void __launch_bounds__((DecodeSmem<KV, GP, W32>::NT), 1)
 bpc_decode_kernel(const DecodeParams p) {
+  constexpr int EAS = VAR == 1 ? 1 : 0;
+  constexpr bool STREAM = VAR == 2;
   typedef DecodeSmem<KV, GP, W32> L;
   typedef typename L::acc_t acc_t;
   constexpr int NT = L::NT, NW = L::NW, B = L::B;
@@ -330,7 +335,7 @@ bpc_decode_kernel(const DecodeParams p) {
 
   // Both early exits depend only on values every block of the cluster sees identically, so either all
   // blocks of a cluster leave here (before any cluster barrier) or none does.
-  if (chunk > p.chunk_cap) {
+  if (!STREAM && chunk > p.chunk_cap) {
     if (tid == 0) atomicOr(p.err, BPC_DEVERR_CHUNK_CAP);
     return;
   }
@@ -368,7 +373,8 @@ bpc_decode_kernel(const DecodeParams p) {
   const float* gsm = nullptr;
   if (appender && p.residual_correction != 0) {
     const size_t union_bytes = plan.total - plan.off_union;
-    const size_t score_bytes = (size_t)((p.chunk_cap + kSegKeys - 1) / kSegKeys) * kSegSlots * 2;
+    const size_t score_bytes = STREAM ? (size_t)NW * nbins * 4      // (streaming: the per-warp histograms sit there)
+                                      : (size_t)((p.chunk_cap + kSegKeys - 1) / kSegKeys) * kSegSlots * 2;
     constexpr size_t kGramPad = 0;
     if (score_bytes + (size_t)B * B * 4 + kGramPad <= union_bytes && L::hashpart_bytes() + (size_t)B * B * 4 + kGramPad <= union_bytes) {
       float* dstg = reinterpret_cast<float*>(uni + union_bytes - (size_t)B * B * 4 - kGramPad);
@@ -406,7 +412,7 @@ bpc_decode_kernel(const DecodeParams p) {
   };
   uint32_t ha[U][W32], hb[U][W32];
   const bool pipelined = tid < nts && c0 + nts * U <= c1s;   // at least one full batch
-  if (pipelined) load_batch(ha, c0);
+  if (!STREAM && pipelined) load_batch(ha, c0);
 
   // ------------------------------------------------------------------ phase 0: query hash
   // p[g][j] = P_h[j] . q_g.  Thread (part, j) covers a slice of the 128 channels of row j: products are
@@ -560,7 +566,7 @@ bpc_decode_kernel(const DecodeParams p) {
         atomicAdd(&hist[key >> hsh], 1u);
       }
     };
-    const int STEP = nts * U;
+    [[maybe_unused]] const int STEP = nts * U;
     if (dbg != nullptr) {                                    // score export (tests): a plain loop, one key at a time
 #pragma unroll 1
       for (int i = c0 + tid; i < c1s; i += nts) {
@@ -569,6 +575,27 @@ bpc_decode_kernel(const DecodeParams p) {
         dbg[i] = ((2 * score_key<W32, NP>(h, sg, mk)) << cs) - rfull;
       }
     }
+    if constexpr (STREAM) {
+      // Streaming selection, first pass: warp w owns the contiguous keys [w0, w1) and counts their score keys in its
+      // own histogram (no score is stored).  A batch is U codes per lane, 32 keys apart.
+      uint32_t* whist = reinterpret_cast<uint32_t*>(uni) + (size_t)warp * nbins;
+      for (int i = lane; i < nbins; i += 32) whist[i] = 0u;
+      __syncwarp();
+      const int nw = nts >> 5;
+      const int wlen = (((c1s - c0) + nw - 1) / nw + 31) & ~31;
+      const int w0 = min(c1s, c0 + warp * wlen), w1 = min(c1s, w0 + wlen);
+#pragma unroll 1
+      for (int base = w0; base < w1; base += 32 * U) {
+        uint32_t h[U][W32];
+#pragma unroll
+        for (int u = 0; u < U; ++u) load_code(h[u], min(base + 32 * u + lane, w1 - 1));
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const int key = score_key<W32, NP>(h[u], sg, mk);
+          if (base + 32 * u + lane < w1) atomicAdd(&whist[key], 1u);
+        }
+      }
+    } else {
     int i0 = c0;
     if (pipelined) {
       // Full batches without bounds checks, software-pipelined over two register buffers so that the
@@ -610,6 +637,7 @@ bpc_decode_kernel(const DecodeParams p) {
           atomicAdd(&hist[key >> hsh], 1u);
         }
       }
+    }
     }
     if (p.dbg_times != nullptr && tid == 0) p.dbg_times[(size_t)blockIdx.x * 16 + 13] = (unsigned long long)clock64();
   } else {
@@ -689,7 +717,29 @@ bpc_decode_kernel(const DecodeParams p) {
     }
     if (p.dbg_times != nullptr && lane == 0) p.dbg_times[(size_t)blockIdx.x * 16 + 11] = (unsigned long long)clock64();
   }
-  if (appender) {
+  int newkey = -1;                                           // streaming: score key of the key appended by this launch
+  if constexpr (STREAM) {
+    __syncthreads();                                         // every warp's histogram is complete (and the new code is known)
+    if (appender) {
+      uint32_t sg[W32], mk[NP][W32], h[W32];
+#pragma unroll
+      for (int w = 0; w < W32; ++w) {
+        sg[w] = st->signw[w]; h[w] = st->newcode[w];
+#pragma unroll
+        for (int pl = 0; pl < NP; ++pl) mk[pl][w] = st->mask[pl][w];
+      }
+      newkey = score_key<W32, NP>(h, sg, mk);
+      if (tid == 0 && p.dbg_scores != nullptr) p.dbg_scores[(size_t)unit * p.n_max + (n - 1)] = ((2 * newkey) << cs) - (st->rsum << cs);
+    }
+    const uint32_t* wh = reinterpret_cast<const uint32_t*>(uni);
+    const int nw = nts >> 5;
+    for (int bin = tid; bin < nbins; bin += NT) {
+      uint32_t sum = bin == newkey ? 1u : 0u;
+      for (int w = 0; w < nw; ++w) sum += wh[(size_t)w * nbins + bin];
+      hist[bin] = sum;
+    }
+  }
+  if (!STREAM && appender) {
     __syncthreads();                                         // the new code is in shared memory; the scan is done
     if (tid == 0) {
       uint32_t sg[W32], mk[NP][W32], h[W32];
@@ -714,7 +764,7 @@ bpc_decode_kernel(const DecodeParams p) {
   uint32_t* pushed = nullptr;
   {
     const size_t union_bytes = plan.total - plan.off_union;
-    size_t push_off = (size_t)((p.chunk_cap + kSegKeys - 1) / kSegKeys) * kSegSlots * 2;
+    size_t push_off = STREAM ? (size_t)NW * nbins * 4 : (size_t)((p.chunk_cap + kSegKeys - 1) / kSegKeys) * kSegSlots * 2;
     if (push_off < L::hashpart_bytes()) push_off = L::hashpart_bytes();   // a peer may still be hashing
     push_off = (push_off + 15) & ~(size_t)15;
     if (fast_sel && CS > 1 && push_off + (size_t)CS * nbins * 4 + (size_t)B * B * 4 <= union_bytes)
@@ -906,7 +956,61 @@ bpc_decode_kernel(const DecodeParams p) {
   if (!kFastOnly && !fast_sel) __syncthreads();                            // (the fast path published its values before its own barrier)
   int32_t* sel_u = p.sel + (size_t)unit * p.n_max;
   BPC_STAMP(10);
-  {
+  if constexpr (STREAM) {
+    // Streaming selection, second pass.  Per-warp numbers of keys above and at the threshold come from the warps'
+    // histograms; a warp's output starts after the keys of the warps before it (ties are granted in warp order, which
+    // is index order), and inside the warp one ballot per 32 keys keeps the order.
+    const int my_take = st->my_take, my_base = st->my_base, Tk = T_exact;
+    const uint32_t* whist = reinterpret_cast<const uint32_t*>(uni) + (size_t)warp * nbins;
+    const int nw = nts >> 5;
+    if (tid < nts) {
+      uint32_t g = 0;
+      for (int bin = Tk + 1 + lane; bin < nbins; bin += 32) g += whist[bin];
+      g = __reduce_add_sync(0xffffffffu, g);
+      if (lane == 0) { st->wgt[warp] = g; st->weq[warp] = whist[Tk]; }
+    }
+    __syncthreads();
+    if (tid < nts && kh > 0) {
+      int gt_before = 0, eq_before = 0;
+      for (int w = 0; w < warp; ++w) { gt_before += (int)st->wgt[w]; eq_before += (int)st->weq[w]; }
+      const int take_w = min(max(my_take - eq_before, 0), (int)st->weq[warp]);
+      int pos = my_base + gt_before + min(eq_before, my_take);
+      int run_eq = 0;
+      uint32_t sg[W32], mk[NP][W32];
+#pragma unroll
+      for (int w = 0; w < W32; ++w) {
+        sg[w] = st->signw[w];
+#pragma unroll
+        for (int pl = 0; pl < NP; ++pl) mk[pl][w] = st->mask[pl][w];
+      }
+      const int wlen = (((c1s - c0) + nw - 1) / nw + 31) & ~31;
+      const int w0 = min(c1s, c0 + warp * wlen), w1 = min(c1s, w0 + wlen);
+      const uint32_t lt = (1u << lane) - 1u;
+#pragma unroll 1
+      for (int base = w0; base < w1; base += 32 * U) {
+        uint32_t h[U][W32];
+#pragma unroll
+        for (int u = 0; u < U; ++u) load_code(h[u], min(base + 32 * u + lane, w1 - 1));
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const int i = base + 32 * u + lane;
+          const int key = score_key<W32, NP>(h[u], sg, mk);
+          const bool valid = i < w1;
+          const uint32_t be = __ballot_sync(0xffffffffu, valid && key == Tk);
+          const bool takes = valid && (key > Tk || (key == Tk && run_eq + __popc(be & lt) < take_w));
+          const uint32_t bs = __ballot_sync(0xffffffffu, takes);
+          if (takes) sel_u[pos + __popc(bs & lt)] = i;
+          pos += __popc(bs);
+          run_eq += __popc(be);
+        }
+      }
+    }
+    if (appender && tid == 0 && kh > 0) {                    // the appended key is the last key of this block's range
+      int gt_all = 0, eq_all = 0;
+      for (int w = 0; w < nw; ++w) { gt_all += (int)st->wgt[w]; eq_all += (int)st->weq[w]; }
+      if (newkey > Tk || (newkey == Tk && eq_all < my_take)) sel_u[my_base + gt_all + min(eq_all, my_take)] = n - 1;
+    }
+  } else {
     // Each thread owns whole 32-key segments, in ascending order within a pass.  Two keys share a 32-bit
     // word; adding (0x8000 - T) to both halves raises bit 15 / bit 31 exactly for keys >= T (keys < 2048),
     // which is shifted into a 32-bit candidate mask without branches.  Only the few candidates are looked

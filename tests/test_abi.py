@@ -33,7 +33,7 @@ def test_size_queries_and_config_validation_without_gpu():
     bad = B.make_config(1, 4, 1, 1024, 96, torch.bfloat16)
     assert B.lib.bpc_codes_bytes(ctypes.byref(bad)) == 0
     off = B.lib.bpc_fit_codes_offset(ctypes.byref(cfg64))
-    assert 0 < off < B.lib.bpc_fit_workspace_bytes(ctypes.byref(cfg64))
+    assert 0 <= off < B.lib.bpc_fit_workspace_bytes(ctypes.byref(cfg64))   # (the fitted codes open the workspace)
     assert off % 256 == 0
 
 

@@ -364,6 +364,44 @@ def test_fit_with_power_iterations(dtype, bits, n, power):
     print(rep)
 
 
+def test_streaming_selection_two_million_keys():
+    """A unit longer than the largest cluster's shared memory holds (the 2M-token point of the paper's latency-vs-context
+    study): the library switches to the streaming selection (per-warp histograms, codes read twice); same checks as
+    everywhere else, on a 2-KV-head model to bound memory: plain and fused steps, fixed budget of 2048 keys."""
+    H = _harness()
+    spec = CONFIGS[1].scaled(name="stream2m", wid=90, batch=1, n_kv_heads=2, n_q_heads=8, n_ctx=2097152, code_bits=64, steps=2)
+    sess = H.Session(spec, gen_device="cuda", interleaved=True)
+    assert sess.ctx.uses_streaming()
+    rep = {}
+    sess.fit()
+    sess.encode(); H.check_encode(sess, [1], rep, max_keys=4096)
+    q, _ = sess.w.queries(sess.lens)
+    H.check_decode(sess, q.cuda(), [0, 1], rep, budget_count=2048)
+    k_new, v_new = sess.w.new_kv(sess.lens)
+    q, _ = sess.w.queries(sess.lens)
+    H.check_decode(sess, q.cuda(), [1], rep, budget_count=1024, append=(k_new.cuda(), v_new.cuda()))
+    print(rep)
+
+
+@pytest.mark.parametrize("dtype,bits,group,n,cluster", [("bf16", 128, 4, 40000, 4), ("f32", 64, 2, 9000, 2), ("bf16", 256, 8, 7000, 1)])
+def test_streaming_selection_forced_at_ordinary_sizes(dtype, bits, group, n, cluster, monkeypatch):
+    """The streaming selection forced on contexts that would fit (diagnostic switch), so that it is checked stage by
+    stage at sizes the checker handles in full: several cluster sizes, both cache types, fused steps and ties."""
+    monkeypatch.setenv("BPC_FORCE_STREAMING", "1")
+    H = _harness()
+    spec = CONFIGS[1].scaled(name="streamf", wid=91 + group, batch=2, n_kv_heads=2, n_q_heads=2 * group, n_ctx=n, dtype=dtype,
+                             code_bits=bits, steps=3)
+    sess = H.Session(spec, gen_device="cuda", cluster_size=cluster)
+    assert sess.ctx.uses_streaming()
+    rep = {}
+    sess.fit(); sess.encode()
+    _decode_loop(sess, 3, [0, 3], rep, H)
+    q, _ = sess.w.queries(sess.lens)
+    for ppm in (1000, 500000, 1000000):
+        H.check_decode(sess, q.cuda(), [1, 2], rep, budget_ppm=ppm)
+    print(rep)
+
+
 @pytest.mark.parametrize("dtype,bits,group,n", [("bf16", 128, 4, 9000), ("f32", 64, 2, 5000), ("bf16", 256, 8, 6000)])
 def test_quality_yardsticks(dtype, bits, group, n):
     """The TOPK (Oracle) selector and dense attention (appendix "Baseline Methods"; cosine-similarity table), and the two
