@@ -533,7 +533,7 @@ def run_sweep(args):
 
 # ----------------------------------------------------------------------------- quality yard-sticks
 def run_quality(args):
-    """Selection quality on the synthetic workload for code lengths 64, 128 and 256: recall of the hash selection with
+    """Selection quality on the synthetic workload for code lengths 32, 64, 128 and 256: recall of the hash selection with
     respect to the exact-score top-k of every query head (the paper's TOPK (Oracle) baseline), cosine similarity between
     the sparse output and dense attention (the paper's output-similarity table), and recall of the planted needles.
     All three selections and both outputs come from the library (bpc_exact_topk, bpc_decode_attn with the workload's
@@ -542,7 +542,7 @@ def run_quality(args):
     torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
     spec0 = CONFIGS[args.workload]
     rows = []
-    for bits in (64, 128, 256):
+    for bits in (32, 64, 128, 256):
         spec = spec0.scaled(code_bits=bits)
         w = Workload(spec, device="cuda", extra_rows=64)
         cfg = B.make_config(spec.batch, spec.n_q_heads, spec.n_kv_heads, w.n_max, bits, spec.torch_dtype)
@@ -589,8 +589,7 @@ def run_quality(args):
         del ctx, mctx, codes, w, hsel, tsel, sparse, dense
         torch.cuda.empty_cache()
     print(json.dumps({"metric": "selection_quality", "data": "synthetic", "dtype": "bf16",
-                      "config": {"workload": spec0.name, "budget_ppm": spec0.budget_ppm, "code_bits": [64, 128, 256],
-                                 "note": "32-bit codes are not supported by this library"},
+                      "config": {"workload": spec0.name, "budget_ppm": spec0.budget_ppm, "code_bits": [32, 64, 128, 256]},
                       "cases": rows}))
 
 
@@ -672,7 +671,7 @@ def main():
     ap.add_argument("--separate-kv", action="store_true", help="separate K and V arrays instead of interleaved rows")
     ap.add_argument("--profile", action="store_true", help="warm-up plus K eager steps only (for ncu captures)")
     ap.add_argument("--sweep", action="store_true", help="second workload: latency over contexts and batch sizes, 64-bit codes, 1K/2K budgets")
-    ap.add_argument("--quality", action="store_true", help="selection quality yard-sticks (recall vs exact top-k, cosine vs dense) for 64/128/256-bit codes")
+    ap.add_argument("--quality", action="store_true", help="selection quality yard-sticks (recall vs exact top-k, cosine vs dense) for 32/64/128/256-bit codes")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

@@ -63,7 +63,7 @@ typedef struct {
   int32_t n_q_heads;
   int32_t n_kv_heads;
   int32_t head_dim;             /* 128 */
-  int32_t code_bits;            /* 64 | 128 | 256 */
+  int32_t code_bits;            /* 32 | 64 | 128 | 256 (with 32, n_max must be a multiple of 4) */
   int32_t n_max;                /* rows per unit in the caches and the code array */
   int32_t kv_dtype;             /* bpc_dtype */
   int32_t score_mode;           /* bpc_score_mode */

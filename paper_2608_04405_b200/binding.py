@@ -157,6 +157,8 @@ class Context:
 
     def alloc_codes(self, device="cuda") -> torch.Tensor:
         c = self.cfg
+        if c.code_bits == 32:            # half a 64-bit word per key: one int32
+            return torch.zeros(c.batch, c.n_kv_heads, c.n_max, 1, dtype=torch.int32, device=device)
         return torch.zeros(c.batch, c.n_kv_heads, c.n_max, c.code_bits // 64, dtype=torch.int64, device=device)
 
     def fit_workspace_bytes(self) -> int:

@@ -27,7 +27,8 @@ bpc_status check_cfg(const bpc_config* c) {
   if (c == nullptr) return BPC_ERR_INVALID_ARG;
   if (c->batch < 1 || c->n_kv_heads < 1 || c->n_q_heads < 1 || c->n_max < 1) return BPC_ERR_INVALID_ARG;
   if (c->head_dim != BPC_D) return BPC_ERR_UNSUPPORTED;
-  if (c->code_bits != 64 && c->code_bits != 128 && c->code_bits != 256) return BPC_ERR_UNSUPPORTED;
+  if (c->code_bits != 32 && c->code_bits != 64 && c->code_bits != 128 && c->code_bits != 256) return BPC_ERR_UNSUPPORTED;
+  if (c->code_bits == 32 && c->n_max % 4 != 0) return BPC_ERR_INVALID_ARG;   // 16-byte aligned code rows per unit
   if (c->n_q_heads % c->n_kv_heads != 0) return BPC_ERR_INVALID_ARG;
   if (c->n_q_heads / c->n_kv_heads > BPC_MAX_GROUP) return BPC_ERR_UNSUPPORTED;
   if (c->kv_dtype != BPC_BF16 && c->kv_dtype != BPC_F32) return BPC_ERR_UNSUPPORTED;

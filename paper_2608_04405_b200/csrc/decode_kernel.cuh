@@ -396,7 +396,9 @@ bpc_decode_kernel(const DecodeParams p) {
   constexpr int U = W32 <= 4 ? 8 : 4;                       // codes in flight per thread and buffer
   auto load_code = [&](uint32_t (&h)[W32], int i) {
     const uint32_t* src = cu + (size_t)i * W32;
-    if (W32 == 2) {
+    if (W32 == 1) {
+      h[0] = ld_stream_u32(src);
+    } else if (W32 == 2) {
       const uint2 v = ld_stream_v2(src); h[0] = v.x; h[1] = v.y;
     } else {
 #pragma unroll

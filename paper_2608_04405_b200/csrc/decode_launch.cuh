@@ -94,6 +94,7 @@ static cudaError_t limits_one(const bpc_ctx* ctx, int nbins, int* max_cluster, i
 
 #define BPC_DISPATCH_W(KV, GP, MODE, EAS, FN, ...)                                   \
   switch (ctx->cfg.code_bits) {                                                      \
+    case 32:  return FN<KV, GP, 1, MODE, EAS>(__VA_ARGS__);                          \
     case 64:  return FN<KV, GP, 2, MODE, EAS>(__VA_ARGS__);                          \
     case 128: return FN<KV, GP, 4, MODE, EAS>(__VA_ARGS__);                          \
     case 256: return FN<KV, GP, 8, MODE, EAS>(__VA_ARGS__);                          \

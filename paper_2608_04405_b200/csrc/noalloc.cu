@@ -70,7 +70,7 @@ bpc_status bpc_decode_attn_static(const bpc_config* cfg, const void* q, const vo
   if (cfg->batch < 1 || cfg->n_kv_heads < 1 || cfg->n_q_heads < 1 || cfg->n_max < 1 || cfg->n_max % 2 != 0)
     return BPC_ERR_INVALID_ARG;
   if (cfg->head_dim != BPC_D) return BPC_ERR_UNSUPPORTED;
-  if (cfg->code_bits != 64 && cfg->code_bits != 128 && cfg->code_bits != 256) return BPC_ERR_UNSUPPORTED;
+  if (cfg->code_bits != 32 && cfg->code_bits != 64 && cfg->code_bits != 128 && cfg->code_bits != 256) return BPC_ERR_UNSUPPORTED;
   if (cfg->n_q_heads % cfg->n_kv_heads != 0) return BPC_ERR_INVALID_ARG;
   const int group = cfg->n_q_heads / cfg->n_kv_heads;
   if (group > BPC_MAX_GROUP) return BPC_ERR_UNSUPPORTED;

@@ -88,7 +88,7 @@ encode_simple_kernel(const KV* __restrict__ k_cache, const float* __restrict__ P
       ts[(size_t)(jb + j) * kEncThreads + threadIdx.x] = (float)((a0 + a1) + (a2 + a3));
     }
   }
-  uint32_t* dst = reinterpret_cast<uint32_t*>(codes + ((size_t)unit * n_max + (live ? key : 0)) * (b / 64));
+  uint32_t* dst = reinterpret_cast<uint32_t*>(codes) + ((size_t)unit * n_max + (live ? key : 0)) * (b / 32);
   uint32_t word = 0;
   double abs_sum = 0.0;                                              // sum of |t_i| at decision time
   for (int i = 0; i < b; ++i) {
@@ -195,7 +195,7 @@ append_kernel(const KV* __restrict__ k_new, const KV* __restrict__ v_new, KV* __
       }
       if (lane == 0) {
         ubits_s[blk] = bits;
-        reinterpret_cast<uint32_t*>(codes + ((size_t)unit * n_max + n) * (b / 64))[blk] = bits;
+        (reinterpret_cast<uint32_t*>(codes) + ((size_t)unit * n_max + n) * (b / 32))[blk] = bits;
       }
     }
     __syncthreads();
@@ -708,9 +708,9 @@ cudaError_t bpc_launch_fit(bpc_ctx* ctx, const void* k_cache, const float* v_sta
     fit_pass_kernel<KV, JPL><<<grid, kFitThreads, 0, stream>>>((const KV*)k_cache, hfit, dir, dots, partials, agree,   \
                                                                 ctx->unit_lens, c.n_max, ctx->row_stride, it, bpu)
     if (c.kv_dtype == BPC_BF16) {
-      if (c.code_bits == 64) BPC_FIT_PASS(__nv_bfloat16, 8); else if (c.code_bits == 128) BPC_FIT_PASS(__nv_bfloat16, 16); else BPC_FIT_PASS(__nv_bfloat16, 32);
+      if (c.code_bits == 32) BPC_FIT_PASS(__nv_bfloat16, 4); else if (c.code_bits == 64) BPC_FIT_PASS(__nv_bfloat16, 8); else if (c.code_bits == 128) BPC_FIT_PASS(__nv_bfloat16, 16); else BPC_FIT_PASS(__nv_bfloat16, 32);
     } else {
-      if (c.code_bits == 64) BPC_FIT_PASS(float, 8); else if (c.code_bits == 128) BPC_FIT_PASS(float, 16); else BPC_FIT_PASS(float, 32);
+      if (c.code_bits == 32) BPC_FIT_PASS(float, 4); else if (c.code_bits == 64) BPC_FIT_PASS(float, 8); else if (c.code_bits == 128) BPC_FIT_PASS(float, 16); else BPC_FIT_PASS(float, 32);
     }
 #undef BPC_FIT_PASS
     fit_reduce_kernel<<<ctx->units, BPC_D * kRedGroups, 0, stream>>>(partials, agree, ctx->P, ctx->unit_lens, c.n_max, c.code_bits, it, bpu);

@@ -30,7 +30,10 @@ def _np64(t: torch.Tensor) -> np.ndarray:
 
 
 def codes_to_bits(codes_unit: torch.Tensor, b: int) -> np.ndarray:
-    """codes [n, b/64] int64 (device or host) -> bits [n, b] uint8."""
+    """codes [n, b/64] int64 (or [n, 1] int32 at b = 32; device or host) -> bits [n, b] uint8."""
+    if b == 32:          # widen the 32-bit words to the 64-bit words the checker unpacks (upper half zero)
+        w = codes_unit.detach().cpu().numpy().view(np.uint32).astype(np.uint64)
+        return O.unpack_bits(w, b)
     w = codes_unit.detach().cpu().numpy().view(np.uint64)
     return O.unpack_bits(w, b)
 
@@ -84,6 +87,10 @@ class Session:
     def hfit_bits(self, u: int) -> np.ndarray:
         s = self.spec
         off = self.ctx.fit_codes_offset()
+        if s.code_bits == 32:
+            raw = self.fit_ws[off: off + self.units * self.w.n_max * 4].view(torch.int32).view(self.units, self.w.n_max, 1)
+            _, _, n = self.unit_views(u)
+            return codes_to_bits(raw[u, :n], 32)
         words = s.code_bits // 64
         n_max = self.w.n_max
         raw = self.fit_ws[off: off + self.units * n_max * words * 8].view(torch.int64).view(self.units, n_max, words)

@@ -30,6 +30,8 @@ def test_size_queries_and_config_validation_without_gpu():
     assert B.lib.bpc_codes_bytes(ctypes.byref(cfg)) == 4 * 8 * (131072 + 256) * 16
     cfg64 = B.make_config(1, 1, 1, 4096, 64, torch.float32)
     assert B.lib.bpc_codes_bytes(ctypes.byref(cfg64)) == 4096 * 8        # one 64-bit word per key
+    cfg32 = B.make_config(1, 4, 1, 4096, 32, torch.float32)
+    assert B.lib.bpc_codes_bytes(ctypes.byref(cfg32)) == 4096 * 4        # half a word per key
     bad = B.make_config(1, 4, 1, 1024, 96, torch.bfloat16)
     assert B.lib.bpc_codes_bytes(ctypes.byref(bad)) == 0
     off = B.lib.bpc_fit_codes_offset(ctypes.byref(cfg64))

@@ -57,7 +57,8 @@ def test_cluster_sizes_agree_with_checker(cluster):
 
 
 @pytest.mark.parametrize("bits,group,dtype", [(64, 1, "bf16"), (64, 4, "bf16"), (256, 4, "bf16"), (128, 7, "bf16"),
-                                              (128, 8, "bf16"), (128, 2, "bf16"), (128, 3, "f32"), (256, 1, "f32")])
+                                              (128, 8, "bf16"), (128, 2, "bf16"), (128, 3, "f32"), (256, 1, "f32"),
+                                              (32, 4, "bf16"), (32, 1, "f32"), (32, 8, "bf16")])
 def test_code_lengths_and_group_sizes(bits, group, dtype):
     H = _harness()
     spec = CONFIGS[1].scaled(n_ctx=3000, n_kv_heads=2, n_q_heads=2 * group, code_bits=bits, dtype=dtype, steps=1,
@@ -191,7 +192,7 @@ def test_fused_append_decode_tiny_and_boundary_lengths():
 
 
 @pytest.mark.parametrize("bits,group,dtype,n", [(128, 4, "bf16", 9000), (64, 8, "bf16", 3000), (256, 1, "bf16", 3000),
-                                                 (64, 2, "f32", 2500), (128, 3, "bf16", 40000)])
+                                                 (64, 2, "f32", 2500), (128, 3, "bf16", 40000), (32, 4, "bf16", 5000)])
 def test_weighted_scores_seven_magnitude_planes(bits, group, dtype, n):
     """Algorithm 3 as printed (sign + 7 magnitude planes per head): scores, selection with the two-level
     histogram, output; separate calls and the fused cache write."""
@@ -383,7 +384,8 @@ def test_streaming_selection_two_million_keys():
     print(rep)
 
 
-@pytest.mark.parametrize("dtype,bits,group,n,cluster", [("bf16", 128, 4, 40000, 4), ("f32", 64, 2, 9000, 2), ("bf16", 256, 8, 7000, 1)])
+@pytest.mark.parametrize("dtype,bits,group,n,cluster", [("bf16", 128, 4, 40000, 4), ("f32", 64, 2, 9000, 2), ("bf16", 256, 8, 7000, 1),
+                                                        ("bf16", 32, 4, 12000, 2)])
 def test_streaming_selection_forced_at_ordinary_sizes(dtype, bits, group, n, cluster, monkeypatch):
     """The streaming selection forced on contexts that would fit (diagnostic switch), so that it is checked stage by
     stage at sizes the checker handles in full: several cluster sizes, both cache types, fused steps and ties."""
@@ -402,7 +404,7 @@ def test_streaming_selection_forced_at_ordinary_sizes(dtype, bits, group, n, clu
     print(rep)
 
 
-@pytest.mark.parametrize("dtype,bits,group,n", [("bf16", 128, 4, 9000), ("f32", 64, 2, 5000), ("bf16", 256, 8, 6000)])
+@pytest.mark.parametrize("dtype,bits,group,n", [("bf16", 128, 4, 9000), ("f32", 64, 2, 5000), ("bf16", 256, 8, 6000), ("bf16", 32, 4, 7000)])
 def test_quality_yardsticks(dtype, bits, group, n):
     """The TOPK (Oracle) selector and dense attention (appendix "Baseline Methods"; cosine-similarity table), and the two
     numbers built on them: recall of the hash selection against the exact top-k, cosine of sparse against dense output."""
@@ -440,7 +442,7 @@ def test_sweep_shapes_single_word_codes_fixed_budgets(n_ctx, batch):
 
 
 @pytest.mark.parametrize("dtype,bits,group,n,cluster", [("bf16", 128, 4, 9000, 0), ("bf16", 128, 4, 9000, 1), ("bf16", 64, 8, 5000, 2),
-                                                        ("f32", 64, 2, 4096, 0), ("bf16", 256, 1, 3000, 0)])
+                                                        ("f32", 64, 2, 4096, 0), ("bf16", 256, 1, 3000, 0), ("bf16", 32, 4, 6000, 0)])
 def test_error_aware_safeguard(dtype, bits, group, n, cluster):
     """EAS: per-key reconstruction errors from both encode paths, the static hard-to-hash set, and decode steps whose
     selection is the union of the hash top-(k - m) and that set (10 % of a 2 % budget), incl. the fused cache write."""
