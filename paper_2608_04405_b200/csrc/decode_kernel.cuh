@@ -586,16 +586,26 @@ bpc_decode_kernel(const DecodeParams p) {
       const int nw = nts >> 5;
       const int wlen = (((c1s - c0) + nw - 1) / nw + 31) & ~31;
       const int w0 = min(c1s, c0 + warp * wlen), w1 = min(c1s, w0 + wlen);
-#pragma unroll 1
-      for (int base = w0; base < w1; base += 32 * U) {
-        uint32_t h[U][W32];
+      constexpr int WSTEP = 32 * U;
+      auto wload = [&](uint32_t (&h)[U][W32], int base) {    // indices past the range are clamped (their scores are dropped)
 #pragma unroll
         for (int u = 0; u < U; ++u) load_code(h[u], min(base + 32 * u + lane, w1 - 1));
+      };
+      auto wcount = [&](const uint32_t (&h)[U][W32], int base) {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
           const int key = score_key<W32, NP>(h[u], sg, mk);
           if (base + 32 * u + lane < w1) atomicAdd(&whist[key], 1u);
         }
+      };
+      if (w0 < w1) wload(ha, w0);
+#pragma unroll 1
+      for (int base = w0; base < w1; base += 2 * WSTEP) {    // two register buffers: one batch in flight while one is scored
+        if (base + WSTEP < w1) wload(hb, base + WSTEP);
+        wcount(ha, base);
+        if (base + WSTEP >= w1) break;
+        if (base + 2 * WSTEP < w1) wload(ha, base + 2 * WSTEP);
+        wcount(hb, base + WSTEP);
       }
     } else {
     int i0 = c0;
@@ -988,11 +998,12 @@ bpc_decode_kernel(const DecodeParams p) {
       const int wlen = (((c1s - c0) + nw - 1) / nw + 31) & ~31;
       const int w0 = min(c1s, c0 + warp * wlen), w1 = min(c1s, w0 + wlen);
       const uint32_t lt = (1u << lane) - 1u;
-#pragma unroll 1
-      for (int base = w0; base < w1; base += 32 * U) {
-        uint32_t h[U][W32];
+      constexpr int WSTEP = 32 * U;
+      auto wload = [&](uint32_t (&h)[U][W32], int base) {
 #pragma unroll
         for (int u = 0; u < U; ++u) load_code(h[u], min(base + 32 * u + lane, w1 - 1));
+      };
+      auto wemit = [&](const uint32_t (&h)[U][W32], int base) {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
           const int i = base + 32 * u + lane;
@@ -1005,6 +1016,15 @@ bpc_decode_kernel(const DecodeParams p) {
           pos += __popc(bs);
           run_eq += __popc(be);
         }
+      };
+      if (w0 < w1) wload(ha, w0);
+#pragma unroll 1
+      for (int base = w0; base < w1; base += 2 * WSTEP) {
+        if (base + WSTEP < w1) wload(hb, base + WSTEP);
+        wemit(ha, base);
+        if (base + WSTEP >= w1) break;
+        if (base + 2 * WSTEP < w1) wload(ha, base + 2 * WSTEP);
+        wemit(hb, base + WSTEP);
       }
     }
     if (appender && tid == 0 && kh > 0) {                    // the appended key is the last key of this block's range
