@@ -248,7 +248,7 @@ fit_prep_kernel(const float* __restrict__ P, const float* __restrict__ v_star, f
 
 // Eight lanes share a row (16 channels and b/8 earlier bits each), so a warp works on four rows at once.
 template <typename KV, int JPL>          // JPL = b / 8 bits per lane
-__global__ void __launch_bounds__(kFitThreads)
+__global__ void __launch_bounds__(kFitThreads, 4)   // latency-bound: four blocks (32 warps) per SM
 fit_pass_kernel(const KV* __restrict__ k_cache, uint32_t* __restrict__ hfit, const float* __restrict__ dir,
                 const float* __restrict__ dots, float* __restrict__ partials, int32_t* __restrict__ agree,
                 const int32_t* __restrict__ unit_lens, int n_max, int row_stride, int it, int blocks_per_unit) {
@@ -259,8 +259,6 @@ fit_pass_kernel(const KV* __restrict__ k_cache, uint32_t* __restrict__ hfit, con
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sub = lane & 7, grp = lane >> 3;                  // lane within the row's group, row within the warp's four
   const int row0 = blockIdx.x * kFitRowsPerBlock;
-  __shared__ float red[kFitThreads / 32][BPC_D];
-  __shared__ int32_t redc[kFitThreads / 32][b];
   float dv[CPLN];
 #pragma unroll
   for (int c = 0; c < CPLN; ++c) dv[c] = dir[(size_t)unit * BPC_D + sub * CPLN + c];
@@ -287,26 +285,59 @@ fit_pass_kernel(const KV* __restrict__ k_cache, uint32_t* __restrict__ hfit, con
   uint32_t pl[6] = {0u, 0u, 0u, 0u, 0u, 0u};
   const int row_end = min(n, row0 + kFitRowsPerBlock);
   constexpr int ROWS_PER_ITER = (kFitThreads / 32) * 4;
-  for (int rb = row0; rb < row_end; rb += ROWS_PER_ITER) {   // uniform trip count: the shuffles below need whole warps
+  // Rows reach the lanes through a small ring in shared memory filled by asynchronous copies, NSTG - 1 row sets ahead
+  // (the pass is bound by memory latency).  Every lane copies and later reads only its own 16-byte pieces, so the ring
+  // needs no barrier.
+  constexpr int NV = CPLN * (int)sizeof(KV) / 16;            // 16-byte vectors per lane and row
+  constexpr int NSTG = sizeof(KV) == 2 ? 4 : 2;
+  __shared__ uint4 ring[NSTG][kFitThreads][NV];
+  __shared__ uint32_t ringw[NSTG][kFitThreads];
+  auto issue = [&](int slot, int rb) {
     const int r = rb + warp * 4 + grp;
-    const bool live = r < row_end;
-    const int rr = live ? r : row0;
-    const KV* kr = k_cache + ((size_t)unit * n_max + rr) * row_stride + sub * CPLN;
-    float x[CPLN];
-    if (sizeof(KV) == 2) {
-      const uint4 w0 = reinterpret_cast<const uint4*>(kr)[0], w1 = reinterpret_cast<const uint4*>(kr)[1];
-      const uint32_t ww[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+    if (r < row_end) {
+      const uint4* kr = reinterpret_cast<const uint4*>(k_cache + ((size_t)unit * n_max + r) * row_stride + sub * CPLN);
 #pragma unroll
-      for (int c = 0; c < 8; ++c) { x[2 * c] = __uint_as_float(ww[c] << 16); x[2 * c + 1] = __uint_as_float(ww[c] & 0xffff0000u); }
-    } else {
-#pragma unroll
-      for (int v = 0; v < 4; ++v) {
-        const float4 f = reinterpret_cast<const float4*>(kr)[v];
-        x[4 * v] = f.x; x[4 * v + 1] = f.y; x[4 * v + 2] = f.z; x[4 * v + 3] = f.w;
+      for (int v = 0; v < NV; ++v) {
+        const unsigned d = (unsigned)__cvta_generic_to_shared(&ring[slot][tid][v]);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(kr + v) : "memory");
+      }
+      if (it > 0) {
+        const unsigned d = (unsigned)__cvta_generic_to_shared(&ringw[slot][tid]);
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d), "l"(hfit + ((size_t)unit * n_max + r) * WORDS + my_word) : "memory");
       }
     }
-    uint32_t* hw = hfit + ((size_t)unit * n_max + rr) * WORDS;
-    const uint32_t mine = it > 0 ? (hw[my_word] >> my_shift) : 0u;                     // this lane's JPL earlier bits
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+#pragma unroll
+  for (int s0 = 0; s0 < NSTG - 1; ++s0) issue(s0, row0 + s0 * ROWS_PER_ITER);
+  int slot = 0;
+  for (int rb = row0; rb < row_end; rb += ROWS_PER_ITER) {   // uniform trip count: the shuffles below need whole warps
+    issue(slot == 0 ? NSTG - 1 : slot - 1, rb + (NSTG - 1) * ROWS_PER_ITER);
+    asm volatile("cp.async.wait_group %0;" ::"n"(NSTG - 1) : "memory");
+    const int r = rb + warp * 4 + grp;
+    const bool live = r < row_end;
+    float x[CPLN];
+    if (sizeof(KV) == 2) {
+#pragma unroll
+      for (int v = 0; v < NV; ++v) {
+        const uint4 q = ring[slot][tid][v];
+        const uint32_t ww[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) { x[8 * v + 2 * c] = __uint_as_float(ww[c] << 16); x[8 * v + 2 * c + 1] = __uint_as_float(ww[c] & 0xffff0000u); }
+      }
+    } else {
+#pragma unroll
+      for (int v = 0; v < NV; ++v) {
+        const uint4 q = ring[slot][tid][v];
+        x[4 * v] = __uint_as_float(q.x); x[4 * v + 1] = __uint_as_float(q.y); x[4 * v + 2] = __uint_as_float(q.z); x[4 * v + 3] = __uint_as_float(q.w);
+      }
+    }
+    if (!live) {                                             // nothing was copied for this lane: keep the arithmetic finite
+#pragma unroll
+      for (int c = 0; c < CPLN; ++c) x[c] = 0.f;
+    }
+    const uint32_t mine = (it > 0 && live) ? (ringw[slot][tid] >> my_shift) : 0u;       // this lane's JPL earlier bits
+    slot = slot + 1 == NSTG ? 0 : slot + 1;
     float tk = 0.f;
 #pragma unroll
     for (int c = 0; c < CPLN; ++c) tk = fmaf(x[c], dv[c], tk);
@@ -319,7 +350,7 @@ fit_pass_kernel(const KV* __restrict__ k_cache, uint32_t* __restrict__ hfit, con
     const bool pos = t >= 0.0;
     if (live) {
       if (sub == 0) {
-        uint32_t* w = hw + (it >> 5);
+        uint32_t* w = hfit + ((size_t)unit * n_max + r) * WORDS + (it >> 5);
         const uint32_t prev = (it & 31) ? *w : 0u;
         *w = prev | ((pos ? 1u : 0u) << (it & 31));
       }
@@ -335,6 +366,10 @@ fit_pass_kernel(const KV* __restrict__ k_cache, uint32_t* __restrict__ hfit, con
       }
     }
   }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();                                           // the ring is free: it now holds the block's partial sums
+  float (*red)[BPC_D] = reinterpret_cast<float (*)[BPC_D]>(&ring[0][0][0]);
+  int32_t (*redc)[b] = reinterpret_cast<int32_t (*)[b]>(reinterpret_cast<unsigned char*>(&ring[0][0][0]) + (kFitThreads / 32) * BPC_D * 4);
   // the four row groups of a warp hold partial sums for the same channels and bits
 #pragma unroll
   for (int c = 0; c < CPLN; ++c) {
