@@ -405,7 +405,55 @@ def run_ours(args):
     ee1.record()
     torch.cuda.synchronize()
     barrier()
-    ms_e2e = max_over_ranks(ee0.elapsed_time(ee1)) / K
+    ms_e2e_copy = max_over_ranks(ee0.elapsed_time(ee1)) / K
+
+    # Variant without copy nodes: the kernel reads q, k_new, v_new straight from the pinned host buffers and writes
+    # the output straight into pinned host memory (pinned allocations are device-accessible at their host address under
+    # unified addressing; checked below through the runtime before it is relied on).  Same bytes cross the bus per step.
+    ms_e2e_zc = None
+    try:
+        from cuda import cudart
+        def _device_visible(t):
+            err, attr = cudart.cudaPointerGetAttributes(t.data_ptr())
+            return int(err) == 0 and int(attr.devicePointer) == t.data_ptr()
+        zc = []
+        ok = True
+        for ly, (_, host_in, host_out) in zip(layers, e2e):
+            nq, nk = ly.q.numel(), ly.k_new.numel()
+            hq, hk, hv = host_in[:nq].view_as(ly.q), host_in[nq:nq + nk].view_as(ly.k_new), host_in[nq + nk:].view_as(ly.v_new)
+            ok = ok and all(_device_visible(t) for t in (host_in, host_out))
+            zc.append((hq, hk, hv, host_out))
+        if ok:
+            reset_after_warmup()
+            def zstep(i):
+                ly = layers[i % L]; hq, hk, hv, ho = zc[i % L]
+                ly.ctx.append_decode_attn(hk, hv, ly.k_cache, ly.v_cache, ly.codes, hq, budget_ppm=spec.budget_ppm, out=ho)
+            graphs = []
+            for i in range(L):
+                zstep(i); torch.cuda.synchronize()
+            reset_after_warmup()
+            layers[0].step(); torch.cuda.synchronize()          # same step with device-resident inputs: same bits expected
+            if not torch.equal(layers[0].out.cpu(), zc[0][3]):
+                raise RuntimeError("zero-copy step differs from the device-resident step")
+            reset_after_warmup()
+            for i in range(L):
+                graphs.append(_graph_of(lambda i=i: zstep(i)))
+            reset_after_warmup()
+            for s_ in range(min(W, 8)):
+                graphs[(W + s_) % L].replay(); torch.cuda.current_stream().synchronize()
+            reset_after_warmup()
+            barrier(); torch.cuda.synchronize()
+            z0, z1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            z0.record()
+            for s_ in range(K):
+                graphs[(W + s_) % L].replay()
+                torch.cuda.current_stream().synchronize()      # the step's result is in host memory
+            z1.record()
+            torch.cuda.synchronize(); barrier()
+            ms_e2e_zc = max_over_ranks(z0.elapsed_time(z1)) / K
+    except Exception as ex:                                      # no cuda-python, or pointers not device-visible
+        ms_e2e_zc = None
+    ms_e2e = ms_e2e_copy if ms_e2e_zc is None else min(ms_e2e_copy, ms_e2e_zc)
 
     # planted-needle recall of the selection (how many of the keys a query was built from are among the selected
     # ones); a property of the synthetic data and of hashing, reported for reference
@@ -441,7 +489,8 @@ def run_ours(args):
                    "kv_layout": "separate k/v arrays" if args.separate_kv else "interleaved k|v rows (row stride 2*head_dim)"},
         "clocks": clocks,
         "e2e": {"value": world * spec.batch / (ms_e2e * 1e-3), "unit": UNIT, "us_per_step": ms_e2e * 1e3,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "us_per_step_copy_nodes": ms_e2e_copy * 1e3, "us_per_step_zero_copy": None if ms_e2e_zc is None else ms_e2e_zc * 1e3},
         "gpu_launches": launches_per_region,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": achieved / peaks["hbm_gbs"], "of": peaks["source"],
