@@ -1142,9 +1142,10 @@ bpc_decode_kernel(const DecodeParams p) {
   BPC_STAMP(4);
 
   // ------------------------------------------------------------------ phase 3: gathered attention
+  // The list was written by other SMs during this launch: it is read at L2 (ld.global.cg), never through this SM's L1.
   auto row_index = [&](int qrow) -> int {                    // qrow in [0, nh + ne): cache row, or -1 for a duplicate
-    if (!EAS) return sel_u[lo + qrow];
-    return qrow < nh ? sel_u[lo + qrow] : sel_u[kh + e0 + (qrow - nh)];
+    if (!EAS) return __ldcg(sel_u + lo + qrow);
+    return qrow < nh ? __ldcg(sel_u + lo + qrow) : __ldcg(sel_u + kh + e0 + (qrow - nh));
   };
   const size_t rstride = (size_t)p.row_stride * sizeof(KV);   // bytes between consecutive cache rows
   const unsigned char* Ku = reinterpret_cast<const unsigned char*>(p.k_cache) + (size_t)unit * (size_t)p.n_max * rstride;
