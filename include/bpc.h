@@ -19,7 +19,8 @@
  *                          caches are separate arrays; 2*head_dim with v_cache = k_cache + head_dim for the
  *                          interleaved layout, where a token's K and V rows are adjacent in memory and one
  *                          gather touches 4*head_dim contiguous bytes instead of two separate rows)
- *       codes            : [batch][n_kv_heads][n_max][code_bits/64] uint64
+ *       codes            : [batch][n_kv_heads][n_max][code_bits/64] uint64 (code_bits/8 bytes per key; with
+ *                          32-bit codes one uint32 per key, the array still passed as uint64_t*)
  *                          bit j of a key (Algorithm 2 iteration j+1) is word j/64, bit j%64,
  *                          least significant first; 1 means the component is +1 (decision value >= 0)
  *       q                : [batch][n_q_heads][head_dim]            kv_dtype
@@ -28,7 +29,7 @@
  *       projection P     : [hash_sets][code_bits][head_dim]        float
  *     Query head hq belongs to KV head hq / (n_q_heads / n_kv_heads).  A "unit" is one
  *     (sequence, KV head) pair, unit = sequence * n_kv_heads + kv_head.
- *   - Limits: head_dim == 128; code_bits in {64,128,256}; n_q_heads a multiple of n_kv_heads with
+ *   - Limits: head_dim == 128; code_bits in {32,64,128,256}; n_q_heads a multiple of n_kv_heads with
  *     at most 8 query heads per KV head; n_max <= bpc_max_context(cfg).
  */
 #ifndef BPC_H_
