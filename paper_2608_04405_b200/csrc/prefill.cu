@@ -418,15 +418,45 @@ fit_reduce_kernel(const float* __restrict__ partials, const int32_t* __restrict_
   const int nblk = (n + kFitRowsPerBlock - 1) / kFitRowsPerBlock;
   __shared__ double corr[256];                               // u_i . u_j for j < it
   __shared__ double part[kRedGroups][BPC_D];
+  __shared__ int agp[kRedGroups][256];
+  // agreement counts: group q adds the blocks k = q, q + 4, ... (eight loads in flight per thread), then the groups are added
+  for (int j = c; j < it; j += BPC_D) {
+    int a8[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    int k = q;
+    for (; k + 7 * kRedGroups < nblk; k += 8 * kRedGroups) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) a8[e] += agree[((size_t)unit * blocks_per_unit + k + e * kRedGroups) * b + j];
+    }
+    for (; k < nblk; k += kRedGroups) a8[0] += agree[((size_t)unit * blocks_per_unit + k) * b + j];
+    agp[q][j] = ((a8[0] + a8[1]) + (a8[2] + a8[3])) + ((a8[4] + a8[5]) + (a8[6] + a8[7]));
+  }
+  __syncthreads();
   for (int j = threadIdx.x; j < it; j += BPC_D * kRedGroups) {
-    long long a = 0;
-    for (int k = 0; k < nblk; ++k) a += agree[((size_t)unit * blocks_per_unit + k) * b + j];
+    const long long a = (long long)agp[0][j] + agp[1][j] + agp[2][j] + agp[3][j];
     corr[j] = (double)(2 * a - (long long)n);
   }
   __syncthreads();
   double s = 0.0;
-  for (int k = q; k < nblk; k += kRedGroups) s += (double)partials[((size_t)unit * blocks_per_unit + k) * BPC_D + c];
-  for (int j = q; j < it; j += kRedGroups) s -= corr[j] * (double)P[((size_t)unit * b + j) * BPC_D + c];
+  {
+    double s8[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    int k = q;
+    for (; k + 7 * kRedGroups < nblk; k += 8 * kRedGroups) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) s8[e] += (double)partials[((size_t)unit * blocks_per_unit + k + e * kRedGroups) * BPC_D + c];
+    }
+    for (; k < nblk; k += kRedGroups) s8[0] += (double)partials[((size_t)unit * blocks_per_unit + k) * BPC_D + c];
+    s = ((s8[0] + s8[1]) + (s8[2] + s8[3])) + ((s8[4] + s8[5]) + (s8[6] + s8[7]));
+  }
+  {
+    double t8[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    int j = q;
+    for (; j + 7 * kRedGroups < it; j += 8 * kRedGroups) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) t8[e] += corr[j + e * kRedGroups] * (double)P[((size_t)unit * b + j + e * kRedGroups) * BPC_D + c];
+    }
+    for (; j < it; j += kRedGroups) t8[0] += corr[j] * (double)P[((size_t)unit * b + j) * BPC_D + c];
+    s -= ((t8[0] + t8[1]) + (t8[2] + t8[3])) + ((t8[4] + t8[5]) + (t8[6] + t8[7]));
+  }
   part[q][c] = s;
   __syncthreads();
   if (q == 0) {
