@@ -10,15 +10,16 @@
 // Phases of a cluster of CS blocks working on one unit with n cached keys:
 //   0  every block hashes the group's queries (identical arithmetic in all blocks)
 //   1  block r scans keys [r*chunk, (r+1)*chunk): 128-bit code loads, LOP3 (+ carry-save compression) and
-//      POPC score, 16-bit score key into shared memory, shared-memory histogram
-//   2  cluster barrier; histograms are summed through distributed shared memory; the threshold key T
-//      and the per-block output offsets follow; each block emits its selected indices in ascending
-//      order (score > T, then the lowest-index ties at T) into the unit's index list
+//      POPC score, 16-bit score key into shared memory, shared-memory histogram.  In a launch that also appends
+//      a key, the last warp of the block that owns the new key codes it (Algorithm 2) meanwhile.
+//   2  every block stores its histogram into its peers' shared memory; cluster barrier; the threshold key T
+//      and the per-block output offsets follow from one block scan; each block emits its selected indices in
+//      ascending order (score > T, then the lowest-index ties at T) into the unit's index list
 //   3  cluster barrier; block r runs online-softmax attention over rows [k*r/CS, k*(r+1)/CS) of the
-//      list.  Rows are gathered into a shared-memory ring with 16-byte asynchronous copies; bf16 caches
+//      list.  Rows are gathered into per-warp shared-memory rings with 16-byte asynchronous copies; bf16 caches
 //      use warp-level tensor-core MMAs (q K^T, then P V with P split in two bf16 halves), fp32 caches use
-//      fp64 arithmetic on the CUDA cores.  Partial (m, l, acc) are merged inside the block, then across
-//      the cluster through distributed shared memory.
+//      fp64 arithmetic on the CUDA cores.  Partial (m, l, acc) are merged inside the block, stored into the
+//      shared memory of the block that owns each output, and finished there after one more cluster barrier.
 // Scores and gathered rows never touch global memory.
 #pragma once
 #include <cooperative_groups.h>
