@@ -268,8 +268,14 @@ def run_ours(args):
         layers[s % L].step()
     torch.cuda.synchronize()
     if args.profile:                      # plain eager steps for a profiler to capture; no graphs, no other legs
+        if args.profile_leg == "weighted7":
+            for ly in layers:
+                ly.make_weighted_twin(B)
+            for s in range(W):
+                layers[s % L].step_weighted()
         for s in range(K):
-            layers[(W + s) % L].step()
+            ly = layers[(W + s) % L]
+            ly.step_weighted() if args.profile_leg == "weighted7" else ly.step()
         torch.cuda.synchronize()
         if rank == 0:
             print(json.dumps({"profile_run": True, "workload": spec.name, "steps": K, "warmup": W, "layer_replicas": L,
@@ -719,6 +725,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--separate-kv", action="store_true", help="separate K and V arrays instead of interleaved rows")
     ap.add_argument("--profile", action="store_true", help="warm-up plus K eager steps only (for ncu captures)")
+    ap.add_argument("--profile-leg", choices=("fused", "weighted7"), default="fused",
+                    help="with --profile: the fused step with Hamming scores (default) or with the weighted score")
     ap.add_argument("--sweep", action="store_true", help="second workload: latency over contexts and batch sizes, 64-bit codes, 1K/2K budgets")
     ap.add_argument("--quality", action="store_true", help="selection quality yard-sticks (recall vs exact top-k, cosine vs dense) for 32/64/128/256-bit codes")
     args = ap.parse_args()

@@ -203,10 +203,45 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&v);
 }
 
+// carry-save adder on 32 bit positions at once
+__device__ __forceinline__ void csa(uint32_t a, uint32_t b, uint32_t c, uint32_t& sum, uint32_t& carry) {
+  sum = a ^ b ^ c;
+  carry = (a & b) | (a & c) | (b & c);
+}
 // ---- score key of one code: sum over planes of weight * popc(agree & mask); agree = ~(h ^ sign)
 template <int W32, int NP>
 __device__ __forceinline__ int score_key(const uint32_t (&h)[W32], const uint32_t (&sg)[W32], const uint32_t (&mk)[NP][W32]) {
   int key = 0;
+  if constexpr (NP >= 4 && W32 >= 2) {
+    // Many planes (weighted scores): one population count per masked word would keep the 16-lane pipe busy for most
+    // of the scan.  A full adder per pair of masked words adds them to a carry word handed down from the plane below
+    // (a + b + c = (a ^ b ^ c) + 2 maj(a, b, c), bit by bit), which halves the counts: W32/2 per plane plus W32/2 for
+    // the last carries.  Each adder is three three-input logic operations, the masks included:
+    // t = a ^ c, s = b ^ t, maj(a, b, c) = c ^ (t & (b ^ c)) with b ^ c = s ^ t ^ c.
+    constexpr int C = W32 / 2;
+    uint32_t cy[C], x[W32];
+#pragma unroll
+    for (int f = 0; f < C; ++f) cy[f] = 0u;
+#pragma unroll
+    for (int w = 0; w < W32; ++w) x[w] = ~(h[w] ^ sg[w]);
+#pragma unroll
+    for (int pl = 0; pl < NP; ++pl) {
+      int c = 0;
+#pragma unroll
+      for (int f = 0; f < C; ++f) {
+        const uint32_t t = (x[2 * f] & mk[pl][2 * f]) ^ cy[f];
+        const uint32_t s = (x[2 * f + 1] & mk[pl][2 * f + 1]) ^ t;
+        cy[f] = cy[f] ^ (t & (s ^ t ^ cy[f]));
+        c += __popc(s);
+      }
+      key += c << pl;
+    }
+    int c = 0;
+#pragma unroll
+    for (int f = 0; f < C; ++f) c += __popc(cy[f]);
+    key += c << NP;
+    return key;
+  }
 #pragma unroll
   for (int pl = 0; pl < NP; ++pl) {
     int c = 0;
@@ -218,10 +253,6 @@ __device__ __forceinline__ int score_key(const uint32_t (&h)[W32], const uint32_
 }
 // 128-bit codes with two planes (weights 1 and 2): carry-save adders fold the eight masked words into five
 // before the population counts, which run on the 16-lane pipe
-__device__ __forceinline__ void csa(uint32_t a, uint32_t b, uint32_t c, uint32_t& sum, uint32_t& carry) {
-  sum = a ^ b ^ c;
-  carry = (a & b) | (a & c) | (b & c);
-}
 template <>
 __device__ __forceinline__ int score_key<4, 2>(const uint32_t (&h)[4], const uint32_t (&sg)[4], const uint32_t (&mk)[2][4]) {
   uint32_t x0[4], x1[4];
@@ -394,7 +425,9 @@ bpc_decode_kernel(const DecodeParams p) {
   const int c1s = appender ? c1 - 1 : c1;
   const uint32_t* cu = reinterpret_cast<const uint32_t*>(p.codes) + (size_t)unit * (size_t)p.n_max * W32;
   int32_t* dbg = p.dbg_scores != nullptr ? p.dbg_scores + (size_t)unit * p.n_max : nullptr;
-  constexpr int U = W32 <= 4 ? 8 : 4;                       // codes in flight per thread and buffer
+  // codes in flight per thread and buffer: the Hamming scan is bound by memory latency and wants many; the weighted
+  // scan is bound by its arithmetic and wants the registers for the plane masks instead
+  constexpr int U = MODE == 1 ? (W32 <= 2 ? 4 : 2) : (W32 <= 4 ? 8 : 4);
   auto load_code = [&](uint32_t (&h)[W32], int i) {
     const uint32_t* src = cu + (size_t)i * W32;
     if (W32 == 1) {
