@@ -218,8 +218,9 @@ bpc_status bpc_debug_set_buffers(bpc_ctx* ctx, int32_t* scores, int32_t* qweight
  * done.  stamps [units * cluster_size][16] uint64. */
 bpc_status bpc_debug_set_phase_timer(bpc_ctx* ctx, uint64_t* stamps);
 
-/* Launch geometry of the decode kernel: thread blocks per cluster (0 = choose automatically).
- * Returns BPC_ERR_UNSUPPORTED if n_max does not fit that many blocks. */
+/* Launch geometry of the decode kernel: thread blocks per cluster, any size from 1 to 16 that the device schedules
+ * (0 = choose automatically: the largest size that keeps all units' clusters resident at once).
+ * Returns BPC_ERR_UNSUPPORTED if n_max does not fit that many blocks or the device cannot schedule the size. */
 bpc_status bpc_set_cluster_size(bpc_ctx* ctx, int32_t cluster_size);
 int32_t    bpc_get_cluster_size(bpc_ctx* ctx);
 /* 1 when this context's decode calls use the streaming selection (units longer than a cluster's shared memory holds). */

@@ -89,27 +89,46 @@ int chunk_for(int n_max, int cs) {
   return fused > plain ? fused : plain;
 }
 
-// Smallest power-of-two cluster whose blocks can hold n_max scores; then grow it while all clusters of the grid
-// can still be resident at the same time (one wave) and a block keeps at least 1024 keys.
+// Cluster size of the decode launch.  Candidates run from the smallest cluster whose blocks can hold n_max scores to
+// the largest the device schedules, as long as a block keeps at least 1024 keys.  The phases of a block are bound by
+// what one SM can have in flight, so more SMs per unit win until the grid no longer fits the device at once.  The
+// estimate, in units of "time to scan one code", is
+//   (waves of resident clusters) x (keys per block + 600 per block of the cluster for the merges across blocks
+//                                   + 4000 per eight-row attention tile of a warp + 20 000 for hash and selection),
+// with the attention tiles counted for a nominal budget of 2 % of n_max, at least 1024 keys (the budget itself is an
+// argument of each call); the cheapest candidate is taken.  Measured on B200: 8 units pick 8 blocks at 32K keys and
+// 10 at 128K; 16 units pick 6, 24 units 5, 40 units 3 at 128K.
 int choose_cluster(const bpc_ctx* ctx, int chunk_cap, int max_cluster) {
-  int cs = 1, li = 0;
-  while (cs <= max_cluster && chunk_for(ctx->cfg.n_max, cs) > chunk_cap) { cs *= 2; ++li; }
+  int cs = 1;
+  while (cs <= max_cluster && (ctx->max_active[cs] < 1 || chunk_for(ctx->cfg.n_max, cs) > chunk_cap)) ++cs;
   if (cs > max_cluster) return 0;
-  while (cs * 2 <= max_cluster && ctx->units <= ctx->max_active[li + 1] && chunk_for(ctx->cfg.n_max, cs * 2) >= 1024) {
-    cs *= 2;
-    ++li;
+  long long k_nom = ((long long)ctx->cfg.n_max * 20000 + 999999) / 1000000;
+  if (k_nom < 1024) k_nom = 1024;
+  if (k_nom > ctx->cfg.n_max) k_nom = ctx->cfg.n_max;
+  int best = cs;
+  long long best_cost = -1;
+  for (int c = cs; c <= max_cluster; ++c) {
+    if (ctx->max_active[c] < 1) continue;
+    const int chunk = chunk_for(ctx->cfg.n_max, c);
+    if (c > cs && chunk < 1024) break;
+    const long long waves = (ctx->units + ctx->max_active[c] - 1) / ctx->max_active[c];
+    const long long rows_per_warp = ((k_nom + c - 1) / c + 15) / 16;
+    const long long tiles = (rows_per_warp + 7) / 8;
+    const long long cost = waves * (chunk + 600LL * c + 4000LL * tiles + 20000LL);
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = c; }
   }
-  return cs;
+  return best;
 }
 
 }  // namespace
 
 cudaError_t bpc_plan_decode_geometry(bpc_ctx* ctx) {
-  int mc[6] = {1, 0, 0, 0, 0, 0}, cap = 0;
+  int mc[BPC_MAX_CLUSTER + 1] = {1}, cap = 0;
   cudaError_t e = decode_limits(ctx, 0, mc, &cap, nullptr);
   if (e != cudaSuccess) return e;
   ctx->max_cluster = mc[0];
-  for (int i = 0; i < 5; ++i) ctx->max_active[i] = mc[1 + i];
+  ctx->max_active[0] = 0;
+  for (int i = 1; i <= BPC_MAX_CLUSTER; ++i) ctx->max_active[i] = mc[i];
   ctx->chunk_cap_limit = cap;
   ctx->cluster_size = choose_cluster(ctx, cap, ctx->max_cluster);
   ctx->streaming = false;
@@ -119,11 +138,8 @@ cudaError_t bpc_plan_decode_geometry(bpc_ctx* ctx) {
     // Units too long for the largest cluster's shared memory: no score is stored, the codes are read twice.  The
     // largest cluster size that still runs all units in one wave is used (at least the largest schedulable one).
     int cs = forced && ctx->cluster_size > 0 ? ctx->cluster_size : ctx->max_cluster;
-    if (!(forced && ctx->cluster_size > 0)) {
-      int li = 0;
-      for (int c = 1; c < ctx->max_cluster; c *= 2) ++li;
-      while (cs > 1 && ctx->units > ctx->max_active[li]) { cs /= 2; --li; }
-    }
+    if (!(forced && ctx->cluster_size > 0))
+      while (cs > 1 && ctx->units > ctx->max_active[cs]) --cs;
     ctx->cluster_size = cs;
     ctx->streaming = true;
   }
@@ -231,7 +247,7 @@ bpc_status bpc_set_cluster_size(bpc_ctx* ctx, int32_t cs) {
   const int cap = ctx->chunk_cap_limit, mc = ctx->max_cluster;
   if (cs == 0 && ctx->streaming) return BPC_OK;            // keeps the size chosen at creation
   if (cs == 0) cs = choose_cluster(ctx, cap, mc);
-  if (cs < 1 || cs > mc || (cs & (cs - 1)) != 0) return BPC_ERR_UNSUPPORTED;
+  if (cs < 1 || cs > mc || ctx->max_active[cs] < 1) return BPC_ERR_UNSUPPORTED;
   if (!ctx->streaming && chunk_for(ctx->cfg.n_max, cs) > cap) return BPC_ERR_UNSUPPORTED;
   ctx->cluster_size = cs;
   return BPC_OK;

@@ -31,7 +31,7 @@ struct bpc_ctx {
   int row_stride;           // cache elements between consecutive rows
   int cluster_size;         // decode: thread blocks per cluster
   int max_cluster;          // largest cluster size the device schedules for the decode kernel
-  int max_active[5];        // clusters of size 1, 2, 4, 8, 16 that can be resident at once
+  int max_active[BPC_MAX_CLUSTER + 1];   // [cs]: clusters of size cs that can be resident at once (0 = not schedulable)
   int sm_count;
   bool fitted;
   bool use_pdl;             // launch the decode kernel with programmatic stream serialization

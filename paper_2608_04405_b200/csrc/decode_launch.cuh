@@ -2,6 +2,8 @@
 #pragma once
 #include "decode_kernel.cuh"
 
+#include <atomic>
+
 namespace bpcdev {
 
 // The shared-memory ceiling is always raised to the device's opt-in maximum, so contexts with different
@@ -51,8 +53,8 @@ static cudaError_t launch_one(bpc_ctx* ctx, const DecodeParams& p_in, cudaStream
   return cudaLaunchKernelEx(&lc, bpc_decode_kernel<KV, GP, W32, MODE, EAS>, p);
 }
 
-// Largest cluster size (power of two) the device can schedule with a full-size block, and the number of
-// score keys one block can hold next to a two-stage gather ring.
+// Largest cluster size the device can schedule with a full-size block, and the number of score keys one block can
+// hold next to a two-stage gather ring.
 template <typename KV, int GP, int W32, int MODE, int EAS>
 static cudaError_t limits_one(const bpc_ctx* ctx, int nbins, int* max_cluster, int* chunk_cap, size_t* smem_bytes) {
   typedef DecodeSmem<KV, GP, W32> L;
@@ -67,12 +69,21 @@ static cudaError_t limits_one(const bpc_ctx* ctx, int nbins, int* max_cluster, i
   if (chunk_cap) *chunk_cap = cap;
   if (smem_bytes) *smem_bytes = (size_t)optin;
   if (max_cluster) {
-    // max_cluster[0] = largest schedulable cluster size; max_cluster[1 + log2(cs)] = clusters of that size that
-    // can be resident at once (a grid with more clusters than that runs in several waves)
+    // max_cluster[0] = largest schedulable cluster size; max_cluster[cs] = clusters of size cs that can be resident
+    // at once (a grid with more clusters than that runs in several waves), cs = 1 .. BPC_MAX_CLUSTER
+    // The answers depend on the kernel and the device only: they are kept per instantiation for the first device
+    // asked about (published with a release store once complete), so that contexts and the allocation-free entry
+    // point do not repeat the sixteen occupancy queries.
+    static std::atomic<int> cached_dev(-1);
+    static int cached[BPC_MAX_CLUSTER + 1];
+    if (cached_dev.load(std::memory_order_acquire) == dev) {
+      for (int i = 0; i <= BPC_MAX_CLUSTER; ++i) max_cluster[i] = cached[i];
+      return cudaSuccess;
+    }
     int best = 1;
     e = configure_kernel<KV, GP, W32, MODE, EAS>(dev);
     if (e != cudaSuccess) return e;
-    for (int cs = 1, li = 0; cs <= BPC_MAX_CLUSTER; cs *= 2, ++li) {
+    for (int cs = 1; cs <= BPC_MAX_CLUSTER; ++cs) {
       cudaLaunchConfig_t lc = {};
       lc.gridDim = dim3((unsigned)cs, 1, 1);
       lc.blockDim = dim3(L::NT, 1, 1);
@@ -84,10 +95,15 @@ static cudaError_t limits_one(const bpc_ctx* ctx, int nbins, int* max_cluster, i
       int nclusters = 0;
       cudaError_t q = cudaOccupancyMaxActiveClusters(&nclusters, bpc_decode_kernel<KV, GP, W32, MODE, EAS>, &lc);
       if (q != cudaSuccess) { (void)cudaGetLastError(); nclusters = 0; }
-      max_cluster[1 + li] = nclusters;
+      max_cluster[cs] = nclusters;
       if (nclusters >= 1) best = cs;
     }
     max_cluster[0] = best;
+    static std::atomic<int> claimed(0);
+    if (claimed.exchange(1) == 0) {                           // the first caller publishes
+      for (int i = 0; i <= BPC_MAX_CLUSTER; ++i) cached[i] = max_cluster[i];
+      cached_dev.store(dev, std::memory_order_release);
+    }
   }
   return cudaSuccess;
 }

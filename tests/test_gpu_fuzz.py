@@ -31,7 +31,7 @@ def _cases(n_cases, seed):
         ragged = rng.random() < 0.5
         mode = rng.choice([0, 0, 0, 1])
         eas = rng.choice([0, 0, 3000]) if mode == 0 else 0
-        cluster = rng.choice([0, 0, 1, 2, 4])
+        cluster = rng.choice([0, 0, 1, 2, 3, 4, 6])
         budget = rng.choice([("ppm", 20000), ("ppm", 1000), ("ppm", 300000), ("count", 1), ("count", 37), ("ppm", 1000000)])
         interleaved = rng.random() < 0.5
         stream = mode == 0 and eas == 0 and rng.random() < 0.3      # streaming selection forced on a shape that would fit

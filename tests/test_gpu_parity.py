@@ -43,7 +43,7 @@ def test_cfg0_tiny_fp32_all_stages():
     print(rep)
 
 
-@pytest.mark.parametrize("cluster", [1, 2, 4, 8])
+@pytest.mark.parametrize("cluster", [1, 2, 3, 4, 5, 6, 7, 8, 9, 12, 16])
 def test_cluster_sizes_agree_with_checker(cluster):
     """Ragged length (several tiles plus a tail) at every cluster size, GQA 4, bf16, 128-bit codes."""
     H = _harness()
@@ -420,11 +420,12 @@ def test_quality_yardsticks(dtype, bits, group, n):
     print(rep)
 
 
-@pytest.mark.parametrize("n_ctx,batch", [(262144, 1), (32768, 16)])
+@pytest.mark.parametrize("n_ctx,batch", [(262144, 1), (32768, 16), (131072, 3)])
 def test_sweep_shapes_single_word_codes_fixed_budgets(n_ctx, batch):
     """The second bench workload's shapes (Section 4 "Setup" / latency-vs-context study: 64-bit codes, budgets of 1024
-    and 2048 keys) at full size in the launch geometry the sweep times: long context at batch 1 (cluster size 8) and
-    short context at batch 16 (cluster size 1); sampled units, plain and fused steps."""
+    and 2048 keys) at full size in the launch geometry the sweep times: long context at batch 1 (cluster size 10),
+    short context at batch 16 (cluster size 1), and a batch that is not a power of two (24 units, cluster size 5);
+    sampled units, plain and fused steps."""
     H = _harness()
     spec = CONFIGS[1].scaled(name="sweep", wid=40 + batch, batch=batch, n_ctx=n_ctx, code_bits=64, steps=2)
     sess = H.Session(spec, gen_device="cuda", interleaved=True)
