@@ -222,6 +222,15 @@ bpc_status bpc_debug_set_phase_timer(bpc_ctx* ctx, uint64_t* stamps);
  * (0 = choose automatically: the largest size that keeps all units' clusters resident at once).
  * Returns BPC_ERR_UNSUPPORTED if n_max does not fit that many blocks or the device cannot schedule the size. */
 bpc_status bpc_set_cluster_size(bpc_ctx* ctx, int32_t cluster_size);
+/* The automatic choice as a pure host function (no device is touched): the cluster size bpc_create would take for
+ * `cfg` on a device whose limits are given by the caller.  max_active (host, 17 entries) holds at index c = 1 .. 16 how
+ * many clusters of c blocks the device keeps resident at once (0 = size not schedulable; entry 0 is ignored);
+ * chunk_cap = score keys one block's shared memory holds.  Candidates are the sizes whose blocks hold n_max scores
+ * and, above the smallest such size, keep at least 1024 keys per block; the result minimises
+ * waves x (keys per block + 600 x size + 4000 x eight-row attention tiles per warp at a nominal budget of
+ * max(2 % of n_max, 1024) + 20000), waves = ceil(units / max_active[size]).  Returns 0 when no size fits (the
+ * streaming selection then applies) or an argument is invalid. */
+int32_t    bpc_plan_cluster_size(const bpc_config* cfg, const int32_t* max_active, int32_t chunk_cap);
 int32_t    bpc_get_cluster_size(bpc_ctx* ctx);
 /* 1 when this context's decode calls use the streaming selection (units longer than a cluster's shared memory holds). */
 int32_t    bpc_uses_streaming(bpc_ctx* ctx);

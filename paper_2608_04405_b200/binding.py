@@ -67,6 +67,7 @@ def _load() -> ctypes.CDLL:
         "bpc_debug_set_buffers": (i32, [vp, vp, vp]),
         "bpc_debug_set_phase_timer": (i32, [vp, vp]),
         "bpc_set_cluster_size": (i32, [vp, i32]),
+        "bpc_plan_cluster_size": (i32, [cfgp, ctypes.POINTER(i32), i32]),
         "bpc_get_cluster_size": (i32, [vp]),
         "bpc_uses_streaming": (i32, [vp]),
         "bpc_last_device_error": (i32, [vp, ctypes.POINTER(i32), vp]),
@@ -87,7 +88,7 @@ EXPORTS = ["bpc_create", "bpc_destroy", "bpc_codes_bytes", "bpc_fit_workspace_by
            "bpc_set_seq_lens", "bpc_get_seq_lens", "bpc_fit", "bpc_set_projection", "bpc_get_projection",
            "bpc_encode_keys", "bpc_build_eas", "bpc_get_eas", "bpc_eas_capacity", "bpc_exact_topk", "bpc_append", "bpc_decode_attn", "bpc_append_decode_attn", "bpc_decode_attn_static", "bpc_static_scratch_entries",
            "bpc_debug_set_buffers", "bpc_debug_set_phase_timer",
-           "bpc_set_cluster_size",
+           "bpc_set_cluster_size", "bpc_plan_cluster_size",
            "bpc_get_cluster_size", "bpc_uses_streaming", "bpc_last_device_error", "bpc_last_cuda_error", "bpc_launch_count", "bpc_version"]
 
 
@@ -126,6 +127,13 @@ def make_config(batch: int, n_q_heads: int, n_kv_heads: int, n_max: int, code_bi
     return bpc_config(batch, n_q_heads, n_kv_heads, head_dim, code_bits, n_max,
                       BPC_BF16 if dtype == torch.bfloat16 else BPC_F32, score_mode, sm_scale,
                       n_kv_heads if shared_projection else batch * n_kv_heads, 1 if residual_correction else 0, kv_row_stride, eas_ppm, fit_power_iters)
+
+
+def plan_cluster_size(cfg: bpc_config, max_active, chunk_cap: int) -> int:
+    """bpc_plan_cluster_size: the automatic cluster size for `cfg` on a device with the given limits (max_active[c] =
+    resident clusters of c blocks, c = 1 .. 16; entry 0 ignored).  Pure host arithmetic."""
+    arr = (ctypes.c_int32 * 17)(*[int(v) for v in max_active])
+    return int(lib.bpc_plan_cluster_size(ctypes.byref(cfg), arr, int(chunk_cap)))
 
 
 class Context:

@@ -253,6 +253,22 @@ bpc_status bpc_set_cluster_size(bpc_ctx* ctx, int32_t cs) {
   return BPC_OK;
 }
 
+int32_t bpc_plan_cluster_size(const bpc_config* cfg, const int32_t* max_active, int32_t chunk_cap) {
+  if (check_cfg(cfg) != BPC_OK || max_active == nullptr || chunk_cap < 0) return 0;
+  bpc_ctx tmp;
+  memset(&tmp, 0, sizeof(tmp));
+  tmp.cfg = *cfg;
+  tmp.units = cfg->batch * cfg->n_kv_heads;
+  tmp.group = cfg->n_q_heads / cfg->n_kv_heads;
+  int mc = 0;
+  for (int c = 1; c <= BPC_MAX_CLUSTER; ++c) {
+    tmp.max_active[c] = max_active[c] > 0 ? max_active[c] : 0;
+    if (tmp.max_active[c] > 0) mc = c;
+  }
+  if (mc == 0) return 0;
+  return choose_cluster(&tmp, chunk_cap, mc);
+}
+
 int32_t bpc_get_cluster_size(bpc_ctx* ctx) { return ctx ? ctx->cluster_size : 0; }
 int32_t bpc_uses_streaming(bpc_ctx* ctx) { return (ctx && ctx->streaming) ? 1 : 0; }
 

@@ -3,6 +3,9 @@ import ctypes
 import os
 import re
 
+import pytest
+import torch
+
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
@@ -50,3 +53,47 @@ def test_product_path_does_not_import_the_checker():
         if f.endswith(".py"):
             txt = open(os.path.join(ROOT, "oracle", f)).read()
             assert "paper_2608_04405_b200" not in txt and "ctypes" not in txt
+
+
+def _binding():
+    from paper_2608_04405_b200 import binding as B
+    return B
+
+
+def _b200_like_limits():
+    """Resident clusters per size as a 148-SM part answers them: one block per SM, a cluster stays inside one GPC, GPCs of
+    unequal size (this split reproduces the counts seen on a B200: 74 clusters of 2, 7 of 12 to 16, fewer than 16 of 8)."""
+    gpcs = [10, 18, 20, 20, 20, 20, 20, 20]
+    return [0] + [sum(g // c for g in gpcs) for c in range(1, 17)]
+
+
+@pytest.mark.parametrize("batch,n_kv,n_max,want", [
+    (1, 8, 131072 + 256, 10),      # 8 units: the largest size with all clusters resident (12+ hold only 7)
+    (4, 8, 131072 + 256, 4),       # 32 units: 5 blocks each would need two waves
+    (2, 8, 131072 + 256, 6),       # 16 units: 6 x 16 = 96 blocks in one wave, 8 x 16 would not be resident
+    (5, 8, 131072 + 256, 3),       # 40 units
+    (16, 8, 65536 + 64, 1),        # 128 units: one block each
+    (1, 8, 1048576 + 64, 16),      # needs >= 13 blocks per unit; two waves either way, the smaller blocks win
+    (1, 8, 4096, 4),               # a block keeps at least 1024 keys
+])
+def test_cluster_size_plan_on_given_device_limits(batch, n_kv, n_max, want):
+    """The automatic cluster choice is host arithmetic over the device's occupancy answers: checked here on a table
+    shaped like a 148-SM part, without a GPU."""
+    B = _binding()
+    cfg = B.make_config(batch, 4 * n_kv, n_kv, n_max, 128, torch.bfloat16)
+    got = B.plan_cluster_size(cfg, _b200_like_limits(), 87000)
+    assert got == want, (got, want)
+
+
+def test_cluster_size_plan_edge_cases():
+    B = _binding()
+    cfg = B.make_config(1, 8, 8, 131072, 128, torch.bfloat16)
+    ma = _b200_like_limits()
+    assert B.plan_cluster_size(cfg, [0] * 17, 87000) == 0                 # nothing schedulable
+    assert B.plan_cluster_size(cfg, ma, 1024) == 0                         # n_max fits no cluster: streaming applies
+    only_pow2 = [v if c in (1, 2, 4, 8, 16) else 0 for c, v in enumerate(ma)]
+    assert B.plan_cluster_size(cfg, only_pow2, 87000) == 8                 # sizes the device refuses are never chosen
+    small = B.make_config(1, 8, 8, 1500, 128, torch.bfloat16)
+    assert B.plan_cluster_size(small, ma, 87000) == 1                      # short contexts stay in one block
+    got = B.plan_cluster_size(cfg, ma, 20000)                              # 131072 keys need >= 7 blocks of 20000
+    assert got >= 7 and ma[got] >= 8
