@@ -287,8 +287,17 @@ cudaError_t launch(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStrea
   cudaError_t e = cudaFuncSetAttribute(encode_tc_kernel<NBITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const int tiles_max = (c.n_max + kTileKeys - 1) / kTileKeys;
-  int bpu = (2 * ctx->sm_count + ctx->units - 1) / ctx->units;    // about two waves of blocks over all units
+  // Blocks per unit.  One block fits an SM (shared memory), so the grid runs in waves of sm_count blocks and a last,
+  // partly filled wave costs as much as a full one: starting from about four waves, take the first count whose last
+  // wave is at least 90 % full (32 units on 148 SMs: 23 blocks per unit = 736 blocks = 4.97 waves; the 10 used before
+  // gave 2.16 waves, i.e. three rounds for two rounds' worth of work).
+  int bpu = (4 * ctx->sm_count + ctx->units - 1) / ctx->units;
   if (bpu < 1) bpu = 1;
+  for (int tries = 0; tries < 16; ++tries) {
+    const int rem = (int)(((long long)ctx->units * bpu) % ctx->sm_count);
+    if (rem == 0 || rem * 10 >= ctx->sm_count * 9) break;
+    ++bpu;
+  }
   if (bpu > tiles_max) bpu = tiles_max;
   const dim3 grid(bpu, ctx->units);
   encode_tc_kernel<NBITS><<<grid, kThreads, smem, stream>>>(
