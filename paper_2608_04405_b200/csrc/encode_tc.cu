@@ -4,11 +4,13 @@
 // channels x bits).  It runs on the 5th-generation tensor cores: per block, tiles of 128 keys (M = 128) against
 // the unit's b projection rows (N = b, 64 or 128) over the 128 channels (eight tcgen05.mma steps of K = 16), bf16
 // operands in shared memory in the 128-byte-swizzled K-major layout, fp32 accumulator in tensor memory with one
-// key per TMEM lane.  Each of the 128 threads then pulls its key's b decision values out of tensor memory
-// (tcgen05.ld) into registers and runs the greedy sweep of Algorithm 2 in its Gram form
+// key per TMEM lane.  Each of the 128 threads of a warpgroup then pulls its key's b decision values out of tensor
+// memory (tcgen05.ld) into registers and runs the greedy sweep of Algorithm 2 in its Gram form
 //     u_i = sign(t_i);  t_j -= u_i * G_ij  (j > i),   G = P_h P_h^T,
 // which equals updating the residual r <- r - u_i P_i and testing r . P_{i+1}.  While the threads sweep tile i,
-// the asynchronous copies and the MMA of tile i+1 are already in flight.
+// the asynchronous copies and the MMA of tile i+1 are already in flight.  A block holds two such warpgroups, which
+// share the projection rows and the Gram matrix in shared memory and otherwise run independent pipelines: the sweep
+// is a chain of dependent FMAs per thread, and one warp per scheduler cannot keep the FP32 pipe busy.
 //
 // Waits on the MMA-completion mbarrier are bounded: on expiry the block raises the device error word, still
 // releases its tensor memory and returns.
@@ -18,7 +20,9 @@
 namespace {
 
 constexpr int kTileKeys = 128;
-constexpr int kThreads = 128;
+constexpr int kGroupThreads = 128;   // one warpgroup sweeps one key tile (a TMEM lane per thread)
+constexpr int kGroups = 2;           // warpgroups per block, each with its own tiles, accumulator columns and barrier
+constexpr int kThreads = kGroupThreads * kGroups;
 
 __device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
 
@@ -27,6 +31,8 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+// barrier among the 128 threads of one warpgroup (hardware barriers 1 and 2; 0 is __syncthreads)
+__device__ __forceinline__ void group_sync(int g) { asm volatile("bar.sync %0, %1;" ::"r"(1 + g), "r"(kGroupThreads) : "memory"); }
 
 // Shared-memory operand descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t umma_desc_sw128(const void* smem_ptr) {
@@ -119,27 +125,29 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   constexpr int A_BYTES = kTileKeys * 256;                 // one key tile (128 rows x 128 bf16)
   constexpr int B_BYTES = NBITS * 256;                     // the projection rows
-  unsigned char* a_s[2] = {smem, smem + A_BYTES};
-  unsigned char* b_s = smem + 2 * A_BYTES;
-  float* g_s = reinterpret_cast<float*>(smem + 2 * A_BYTES + B_BYTES);   // [NBITS][NBITS]
-  __shared__ unsigned long long mma_bar;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int grp = tid / kGroupThreads, gtid = tid % kGroupThreads;   // warpgroup and thread within it
+  unsigned char* a_s[2] = {smem + (size_t)(2 * grp) * A_BYTES, smem + (size_t)(2 * grp + 1) * A_BYTES};
+  unsigned char* b_s = smem + 2 * kGroups * A_BYTES;
+  float* g_s = reinterpret_cast<float*>(smem + 2 * kGroups * A_BYTES + B_BYTES);   // [NBITS][NBITS]
+  __shared__ unsigned long long mma_bar_s[kGroups];
   __shared__ uint32_t tmem_base_s;
-  __shared__ int timed_out_s;
+  __shared__ int timed_out_g[kGroups];
+  unsigned long long* mma_bar = &mma_bar_s[grp];
+  constexpr int kTmemCols = kGroups * NBITS < 32 ? 32 : kGroups * NBITS;   // a power of two >= 32
 
   const int unit = blockIdx.y;
-  const int tid = threadIdx.x, warp = tid >> 5;
   const int n = min(unit_lens[unit], n_max);
   const int ntiles = (n + kTileKeys - 1) / kTileKeys;
   const int set = shared_sets ? unit % n_kv_heads : unit;
 
   // ---- one-time set-up: barrier, tensor memory, projection and Gram matrix in shared memory
   if (tid == 0) {
-    mbar_init(&mma_bar, 1);
-    timed_out_s = 0;
+    for (int g = 0; g < kGroups; ++g) { mbar_init(&mma_bar_s[g], 1); timed_out_g[g] = 0; }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(NBITS < 32 ? 32 : NBITS) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   {
@@ -154,7 +162,8 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const uint32_t tmem_base = tmem_base_s;
+  const uint32_t tmem_all = tmem_base_s;
+  const uint32_t tmem_base = tmem_all + (uint32_t)(grp * NBITS);   // this warpgroup's accumulator columns
   float trace_g = 0.f;
   if (key_err != nullptr)
     for (int i = 0; i < NBITS; ++i) trace_g += g_s[i * NBITS + i];
@@ -162,7 +171,7 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
   const unsigned char* kbase = reinterpret_cast<const unsigned char*>(k_cache) + (size_t)unit * n_max * (size_t)row_stride * 2;
   auto load_tile = [&](int tile, unsigned char* dst) {
     const int r0 = tile * kTileKeys;
-    for (int c = tid; c < kTileKeys * 16; c += kThreads) {
+    for (int c = gtid; c < kTileKeys * 16; c += kGroupThreads) {
       const int r = c >> 4, ch = c & 15;
       unsigned char* d = dst + sw128_offset(kTileKeys, r, ch);
       if (r0 + r < n) cp_async16(d, kbase + (size_t)(r0 + r) * row_stride * 2 + ch * 16);
@@ -178,30 +187,34 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
       const size_t boff = (size_t)(ks >> 2) * (NBITS * 128) + (size_t)(ks & 3) * 32;
       umma_bf16(tmem_base, umma_desc_sw128(a_tile + aoff), umma_desc_sw128(b_s + boff), idesc, ks > 0 ? 1u : 0u);
     }
-    umma_commit(&mma_bar);
+    umma_commit(mma_bar);
   };
 
-  // tiles of this block: blockIdx.x, blockIdx.x + blocks_per_unit, ...
-  int tile = blockIdx.x;
+  // Tiles of this warpgroup: kGroups * blockIdx.x + grp, then every kGroups * blocks_per_unit-th.  The two warpgroups
+  // run independent pipelines (own tiles, own accumulator columns, own MMA barrier, own hardware barrier), so that
+  // eight warps instead of four keep the FP32 pipe busy during the sweeps; all threads of a warpgroup take the same
+  // branches, so its barrier is always reached by all 128 of them.
+  const int tile_step = kGroups * blocks_per_unit;
+  int tile = kGroups * blockIdx.x + grp;
   int it = 0;
   if (tile < ntiles) {
     load_tile(tile, a_s[0]);
     cp_async_wait_all();
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the tensor core
-    __syncthreads();
-    if (tid == 0) {
+    group_sync(grp);
+    if (gtid == 0) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       issue_mma(a_s[0]);
     }
   }
-  for (; tile < ntiles; tile += blocks_per_unit, ++it) {
-    const int next = tile + blocks_per_unit;
+  for (; tile < ntiles; tile += tile_step, ++it) {
+    const int next = tile + tile_step;
     if (next < ntiles) load_tile(next, a_s[(it + 1) & 1]);  // overlaps the MMA and the sweep of this tile
     // decision values of this tile: wait for the MMA, then one TMEM lane (key) per thread
-    bool ok = mbar_wait(&mma_bar, (unsigned)(it & 1));
-    if (!ok) timed_out_s = 1;
+    bool ok = mbar_wait(mma_bar, (unsigned)(it & 1));
+    if (!ok) timed_out_g[grp] = 1;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t taddr = tmem_base + ((uint32_t)(32 * warp) << 16);
+    const uint32_t taddr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);   // a warp reaches the lanes of its quarter
     // Column blocks of 32 bits: pull the block out of tensor memory, apply the corrections of all earlier
     // bits (t_j -= u_i G_ij, G rows are broadcast reads from shared memory), then sweep the block itself.
     uint32_t words[NBITS / 32];
@@ -237,13 +250,13 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
     // squared reconstruction error (Eq. 8) from the sweep: ||k - hP||^2 = ||k||^2 - 2 sum|t_i| + trace(G).  The key's
     // channels are read from this tile's operand buffer before the barrier below: after it, other threads refill
     // that buffer with the tile after next.
-    const int key = tile * kTileKeys + tid;
+    const int key = tile * kTileKeys + gtid;
     float k2 = 0.f;
     if (key_err != nullptr && key < n) {
       const unsigned char* arow = a_s[it & 1];
 #pragma unroll
       for (int ch = 0; ch < 16; ++ch) {
-        const uint4 w = *reinterpret_cast<const uint4*>(arow + sw128_offset(kTileKeys, tid, ch));
+        const uint4 w = *reinterpret_cast<const uint4*>(arow + sw128_offset(kTileKeys, gtid, ch));
         const float f0 = bf16_lo(w.x), f1 = bf16_hi(w.x), f2 = bf16_lo(w.y), f3 = bf16_hi(w.y);
         const float f4 = bf16_lo(w.z), f5 = bf16_hi(w.z), f6 = bf16_lo(w.w), f7 = bf16_hi(w.w);
         k2 += (f0 * f0 + f1 * f1) + (f2 * f2 + f3 * f3) + (f4 * f4 + f5 * f5) + (f6 * f6 + f7 * f7);
@@ -254,9 +267,9 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
       cp_async_wait_all();
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    __syncthreads();                                         // TMEM has been read by everyone; next tile has landed
-    if (timed_out_s) break;
-    if (next < ntiles && tid == 0) {
+    group_sync(grp);                                         // the accumulator has been read by the whole warpgroup; its next tile has landed
+    if (timed_out_g[grp]) break;                             // (written only by this warpgroup, before the barrier)
+    if (next < ntiles && gtid == 0) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       issue_mma(a_s[(it + 1) & 1]);
     }
@@ -271,22 +284,22 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
       }
     }
   }
-  if (timed_out_s && tid == 0) atomicOr(err, BPC_DEVERR_TIMEOUT);
+  if (timed_out_g[grp] && gtid == 0) atomicOr(err, BPC_DEVERR_TIMEOUT);
   cp_async_wait_all();
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
+  __syncthreads();                                           // both warpgroups are done with tensor memory
   if (warp == 0) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(NBITS < 32 ? 32 : NBITS) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_all), "r"(kTmemCols) : "memory");
   }
 }
 
 template <int NBITS>
 cudaError_t launch(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStream_t stream) {
   const bpc_config& c = ctx->cfg;
-  const size_t smem = 2 * kTileKeys * 256 + (size_t)NBITS * 256 + (size_t)NBITS * NBITS * 4 + 1024;
+  const size_t smem = (size_t)2 * kGroups * kTileKeys * 256 + (size_t)NBITS * 256 + (size_t)NBITS * NBITS * 4 + 1024;
   cudaError_t e = cudaFuncSetAttribute(encode_tc_kernel<NBITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  const int tiles_max = (c.n_max + kTileKeys - 1) / kTileKeys;
+  const int tiles_max = ((c.n_max + kTileKeys - 1) / kTileKeys + kGroups - 1) / kGroups;   // a block takes kGroups tiles at a time
   // Blocks per unit.  One block fits an SM (shared memory), so the grid runs in waves of sm_count blocks and a last,
   // partly filled wave costs as much as a full one: starting from about four waves, take the first count whose last
   // wave is at least 90 % full (32 units on 148 SMs: 23 blocks per unit = 736 blocks = 4.97 waves; the 10 used before
