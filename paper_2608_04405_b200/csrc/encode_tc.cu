@@ -8,7 +8,7 @@
 // memory (tcgen05.ld) into registers and runs the greedy sweep of Algorithm 2 in its Gram form
 //     u_i = sign(t_i);  t_j -= u_i * G_ij  (j > i),   G = P_h P_h^T,
 // which equals updating the residual r <- r - u_i P_i and testing r . P_{i+1}.  While the threads sweep tile i,
-// the asynchronous copies and the MMA of tile i+1 are already in flight.  A block holds two such warpgroups, which
+// the asynchronous copy of tile i+1 is already in flight.  A block holds three such warpgroups, which
 // share the projection rows and the Gram matrix in shared memory and otherwise run independent pipelines: the sweep
 // is a chain of dependent FMAs per thread, and one warp per scheduler cannot keep the FP32 pipe busy.
 //
@@ -21,7 +21,7 @@ namespace {
 
 constexpr int kTileKeys = 128;
 constexpr int kGroupThreads = 128;   // one warpgroup sweeps one key tile (a TMEM lane per thread)
-constexpr int kGroups = 2;           // warpgroups per block, each with its own tiles, accumulator columns and barrier
+constexpr int kGroups = 4;           // warpgroups per block, each with its own tiles, accumulator columns and barrier
 constexpr int kThreads = kGroupThreads * kGroups;
 
 __device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
@@ -31,7 +31,7 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
-// barrier among the 128 threads of one warpgroup (hardware barriers 1 and 2; 0 is __syncthreads)
+// barrier among the 128 threads of one warpgroup (hardware barriers 1 .. kGroups; 0 is __syncthreads)
 __device__ __forceinline__ void group_sync(int g) { asm volatile("bar.sync %0, %1;" ::"r"(1 + g), "r"(kGroupThreads) : "memory"); }
 
 // Shared-memory operand descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
@@ -127,14 +127,15 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
   constexpr int B_BYTES = NBITS * 256;                     // the projection rows
   const int tid = threadIdx.x, warp = tid >> 5;
   const int grp = tid / kGroupThreads, gtid = tid % kGroupThreads;   // warpgroup and thread within it
-  unsigned char* a_s[2] = {smem + (size_t)(2 * grp) * A_BYTES, smem + (size_t)(2 * grp + 1) * A_BYTES};
-  unsigned char* b_s = smem + 2 * kGroups * A_BYTES;
-  float* g_s = reinterpret_cast<float*>(smem + 2 * kGroups * A_BYTES + B_BYTES);   // [NBITS][NBITS]
+  unsigned char* a_t = smem + (size_t)grp * A_BYTES;       // this warpgroup's key tile (one buffer: see the loop)
+  unsigned char* b_s = smem + kGroups * A_BYTES;
+  float* g_s = reinterpret_cast<float*>(smem + kGroups * A_BYTES + B_BYTES);   // [NBITS][NBITS]
   __shared__ unsigned long long mma_bar_s[kGroups];
   __shared__ uint32_t tmem_base_s;
   __shared__ int timed_out_g[kGroups];
   unsigned long long* mma_bar = &mma_bar_s[grp];
-  constexpr int kTmemCols = kGroups * NBITS < 32 ? 32 : kGroups * NBITS;   // a power of two >= 32
+  constexpr int kTmemCols = kGroups * NBITS <= 32 ? 32 : kGroups * NBITS <= 64 ? 64 : kGroups * NBITS <= 128 ? 128 : kGroups * NBITS <= 256 ? 256 : 512;   // a power of two >= 32
+  static_assert(kGroups * NBITS <= 512, "accumulators exceed tensor memory");
 
   const int unit = blockIdx.y;
   const int n = min(unit_lens[unit], n_max);
@@ -190,30 +191,47 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
     umma_commit(mma_bar);
   };
 
-  // Tiles of this warpgroup: kGroups * blockIdx.x + grp, then every kGroups * blocks_per_unit-th.  The two warpgroups
+  // Tiles of this warpgroup: kGroups * blockIdx.x + grp, then every kGroups * blocks_per_unit-th.  The warpgroups
   // run independent pipelines (own tiles, own accumulator columns, own MMA barrier, own hardware barrier), so that
-  // eight warps instead of four keep the FP32 pipe busy during the sweeps; all threads of a warpgroup take the same
+  // twelve warps instead of four keep the FP32 pipe busy during the sweeps; all threads of a warpgroup take the same
   // branches, so its barrier is always reached by all 128 of them.
   const int tile_step = kGroups * blocks_per_unit;
   int tile = kGroups * blockIdx.x + grp;
   int it = 0;
   if (tile < ntiles) {
-    load_tile(tile, a_s[0]);
+    load_tile(tile, a_t);
     cp_async_wait_all();
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the tensor core
     group_sync(grp);
     if (gtid == 0) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      issue_mma(a_s[0]);
+      issue_mma(a_t);
     }
   }
   for (; tile < ntiles; tile += tile_step, ++it) {
     const int next = tile + tile_step;
-    if (next < ntiles) load_tile(next, a_s[(it + 1) & 1]);  // overlaps the MMA and the sweep of this tile
     // decision values of this tile: wait for the MMA, then one TMEM lane (key) per thread
     bool ok = mbar_wait(mma_bar, (unsigned)(it & 1));
     if (!ok) timed_out_g[grp] = 1;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    // The MMA is the only reader of the key tile (besides the key norms below), and it has completed: the buffer is
+    // refilled with the warpgroup's next tile right away, under the sweep, which is many times longer than the copy.
+    // One buffer per warpgroup instead of two leaves room for a third warpgroup.
+    const int key = tile * kTileKeys + gtid;
+    float k2 = 0.f;
+    if (key_err != nullptr) {                                // squared norm of this thread's key, from the operand tile
+      if (key < n) {
+#pragma unroll
+        for (int ch = 0; ch < 16; ++ch) {
+          const uint4 w = *reinterpret_cast<const uint4*>(a_t + sw128_offset(kTileKeys, gtid, ch));
+          const float f0 = bf16_lo(w.x), f1 = bf16_hi(w.x), f2 = bf16_lo(w.y), f3 = bf16_hi(w.y);
+          const float f4 = bf16_lo(w.z), f5 = bf16_hi(w.z), f6 = bf16_lo(w.w), f7 = bf16_hi(w.w);
+          k2 += (f0 * f0 + f1 * f1) + (f2 * f2 + f3 * f3) + (f4 * f4 + f5 * f5) + (f6 * f6 + f7 * f7);
+        }
+      }
+      group_sync(grp);                                       // every thread has read its row before the refill starts
+    }
+    if (next < ntiles) load_tile(next, a_t);
     const uint32_t taddr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);   // a warp reaches the lanes of its quarter
     // Column blocks of 32 bits: pull the block out of tensor memory, apply the corrections of all earlier
     // bits (t_j -= u_i G_ij, G rows are broadcast reads from shared memory), then sweep the block itself.
@@ -247,21 +265,7 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
       DiagSweep<0>::run(t, word, abs_sum, g_s + (size_t)(32 * cb) * NBITS + 32 * cb, NBITS, residual_correction);
       words[cb] = word;
     }
-    // squared reconstruction error (Eq. 8) from the sweep: ||k - hP||^2 = ||k||^2 - 2 sum|t_i| + trace(G).  The key's
-    // channels are read from this tile's operand buffer before the barrier below: after it, other threads refill
-    // that buffer with the tile after next.
-    const int key = tile * kTileKeys + gtid;
-    float k2 = 0.f;
-    if (key_err != nullptr && key < n) {
-      const unsigned char* arow = a_s[it & 1];
-#pragma unroll
-      for (int ch = 0; ch < 16; ++ch) {
-        const uint4 w = *reinterpret_cast<const uint4*>(arow + sw128_offset(kTileKeys, gtid, ch));
-        const float f0 = bf16_lo(w.x), f1 = bf16_hi(w.x), f2 = bf16_lo(w.y), f3 = bf16_hi(w.y);
-        const float f4 = bf16_lo(w.z), f5 = bf16_hi(w.z), f6 = bf16_lo(w.w), f7 = bf16_hi(w.w);
-        k2 += (f0 * f0 + f1 * f1) + (f2 * f2 + f3 * f3) + (f4 * f4 + f5 * f5) + (f6 * f6 + f7 * f7);
-      }
-    }
+    // squared reconstruction error (Eq. 8) from the sweep: ||k - hP||^2 = ||k||^2 - 2 sum|t_i| + trace(G), stored below
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     if (next < ntiles) {
       cp_async_wait_all();
@@ -271,7 +275,7 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
     if (timed_out_g[grp]) break;                             // (written only by this warpgroup, before the barrier)
     if (next < ntiles && gtid == 0) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      issue_mma(a_s[(it + 1) & 1]);
+      issue_mma(a_t);
     }
     if (key_err != nullptr && key < n) key_err[(size_t)unit * n_max + key] = fmaxf(0.f, k2 - 2.f * abs_sum + trace_g);
     if (key < n) {
@@ -296,7 +300,7 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
 template <int NBITS>
 cudaError_t launch(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStream_t stream) {
   const bpc_config& c = ctx->cfg;
-  const size_t smem = (size_t)2 * kGroups * kTileKeys * 256 + (size_t)NBITS * 256 + (size_t)NBITS * NBITS * 4 + 1024;
+  const size_t smem = (size_t)kGroups * kTileKeys * 256 + (size_t)NBITS * 256 + (size_t)NBITS * NBITS * 4 + 1024;
   cudaError_t e = cudaFuncSetAttribute(encode_tc_kernel<NBITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const int tiles_max = ((c.n_max + kTileKeys - 1) / kTileKeys + kGroups - 1) / kGroups;   // a block takes kGroups tiles at a time
