@@ -8,9 +8,11 @@
 // memory (tcgen05.ld) into registers and runs the greedy sweep of Algorithm 2 in its Gram form
 //     u_i = sign(t_i);  t_j -= u_i * G_ij  (j > i),   G = P_h P_h^T,
 // which equals updating the residual r <- r - u_i P_i and testing r . P_{i+1}.  While the threads sweep tile i,
-// the asynchronous copy of tile i+1 is already in flight.  A block holds three such warpgroups, which
-// share the projection rows and the Gram matrix in shared memory and otherwise run independent pipelines: the sweep
-// is a chain of dependent FMAs per thread, and one warp per scheduler cannot keep the FP32 pipe busy.
+// the asynchronous copy of tile i+1 is already in flight.  A block holds two such warpgroups, which share the
+// projection rows and the Gram matrix in shared memory and otherwise run independent pipelines, and every warpgroup
+// works on two key tiles at once, one key of each per thread: the sweep is a chain of dependent FMAs per key fed by
+// broadcast reads of the Gram matrix, so one warp per scheduler cannot keep the FP32 pipe busy, and with one key per
+// thread the shared-memory reads (one 16-byte read per four FMAs) bound it.
 //
 // Waits on the MMA-completion mbarrier are bounded: on expiry the block raises the device error word, still
 // releases its tensor memory and returns.
@@ -21,7 +23,9 @@ namespace {
 
 constexpr int kTileKeys = 128;
 constexpr int kGroupThreads = 128;   // one warpgroup sweeps one key tile (a TMEM lane per thread)
-constexpr int kGroups = 4;           // warpgroups per block, each with its own tiles, accumulator columns and barrier
+constexpr int kGroups = 2;           // warpgroups per block, each with its own tiles, accumulator columns and barrier
+constexpr int kPair = 2;             // key tiles a warpgroup sweeps together, one key of each per thread: every Gram
+                                     // value read from shared memory then feeds two FMAs (the loads bound the sweep)
 constexpr int kThreads = kGroupThreads * kGroups;
 
 __device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
@@ -86,26 +90,36 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[N]) {
   for (int i = 0; i < 32; ++i) v[OFF + i] = __uint_as_float(r[i]);
 }
 
-// Greedy sweep of one 32-bit column block held in registers (every index a compile-time constant).
-// On entry t[j] already carries the corrections of all earlier blocks; on exit `word` holds the 32 signs.
+// Greedy sweep of one 32-bit column block held in registers (every index a compile-time constant), for the kPair
+// keys of a thread at once.  On entry t[q][j] already carries the corrections of all earlier blocks; on exit word[q]
+// holds the 32 signs of key q.  Each key sees exactly the operations of a sweep on its own.
 template <int I>
 struct DiagSweep {
-  static __device__ __forceinline__ void run(float (&t)[32], uint32_t& word, float& abs_sum, const float* g_diag, int ld, int rc) {
-    const bool pos = t[I] >= 0.f;
-    word |= (pos ? 1u : 0u) << I;
-    abs_sum += fabsf(t[I]);
+  static __device__ __forceinline__ void run(float (&t)[kPair][32], uint32_t (&word)[kPair], float (&abs_sum)[kPair],
+                                             const float* g_diag, int ld, int rc) {
+    float u[kPair];
+#pragma unroll
+    for (int q = 0; q < kPair; ++q) {
+      const bool pos = t[q][I] >= 0.f;
+      word[q] |= (pos ? 1u : 0u) << I;
+      abs_sum[q] += fabsf(t[q][I]);
+      u[q] = pos ? 1.f : -1.f;
+    }
     if (rc) {
-      const float u = pos ? 1.f : -1.f;
       const float* gi = g_diag + I * ld;
 #pragma unroll
-      for (int j = I + 1; j < 32; ++j) t[j] = fmaf(-u, gi[j], t[j]);
+      for (int j = I + 1; j < 32; ++j) {
+        const float g = gi[j];
+#pragma unroll
+        for (int q = 0; q < kPair; ++q) t[q][j] = fmaf(-u[q], g, t[q][j]);
+      }
     }
     DiagSweep<I + 1>::run(t, word, abs_sum, g_diag, ld, rc);
   }
 };
 template <>
 struct DiagSweep<32> {
-  static __device__ __forceinline__ void run(float (&)[32], uint32_t&, float&, const float*, int, int) {}
+  static __device__ __forceinline__ void run(float (&)[kPair][32], uint32_t (&)[kPair], float (&)[kPair], const float*, int, int) {}
 };
 
 // byte offset of 16-byte chunk `ch` (0..15) of row `r` inside a [rows x 128 channels] bf16 operand tile:
@@ -127,15 +141,16 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
   constexpr int B_BYTES = NBITS * 256;                     // the projection rows
   const int tid = threadIdx.x, warp = tid >> 5;
   const int grp = tid / kGroupThreads, gtid = tid % kGroupThreads;   // warpgroup and thread within it
-  unsigned char* a_t = smem + (size_t)grp * A_BYTES;       // this warpgroup's key tile (one buffer: see the loop)
-  unsigned char* b_s = smem + kGroups * A_BYTES;
-  float* g_s = reinterpret_cast<float*>(smem + kGroups * A_BYTES + B_BYTES);   // [NBITS][NBITS]
+  unsigned char* a_t = smem + (size_t)(grp * kPair) * A_BYTES;   // this warpgroup's kPair key tiles (one buffer each: see the loop)
+  unsigned char* b_s = smem + kGroups * kPair * A_BYTES;
+  float* g_s = reinterpret_cast<float*>(smem + kGroups * kPair * A_BYTES + B_BYTES);   // [NBITS][NBITS]
   __shared__ unsigned long long mma_bar_s[kGroups];
   __shared__ uint32_t tmem_base_s;
   __shared__ int timed_out_g[kGroups];
   unsigned long long* mma_bar = &mma_bar_s[grp];
-  constexpr int kTmemCols = kGroups * NBITS <= 32 ? 32 : kGroups * NBITS <= 64 ? 64 : kGroups * NBITS <= 128 ? 128 : kGroups * NBITS <= 256 ? 256 : 512;   // a power of two >= 32
-  static_assert(kGroups * NBITS <= 512, "accumulators exceed tensor memory");
+  constexpr int kAccCols = kGroups * kPair * NBITS;        // fp32 accumulator columns of all tiles in flight
+  constexpr int kTmemCols = kAccCols <= 32 ? 32 : kAccCols <= 64 ? 64 : kAccCols <= 128 ? 128 : kAccCols <= 256 ? 256 : 512;   // a power of two >= 32
+  static_assert(kAccCols <= 512, "accumulators exceed tensor memory");
 
   const int unit = blockIdx.y;
   const int n = min(unit_lens[unit], n_max);
@@ -164,7 +179,7 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_all = tmem_base_s;
-  const uint32_t tmem_base = tmem_all + (uint32_t)(grp * NBITS);   // this warpgroup's accumulator columns
+  const uint32_t tmem_base = tmem_all + (uint32_t)(grp * kPair * NBITS);   // this warpgroup's accumulator columns (tile q at + q * NBITS)
   float trace_g = 0.f;
   if (key_err != nullptr)
     for (int i = 0; i < NBITS; ++i) trace_g += g_s[i * NBITS + i];
@@ -181,110 +196,135 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
     cp_async_commit();
   };
   const uint32_t idesc = umma_idesc_bf16(kTileKeys, NBITS);
-  auto issue_mma = [&](const unsigned char* a_tile) {       // one thread: 8 steps of K = 16 over the 128 channels
+  auto issue_mma = [&]() {                                  // one thread: per tile 8 steps of K = 16 over the 128 channels
 #pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {
-      const size_t aoff = (size_t)(ks >> 2) * (kTileKeys * 128) + (size_t)(ks & 3) * 32;
-      const size_t boff = (size_t)(ks >> 2) * (NBITS * 128) + (size_t)(ks & 3) * 32;
-      umma_bf16(tmem_base, umma_desc_sw128(a_tile + aoff), umma_desc_sw128(b_s + boff), idesc, ks > 0 ? 1u : 0u);
+    for (int q = 0; q < kPair; ++q) {
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        const size_t aoff = (size_t)q * A_BYTES + (size_t)(ks >> 2) * (kTileKeys * 128) + (size_t)(ks & 3) * 32;
+        const size_t boff = (size_t)(ks >> 2) * (NBITS * 128) + (size_t)(ks & 3) * 32;
+        umma_bf16(tmem_base + (uint32_t)(q * NBITS), umma_desc_sw128(a_t + aoff), umma_desc_sw128(b_s + boff), idesc, ks > 0 ? 1u : 0u);
+      }
     }
-    umma_commit(mma_bar);
+    umma_commit(mma_bar);                                    // arrives when all MMAs issued so far have completed
+  };
+  auto load_pair = [&](int pr) {                             // tiles kPair * pr + q; rows past n are zero-filled
+#pragma unroll
+    for (int q = 0; q < kPair; ++q) load_tile(kPair * pr + q, a_t + (size_t)q * A_BYTES);
   };
 
-  // Tiles of this warpgroup: kGroups * blockIdx.x + grp, then every kGroups * blocks_per_unit-th.  The warpgroups
-  // run independent pipelines (own tiles, own accumulator columns, own MMA barrier, own hardware barrier), so that
-  // twelve warps instead of four keep the FP32 pipe busy during the sweeps; all threads of a warpgroup take the same
-  // branches, so its barrier is always reached by all 128 of them.
-  const int tile_step = kGroups * blocks_per_unit;
-  int tile = kGroups * blockIdx.x + grp;
+  // Tile pairs of this warpgroup: kGroups * blockIdx.x + grp, then every kGroups * blocks_per_unit-th.  The warpgroups
+  // run independent pipelines (own tiles, own accumulator columns, own MMA barrier, own hardware barrier); all threads
+  // of a warpgroup take the same branches, so its barrier is always reached by all 128 of them.
+  const int npairs = (ntiles + kPair - 1) / kPair;
+  const int pair_step = kGroups * blocks_per_unit;
+  int pr = kGroups * blockIdx.x + grp;
   int it = 0;
-  if (tile < ntiles) {
-    load_tile(tile, a_t);
+  if (pr < npairs) {
+    load_pair(pr);
     cp_async_wait_all();
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the tensor core
     group_sync(grp);
     if (gtid == 0) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      issue_mma(a_t);
+      issue_mma();
     }
   }
-  for (; tile < ntiles; tile += tile_step, ++it) {
-    const int next = tile + tile_step;
-    // decision values of this tile: wait for the MMA, then one TMEM lane (key) per thread
+  for (; pr < npairs; pr += pair_step, ++it) {
+    const int next = pr + pair_step;
+    // decision values of these tiles: wait for the MMAs, then one TMEM lane (one key of each tile) per thread
     bool ok = mbar_wait(mma_bar, (unsigned)(it & 1));
     if (!ok) timed_out_g[grp] = 1;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    // The MMA is the only reader of the key tile (besides the key norms below), and it has completed: the buffer is
-    // refilled with the warpgroup's next tile right away, under the sweep, which is many times longer than the copy.
-    // One buffer per warpgroup instead of two leaves room for a third warpgroup.
-    const int key = tile * kTileKeys + gtid;
-    float k2 = 0.f;
-    if (key_err != nullptr) {                                // squared norm of this thread's key, from the operand tile
-      if (key < n) {
+    // The MMAs are the only readers of the key tiles (besides the key norms below), and they have completed: the
+    // buffers are refilled with the warpgroup's next tiles right away, under the sweep, which is many times longer
+    // than the copy.
+    int key[kPair];
+    float k2[kPair];
 #pragma unroll
-        for (int ch = 0; ch < 16; ++ch) {
-          const uint4 w = *reinterpret_cast<const uint4*>(a_t + sw128_offset(kTileKeys, gtid, ch));
-          const float f0 = bf16_lo(w.x), f1 = bf16_hi(w.x), f2 = bf16_lo(w.y), f3 = bf16_hi(w.y);
-          const float f4 = bf16_lo(w.z), f5 = bf16_hi(w.z), f6 = bf16_lo(w.w), f7 = bf16_hi(w.w);
-          k2 += (f0 * f0 + f1 * f1) + (f2 * f2 + f3 * f3) + (f4 * f4 + f5 * f5) + (f6 * f6 + f7 * f7);
+    for (int q = 0; q < kPair; ++q) { key[q] = (kPair * pr + q) * kTileKeys + gtid; k2[q] = 0.f; }
+    if (key_err != nullptr) {                                // squared norms of this thread's keys, from the operand tiles
+#pragma unroll
+      for (int q = 0; q < kPair; ++q) {
+        if (key[q] < n) {
+#pragma unroll
+          for (int ch = 0; ch < 16; ++ch) {
+            const uint4 w = *reinterpret_cast<const uint4*>(a_t + (size_t)q * A_BYTES + sw128_offset(kTileKeys, gtid, ch));
+            const float f0 = bf16_lo(w.x), f1 = bf16_hi(w.x), f2 = bf16_lo(w.y), f3 = bf16_hi(w.y);
+            const float f4 = bf16_lo(w.z), f5 = bf16_hi(w.z), f6 = bf16_lo(w.w), f7 = bf16_hi(w.w);
+            k2[q] += (f0 * f0 + f1 * f1) + (f2 * f2 + f3 * f3) + (f4 * f4 + f5 * f5) + (f6 * f6 + f7 * f7);
+          }
         }
       }
-      group_sync(grp);                                       // every thread has read its row before the refill starts
+      group_sync(grp);                                       // every thread has read its rows before the refill starts
     }
-    if (next < ntiles) load_tile(next, a_t);
+    if (next < npairs) load_pair(next);
     const uint32_t taddr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);   // a warp reaches the lanes of its quarter
     // Column blocks of 32 bits: pull the block out of tensor memory, apply the corrections of all earlier
     // bits (t_j -= u_i G_ij, G rows are broadcast reads from shared memory), then sweep the block itself.
-    uint32_t words[NBITS / 32];
-    float abs_sum = 0.f;                                     // sum of |t_i| at decision time (for Eq. 8)
+    uint32_t words[kPair][NBITS / 32];
+    float abs_sum[kPair];                                    // sum of |t_i| at decision time (for Eq. 8)
+#pragma unroll
+    for (int q = 0; q < kPair; ++q) abs_sum[q] = 0.f;
 #pragma unroll
     for (int cb = 0; cb < NBITS / 32; ++cb) {
-      float t[32];
-      tmem_ld32<0>(taddr + 32 * cb, t);
+      float t[kPair][32];
+#pragma unroll
+      for (int q = 0; q < kPair; ++q) tmem_ld32<0>(taddr + (uint32_t)(q * NBITS + 32 * cb), t[q]);
       asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
       if (residual_correction) {
 #pragma unroll
         for (int pb = 0; pb < cb; ++pb) {
-          const uint32_t bits = words[pb];
 #pragma unroll 4
           for (int i = 0; i < 32; ++i) {
-            const float u = ((bits >> i) & 1u) ? 1.f : -1.f;
+            float mu[kPair];                                 // minus the sign of bit 32 pb + i
+#pragma unroll
+            for (int q = 0; q < kPair; ++q) mu[q] = ((words[q][pb] >> i) & 1u) ? -1.f : 1.f;
             const float4* gi = reinterpret_cast<const float4*>(g_s + (size_t)(32 * pb + i) * NBITS + 32 * cb);
 #pragma unroll
             for (int j4 = 0; j4 < 8; ++j4) {
               const float4 gv = gi[j4];
-              t[4 * j4] = fmaf(-u, gv.x, t[4 * j4]);
-              t[4 * j4 + 1] = fmaf(-u, gv.y, t[4 * j4 + 1]);
-              t[4 * j4 + 2] = fmaf(-u, gv.z, t[4 * j4 + 2]);
-              t[4 * j4 + 3] = fmaf(-u, gv.w, t[4 * j4 + 3]);
+#pragma unroll
+              for (int q = 0; q < kPair; ++q) {
+                t[q][4 * j4] = fmaf(mu[q], gv.x, t[q][4 * j4]);
+                t[q][4 * j4 + 1] = fmaf(mu[q], gv.y, t[q][4 * j4 + 1]);
+                t[q][4 * j4 + 2] = fmaf(mu[q], gv.z, t[q][4 * j4 + 2]);
+                t[q][4 * j4 + 3] = fmaf(mu[q], gv.w, t[q][4 * j4 + 3]);
+              }
             }
           }
         }
       }
-      uint32_t word = 0u;
+      uint32_t word[kPair];
+#pragma unroll
+      for (int q = 0; q < kPair; ++q) word[q] = 0u;
       DiagSweep<0>::run(t, word, abs_sum, g_s + (size_t)(32 * cb) * NBITS + 32 * cb, NBITS, residual_correction);
-      words[cb] = word;
+#pragma unroll
+      for (int q = 0; q < kPair; ++q) words[q][cb] = word[q];
     }
-    // squared reconstruction error (Eq. 8) from the sweep: ||k - hP||^2 = ||k||^2 - 2 sum|t_i| + trace(G), stored below
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    if (next < ntiles) {
+    if (next < npairs) {
       cp_async_wait_all();
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    group_sync(grp);                                         // the accumulator has been read by the whole warpgroup; its next tile has landed
+    group_sync(grp);                                         // the accumulators have been read by the whole warpgroup; its next tiles have landed
     if (timed_out_g[grp]) break;                             // (written only by this warpgroup, before the barrier)
-    if (next < ntiles && gtid == 0) {
+    if (next < npairs && gtid == 0) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      issue_mma(a_t);
+      issue_mma();
     }
-    if (key_err != nullptr && key < n) key_err[(size_t)unit * n_max + key] = fmaxf(0.f, k2 - 2.f * abs_sum + trace_g);
-    if (key < n) {
-      uint32_t* dst = reinterpret_cast<uint32_t*>(codes + ((size_t)unit * n_max + key) * (NBITS / 64));
-      if (NBITS == 64) {
-        *reinterpret_cast<uint2*>(dst) = make_uint2(words[0], words[1]);
-      } else {
 #pragma unroll
-        for (int w = 0; w < NBITS / 32; w += 4) *reinterpret_cast<uint4*>(dst + w) = make_uint4(words[w], words[w + 1], words[w + 2], words[w + 3]);
+    for (int q = 0; q < kPair; ++q) {
+      // squared reconstruction error (Eq. 8) from the sweep: ||k - hP||^2 = ||k||^2 - 2 sum|t_i| + trace(G)
+      if (key_err != nullptr && key[q] < n) key_err[(size_t)unit * n_max + key[q]] = fmaxf(0.f, k2[q] - 2.f * abs_sum[q] + trace_g);
+      if (key[q] < n) {
+        uint32_t* dst = reinterpret_cast<uint32_t*>(codes + ((size_t)unit * n_max + key[q]) * (NBITS / 64));
+        if (NBITS == 64) {
+          *reinterpret_cast<uint2*>(dst) = make_uint2(words[q][0], words[q][1]);
+        } else {
+#pragma unroll
+          for (int w = 0; w < NBITS / 32; w += 4) *reinterpret_cast<uint4*>(dst + w) = make_uint4(words[q][w], words[q][w + 1], words[q][w + 2], words[q][w + 3]);
+        }
       }
     }
   }
@@ -300,10 +340,10 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
 template <int NBITS>
 cudaError_t launch(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStream_t stream) {
   const bpc_config& c = ctx->cfg;
-  const size_t smem = (size_t)kGroups * kTileKeys * 256 + (size_t)NBITS * 256 + (size_t)NBITS * NBITS * 4 + 1024;
+  const size_t smem = (size_t)kGroups * kPair * kTileKeys * 256 + (size_t)NBITS * 256 + (size_t)NBITS * NBITS * 4 + 1024;
   cudaError_t e = cudaFuncSetAttribute(encode_tc_kernel<NBITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  const int tiles_max = ((c.n_max + kTileKeys - 1) / kTileKeys + kGroups - 1) / kGroups;   // a block takes kGroups tiles at a time
+  const int tiles_max = ((c.n_max + kTileKeys - 1) / kTileKeys + kGroups * kPair - 1) / (kGroups * kPair);   // a block takes kGroups * kPair tiles at a time
   // Blocks per unit.  One block fits an SM (shared memory), so the grid runs in waves of sm_count blocks and a last,
   // partly filled wave costs as much as a full one: starting from about four waves, take the first count whose last
   // wave is at least 90 % full (32 units on 148 SMs: 23 blocks per unit = 736 blocks = 4.97 waves; the 10 used before
