@@ -265,21 +265,32 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
     uint32_t words[kPair][NBITS / 32];
     float abs_sum[kPair];                                    // sum of |t_i| at decision time (for Eq. 8)
 #pragma unroll
-    for (int q = 0; q < kPair; ++q) abs_sum[q] = 0.f;
+    for (int q = 0; q < kPair; ++q) {
+      abs_sum[q] = 0.f;
 #pragma unroll
+      for (int w = 0; w < NBITS / 32; ++w) words[q][w] = 0u;
+    }
+#pragma unroll 1
     for (int cb = 0; cb < NBITS / 32; ++cb) {
       float t[kPair][32];
 #pragma unroll
       for (int q = 0; q < kPair; ++q) tmem_ld32<0>(taddr + (uint32_t)(q * NBITS + 32 * cb), t[q]);
       asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
       if (residual_correction) {
-#pragma unroll
+#pragma unroll 1
         for (int pb = 0; pb < cb; ++pb) {
+          uint32_t wprev[kPair];                             // words[q][pb], selected without indexing registers
+#pragma unroll
+          for (int q = 0; q < kPair; ++q) {
+            wprev[q] = words[q][0];
+#pragma unroll
+            for (int w = 1; w < NBITS / 32; ++w) wprev[q] = pb == w ? words[q][w] : wprev[q];
+          }
 #pragma unroll 4
           for (int i = 0; i < 32; ++i) {
             float mu[kPair];                                 // minus the sign of bit 32 pb + i
 #pragma unroll
-            for (int q = 0; q < kPair; ++q) mu[q] = ((words[q][pb] >> i) & 1u) ? -1.f : 1.f;
+            for (int q = 0; q < kPair; ++q) mu[q] = ((wprev[q] >> i) & 1u) ? -1.f : 1.f;
             const float4* gi = reinterpret_cast<const float4*>(g_s + (size_t)(32 * pb + i) * NBITS + 32 * cb);
 #pragma unroll
             for (int j4 = 0; j4 < 8; ++j4) {
@@ -300,7 +311,10 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
       for (int q = 0; q < kPair; ++q) word[q] = 0u;
       DiagSweep<0>::run(t, word, abs_sum, g_s + (size_t)(32 * cb) * NBITS + 32 * cb, NBITS, residual_correction);
 #pragma unroll
-      for (int q = 0; q < kPair; ++q) words[q][cb] = word[q];
+      for (int q = 0; q < kPair; ++q) {
+#pragma unroll
+        for (int w = 0; w < NBITS / 32; ++w) words[q][w] = cb == w ? word[q] : words[q][w];
+      }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     if (next < npairs) {
