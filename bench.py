@@ -528,7 +528,7 @@ def run_ours(args):
 
 # ----------------------------------------------------------------------------- paper-scale sweep (second workload)
 SWEEP_CASES = [  # (context, batch): 64-bit codes, fixed budgets, 32/8 heads, bf16, as in the paper's latency-vs-context study
-    (32768, 1), (32768, 16), (131072, 1), (131072, 8), (262144, 1), (262144, 4), (1048576, 1), (2097152, 1),
+    (32768, 1), (32768, 16), (131072, 1), (131072, 3), (131072, 8), (262144, 1), (262144, 4), (1048576, 1), (2097152, 1),
 ]
 
 
