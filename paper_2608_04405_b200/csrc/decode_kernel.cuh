@@ -214,8 +214,9 @@ __device__ __forceinline__ void csa(uint32_t a, uint32_t b, uint32_t c, uint32_t
 template <int W32, int NP>
 __device__ __forceinline__ int score_key(const uint32_t (&h)[W32], const uint32_t (&sg)[W32], const uint32_t (&mk)[NP][W32]) {
   int key = 0;
-  if constexpr (NP >= 4 && W32 >= 2) {
-    // Many planes (weighted scores): one population count per masked word would keep the 16-lane pipe busy for most
+  if constexpr (NP >= 3 && W32 >= 2) {
+    // Three or more planes (weighted scores; Hamming scores with five to eight query heads per KV head, where it took
+    // config 4's step from 46.7 to 44.7 us): one population count per masked word would keep the 16-lane pipe busy for most
     // of the scan.  A full adder per pair of masked words adds them to a carry word handed down from the plane below
     // (a + b + c = (a ^ b ^ c) + 2 maj(a, b, c), bit by bit), which halves the counts: W32/2 per plane plus W32/2 for
     // the last carries.  Each adder is three three-input logic operations, the masks included:
