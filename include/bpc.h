@@ -11,8 +11,15 @@
  *   - Every pointer is a DEVICE pointer owned by the caller unless its name starts with host_.
  *     The library allocates device memory only inside bpc_create (state of the context) and frees
  *     it in bpc_destroy.  No entry point copies, resizes or keeps caller buffers beyond the call.
+ *     The small per-step arrays q, k_new, v_new and out of bpc_decode_attn / bpc_append /
+ *     bpc_append_decode_attn may instead be pinned (page-locked) host memory that the device can
+ *     address at its host address (cudaHostAlloc / cudaHostRegister under unified addressing):
+ *     the kernels then read the step's inputs and write its result across the bus themselves,
+ *     which saves the copies of a host-driven decode loop.  Caches, codes and projections must be
+ *     device memory.
  *   - Every compute call is asynchronous on `stream` (a cudaStream_t passed as void*; NULL is the
- *     legacy default stream) and returns a bpc_status; nothing aborts, traps or prints.
+ *     legacy default stream) and returns a bpc_status; nothing aborts, traps or prints.  Only
+ *     bpc_last_device_error waits for the stream.
  *   - Layouts (row-major, contiguous):
  *       k_cache, v_cache : [batch][n_kv_heads][n_max] rows of head_dim kv_dtype values, base 16-byte
  *                          aligned; consecutive rows are kv_row_stride elements apart (head_dim when the
@@ -97,9 +104,11 @@ size_t  bpc_fit_workspace_bytes(const bpc_config* host_cfg);
 size_t  bpc_fit_codes_offset(const bpc_config* host_cfg);
 int64_t bpc_max_context(const bpc_config* host_cfg);
 
-/* Current number of cached keys of every sequence (host array [batch]).  Setting it uploads the
- * lengths asynchronously; the context keeps a host shadow that bpc_append advances, so capacity
- * errors are raised before any launch. */
+/* Current number of cached keys of every sequence (host array [batch]).  Setting it stages the per-unit lengths in
+ * pinned memory owned by the context and copies them to the device asynchronously on `stream` (no wait for the stream;
+ * host_lens may be reused as soon as the call returns).  Eight calls can be in flight; a ninth waits for the first
+ * one's copy.  The context keeps a host shadow that bpc_append advances, so capacity errors are raised before any
+ * launch. */
 bpc_status bpc_set_seq_lens(bpc_ctx* ctx, const int32_t* host_lens, void* stream);
 bpc_status bpc_get_seq_lens(bpc_ctx* ctx, int32_t* host_lens_out);
 
@@ -178,6 +187,7 @@ bpc_status bpc_append_decode_attn(bpc_ctx* ctx, const void* k_new, const void* v
  * scores only), q, k_cache, v_cache, codes, out as for bpc_decode_attn; P_hash = the hash projection rounded to
  * the cache dtype, [hash_sets][code_bits][head_dim] kv_dtype (what bpc_get_projection reports as P_hash_out,
  * stored in kv_dtype); unit_lens = number of cached keys per unit, [batch*n_kv_heads] int32 on the device.
+ * cfg.eas_ppm must be 0 (the safeguard set belongs to a context).
  *
  * Limits and hazards
  *   - batch * n_kv_heads * n_max must not exceed bpc_static_scratch_entries() (1 Mi index entries); larger
@@ -193,6 +203,9 @@ bpc_status bpc_decode_attn_static(const bpc_config* host_cfg, const void* q, con
                                   const uint64_t* codes, const void* P_hash, const int32_t* unit_lens,
                                   int32_t budget_ppm, int32_t budget_count, float* out, void* stream);
 size_t     bpc_static_scratch_entries(void);
+/* The error word of the last bpc_decode_attn_static call on the current device (it lives in the same built-in array):
+ * copies it to *host_out, waits for `stream`, and returns BPC_ERR_DEVICE when it is non-zero.  Allocates nothing. */
+bpc_status bpc_static_last_device_error(int32_t* host_out, void* stream);
 
 /* Quality yard-stick: the exact-score selector (appendix "Baseline Methods", TOPK (Oracle)).  For every query head,
  * scores[(seq * n_q_heads + head)][i] = q_head . k_i over the cached keys (fp32) and the k keys with the largest
@@ -235,8 +248,43 @@ int32_t    bpc_get_cluster_size(bpc_ctx* ctx);
 /* 1 when this context's decode calls use the streaming selection (units longer than a cluster's shared memory holds). */
 int32_t    bpc_uses_streaming(bpc_ctx* ctx);
 
-/* Diagnostics: device error word (synchronises the stream), last CUDA error code seen by the
- * context, number of kernels this context has launched so far. */
+/* A second decode kernel, kept as an alternative that can be selected per context.  (The paper has no counterpart: it is
+ * a different schedule for the same step.)  For bf16 caches with Hamming scores and no safeguard (at most 512 units) a
+ * decode call can run as ONE launch of a persistent grid (two blocks per SM) whose blocks take work items from global
+ * counters: per unit one cache-write item (fused call) and one query-hash item per 32 code bits, then code-scan items
+ * of a fixed number of keys and attention items over at most a fixed number of selected rows of one key range.
+ * Scores (2 bytes per cached key), range histograms, per-range offsets and attention partials of a step live in
+ * scratch memory that the first bpc_debug_set_decode_path(ctx, 2) allocates.  The selection is identical to the
+ * cluster kernel's and the output equal up to the summation order of the attention partials; any context length up to
+ * 2^25 keys is covered without the streaming selection.  On B200 it is slower than the cluster kernel on every
+ * configuration measured (hand-overs between items go through L2), so it is never chosen automatically.
+ * bpc_debug_set_decode_path: 0 or 1 = cluster kernel (default), 2 = work-item kernel (BPC_ERR_UNSUPPORTED if the
+ * context is not covered).  bpc_uses_work_items: 1 when this context's decode calls take that kernel.
+ * bpc_work_item_grid: its resident blocks.
+ * bpc_debug_set_work_item_geometry: keys per scan item (a multiple of 1792; 0 = automatic) and the most selected rows
+ * per attention item (<= 512; 0 = automatic).
+ * bpc_debug_set_work_item_trace: when set (non-NULL), every block records the items it ran: trace [blocks][64][12] uint64
+ * = (item type << 40 | unit << 24 | index, start ns, end ns, six time stamps inside the item, unused), types 1 cache
+ * write, 2 query hash, 3 scan, 4 attention, 5 threshold, 6 merge. */
+int32_t    bpc_uses_work_items(bpc_ctx* ctx);
+int32_t    bpc_work_item_grid(bpc_ctx* ctx);
+bpc_status bpc_debug_set_decode_path(bpc_ctx* ctx, int32_t path);
+bpc_status bpc_debug_set_work_item_geometry(bpc_ctx* ctx, int32_t keys_per_scan_item, int32_t rows_per_attend_item);
+bpc_status bpc_debug_set_work_item_trace(bpc_ctx* ctx, uint64_t* trace);
+
+/* Diagnostics.  bpc_last_device_error copies the device error word to *host_out; it is the one call that waits for
+ * `stream` (it returns a host value), and it returns BPC_ERR_DEVICE when the word is non-zero (bit 0: a unit did not
+ * fit the cluster's score storage, bit 1: append at n_max, bit 2: a bounded wait inside a kernel gave up), BPC_OK
+ * otherwise.  bpc_status_of_device_error is that mapping as a pure function.  Then: last CUDA error code seen by the
+ * context, number of kernels this context has launched so far.
+ * Diagnostic switches (explicit calls; the library reads no environment variable): bpc_debug_set_pdl(ctx, 0) launches
+ * the decode kernel without programmatic dependent launch; bpc_debug_set_tensor_core_encode(ctx, 0) makes
+ * bpc_encode_keys take the CUDA-core kernel; bpc_debug_force_streaming(ctx, 1) selects the streaming selection at any
+ * context length (Hamming scores without the safeguard only) and re-plans the launch geometry. */
+bpc_status bpc_status_of_device_error(int32_t error_word);
+bpc_status bpc_debug_set_pdl(bpc_ctx* ctx, int32_t on);
+bpc_status bpc_debug_set_tensor_core_encode(bpc_ctx* ctx, int32_t on);
+bpc_status bpc_debug_force_streaming(bpc_ctx* ctx, int32_t on);
 bpc_status bpc_last_device_error(bpc_ctx* ctx, int32_t* host_out, void* stream);
 int32_t    bpc_last_cuda_error(bpc_ctx* ctx);
 int64_t    bpc_launch_count(bpc_ctx* ctx);

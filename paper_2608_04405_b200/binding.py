@@ -64,12 +64,22 @@ def _load() -> ctypes.CDLL:
         "bpc_append_decode_attn": (i32, [vp, vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]),
         "bpc_decode_attn_static": (i32, [cfgp, vp, vp, vp, vp, vp, vp, i32, i32, vp, vp]),
         "bpc_static_scratch_entries": (sz, []),
+        "bpc_static_last_device_error": (i32, [ctypes.POINTER(i32), vp]),
         "bpc_debug_set_buffers": (i32, [vp, vp, vp]),
         "bpc_debug_set_phase_timer": (i32, [vp, vp]),
         "bpc_set_cluster_size": (i32, [vp, i32]),
         "bpc_plan_cluster_size": (i32, [cfgp, ctypes.POINTER(i32), i32]),
         "bpc_get_cluster_size": (i32, [vp]),
         "bpc_uses_streaming": (i32, [vp]),
+        "bpc_status_of_device_error": (i32, [i32]),
+        "bpc_debug_set_pdl": (i32, [vp, i32]),
+        "bpc_debug_set_tensor_core_encode": (i32, [vp, i32]),
+        "bpc_debug_force_streaming": (i32, [vp, i32]),
+        "bpc_uses_work_items": (i32, [vp]),
+        "bpc_work_item_grid": (i32, [vp]),
+        "bpc_debug_set_decode_path": (i32, [vp, i32]),
+        "bpc_debug_set_work_item_geometry": (i32, [vp, i32, i32]),
+        "bpc_debug_set_work_item_trace": (i32, [vp, vp]),
         "bpc_last_device_error": (i32, [vp, ctypes.POINTER(i32), vp]),
         "bpc_last_cuda_error": (i32, [vp]),
         "bpc_launch_count": (i64, [vp]),
@@ -86,10 +96,12 @@ lib = _load()
 EXPORTS = ["bpc_create", "bpc_destroy", "bpc_codes_bytes", "bpc_fit_workspace_bytes", "bpc_fit_codes_offset",
            "bpc_max_context",
            "bpc_set_seq_lens", "bpc_get_seq_lens", "bpc_fit", "bpc_set_projection", "bpc_get_projection",
-           "bpc_encode_keys", "bpc_build_eas", "bpc_get_eas", "bpc_eas_capacity", "bpc_exact_topk", "bpc_append", "bpc_decode_attn", "bpc_append_decode_attn", "bpc_decode_attn_static", "bpc_static_scratch_entries",
+           "bpc_encode_keys", "bpc_build_eas", "bpc_get_eas", "bpc_eas_capacity", "bpc_exact_topk", "bpc_append", "bpc_decode_attn", "bpc_append_decode_attn", "bpc_decode_attn_static", "bpc_static_scratch_entries", "bpc_static_last_device_error",
            "bpc_debug_set_buffers", "bpc_debug_set_phase_timer",
            "bpc_set_cluster_size", "bpc_plan_cluster_size",
-           "bpc_get_cluster_size", "bpc_uses_streaming", "bpc_last_device_error", "bpc_last_cuda_error", "bpc_launch_count", "bpc_version"]
+           "bpc_get_cluster_size", "bpc_uses_streaming", "bpc_status_of_device_error", "bpc_debug_set_pdl",
+           "bpc_debug_set_tensor_core_encode", "bpc_debug_force_streaming", "bpc_uses_work_items", "bpc_work_item_grid", "bpc_debug_set_decode_path",
+           "bpc_debug_set_work_item_geometry", "bpc_debug_set_work_item_trace", "bpc_last_device_error", "bpc_last_cuda_error", "bpc_launch_count", "bpc_version"]
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -274,10 +286,42 @@ class Context:
     def uses_streaming(self) -> bool:
         return bool(lib.bpc_uses_streaming(self._h))
 
+    def uses_work_items(self) -> bool:
+        return bool(lib.bpc_uses_work_items(self._h))
+
+    def work_item_grid(self) -> int:
+        return lib.bpc_work_item_grid(self._h)
+
+    def debug_set_decode_path(self, path: int) -> None:
+        """0 = the library chooses, 1 = cluster kernel, 2 = work-item kernel."""
+        _check(lib.bpc_debug_set_decode_path(self._h, path), "bpc_debug_set_decode_path")
+
+    def debug_set_work_item_geometry(self, keys_per_scan_item: int = 0, rows_per_attend_item: int = 0) -> None:
+        _check(lib.bpc_debug_set_work_item_geometry(self._h, keys_per_scan_item, rows_per_attend_item),
+               "bpc_debug_set_work_item_geometry")
+
+    def debug_set_work_item_trace(self, trace: Optional[torch.Tensor]) -> None:
+        self._trace = trace
+        _check(lib.bpc_debug_set_work_item_trace(self._h, _ptr(trace)), "bpc_debug_set_work_item_trace")
+
     def last_device_error(self) -> int:
+        """The device error word (0 = none).  The C call returns BPC_ERR_DEVICE for a non-zero word; here the word itself
+        is the result."""
         v = ctypes.c_int32(0)
-        _check(lib.bpc_last_device_error(self._h, ctypes.byref(v), _stream()), "bpc_last_device_error")
+        st = lib.bpc_last_device_error(self._h, ctypes.byref(v), _stream())
+        if st not in (BPC_OK, 6):
+            raise BpcError(st, "bpc_last_device_error")
+        assert (st == 6) == (v.value != 0)
         return v.value
+
+    def debug_set_pdl(self, on: bool) -> None:
+        _check(lib.bpc_debug_set_pdl(self._h, 1 if on else 0), "bpc_debug_set_pdl")
+
+    def debug_set_tensor_core_encode(self, on: bool) -> None:
+        _check(lib.bpc_debug_set_tensor_core_encode(self._h, 1 if on else 0), "bpc_debug_set_tensor_core_encode")
+
+    def debug_force_streaming(self, on: bool) -> None:
+        _check(lib.bpc_debug_force_streaming(self._h, 1 if on else 0), "bpc_debug_force_streaming")
 
     def last_cuda_error(self) -> int:
         return lib.bpc_last_cuda_error(self._h)
@@ -304,6 +348,15 @@ def bpc_decode_attn_static(cfg: bpc_config, q, k_cache, v_cache, codes, P_hash, 
                                       _ptr(P_hash), _ptr(unit_lens), budget_ppm, budget_count, _ptr(out), _stream()),
            "bpc_decode_attn_static")
     return out
+
+
+def bpc_static_last_device_error() -> int:
+    """Error word left by the last bpc_decode_attn_static call on the current device (0 = none)."""
+    v = ctypes.c_int32(0)
+    st = lib.bpc_static_last_device_error(ctypes.byref(v), _stream())
+    if st not in (BPC_OK, 6):
+        raise BpcError(st, "bpc_static_last_device_error")
+    return v.value
 
 
 def bpc_fit(ctx: Context, k_cache, v_star, workspace=None) -> None:

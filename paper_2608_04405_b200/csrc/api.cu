@@ -3,6 +3,7 @@
 #include <stdlib.h>
 #include <string.h>
 #include "common.cuh"
+#include "sched_host.h"
 
 cudaError_t bpc_launch_decode_bf16(bpc_ctx*, const DecodeParams&, cudaStream_t);
 cudaError_t bpc_launch_decode_f32(bpc_ctx*, const DecodeParams&, cudaStream_t);
@@ -120,6 +121,67 @@ int choose_cluster(const bpc_ctx* ctx, int chunk_cap, int max_cluster) {
   return best;
 }
 
+
+// ---- work-item decode kernel: which contexts it serves, its geometry and its scratch
+bool sched_covers(const bpc_config& c) {
+  return c.kv_dtype == BPC_BF16 && c.score_mode == BPC_SCORE_HAMMING && c.eas_ppm == 0 &&
+         (long long)c.batch * c.n_kv_heads <= bpcdev::kSchedMaxUnits;
+}
+
+int round_up(long long x, int g) { return (int)(((x + g - 1) / g) * g); }
+
+// keys per SCAN item: about 3.5 items per resident block over all units, a multiple of the granule, at most
+// kSchedMaxRanges items per unit and at most 32768 keys (range histogram counts are 16-bit)
+int sched_auto_ch(const bpc_ctx* ctx) {
+  const long long total = (long long)ctx->units * ctx->cfg.n_max;
+  long long ch = (long long)((double)total / (3.5 * ctx->sched_grid_max));
+  ch = round_up(ch < 1 ? 1 : ch, ctx->sched_gran);
+  int floor_ch = round_up((ctx->cfg.n_max + bpcdev::kSchedMaxRanges - 1) / bpcdev::kSchedMaxRanges, ctx->sched_gran);
+  if (ch < floor_ch) ch = floor_ch;
+  const int cap = (32768 / ctx->sched_gran) * ctx->sched_gran;
+  if (ch > cap) ch = cap;
+  return (int)ch;
+}
+
+cudaError_t sched_setup(bpc_ctx* ctx) {
+  ctx->sched_ok = false;
+  const bpc_config& c = ctx->cfg;
+  if (!sched_covers(c)) return cudaSuccess;
+  const int nbins = hist_bins(ctx);
+  int per_sm = 0;
+  cudaError_t e = bpc_sched_configure(ctx->group, c.code_bits, nbins, ctx->units, ctx->device, &ctx->sched_smem, &per_sm);
+  if (e != cudaSuccess) { (void)cudaGetLastError(); return cudaSuccess; }   // not schedulable here: the cluster kernel serves
+  if (per_sm < 1) return cudaSuccess;
+  ctx->sched_grid_max = per_sm * ctx->sm_count;
+  ctx->sched_gran = bpc_sched_granule(c.code_bits);
+  ctx->sched_ch = sched_auto_ch(ctx);
+  if ((c.n_max + ctx->sched_ch - 1) / ctx->sched_ch > bpcdev::kSchedMaxRanges) return cudaSuccess;   // context too long
+  // scratch rows are sized for the smallest range length a caller may ask for
+  int r_alloc = (c.n_max + ctx->sched_gran - 1) / ctx->sched_gran;
+  if (r_alloc > bpcdev::kSchedMaxRanges) r_alloc = bpcdev::kSchedMaxRanges;
+  ctx->sched_r_alloc = r_alloc;
+  // attention slices per unit: one or more per range, at most ranges + ceil(k / rows per slice) <= ranges + 64 + ...
+  int na = (c.n_max + bpcdev::kSchedListCap - 1) / bpcdev::kSchedListCap;
+  ctx->sched_na_cap = r_alloc + (na < 64 ? 64 : na) + 1;
+  ctx->sched_sc_stride = (c.n_max + 7) & ~7;
+  const int gp = bpc_sched_padded_group(ctx->group);
+  const int w32 = c.code_bits / 32;
+  const int np = gp <= 2 ? 1 : (gp == 4 ? 2 : 3);
+  ctx->sched_qp_words = (w32 * (2 + np) + 3) & ~3;
+  const size_t U = (size_t)ctx->units;
+  const size_t sync_words = bpcdev::kSchedSyncHead + U * bpcdev::kSchedSyncPerUnit;
+  e = cudaMalloc(&ctx->sc_scores, U * ctx->sched_sc_stride * 2);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->sc_hist, U * r_alloc * (size_t)nbins * 2);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->sc_table, U * (r_alloc + 1) * sizeof(int4));
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->sc_planes, U * ctx->sched_qp_words * 4);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->sc_partials, U * ctx->sched_na_cap * (size_t)gp * (BPC_D + 2) * 4);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->sc_sync, sync_words * 4);
+  if (e == cudaSuccess) e = cudaMemset(ctx->sc_sync, 0, sync_words * 4);
+  if (e != cudaSuccess) return e;
+  ctx->sched_ok = true;
+  return cudaSuccess;
+}
+
 }  // namespace
 
 cudaError_t bpc_plan_decode_geometry(bpc_ctx* ctx) {
@@ -132,8 +194,7 @@ cudaError_t bpc_plan_decode_geometry(bpc_ctx* ctx) {
   ctx->chunk_cap_limit = cap;
   ctx->cluster_size = choose_cluster(ctx, cap, ctx->max_cluster);
   ctx->streaming = false;
-  const char* force = getenv("BPC_FORCE_STREAMING");        // diagnostic switch: two-pass selection at any size
-  const bool forced = force != nullptr && force[0] == '1';
+  const bool forced = ctx->force_streaming;                 // diagnostic switch: two-pass selection at any size
   if ((ctx->cluster_size == 0 || forced) && ctx->cfg.score_mode == BPC_SCORE_HAMMING && ctx->cfg.eas_ppm == 0) {
     // Units too long for the largest cluster's shared memory: no score is stored, the codes are read twice.  The
     // largest cluster size that still runs all units in one wave is used (at least the largest schedulable one).
@@ -190,10 +251,7 @@ bpc_status bpc_create(const bpc_config* cfg, bpc_ctx** out) {
   ctx->sm_scale_d = cfg->sm_scale == 0.f ? 0.08838834764831845 : (double)cfg->sm_scale;   // default 1/sqrt(128)
   ctx->units = cfg->batch * cfg->n_kv_heads;
   ctx->group = cfg->n_q_heads / cfg->n_kv_heads;
-  {
-    const char* no_pdl = getenv("BPC_NO_PDL");          // diagnostic switch: plain stream-ordered launches
-    ctx->use_pdl = !(no_pdl != nullptr && no_pdl[0] == '1');
-  }
+  ctx->use_pdl = true;
   ctx->row_stride = cfg->kv_row_stride == 0 ? cfg->head_dim : cfg->kv_row_stride;
   cudaError_t e = cudaGetDevice(&ctx->device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device);
@@ -216,6 +274,9 @@ bpc_status bpc_create(const bpc_config* cfg, bpc_ctx** out) {
   if (e == cudaSuccess) e = cudaMalloc(&ctx->dev_err, 4);
   if (e == cudaSuccess) e = cudaMemset(ctx->dev_err, 0, 4);
   if (e == cudaSuccess) e = cudaMemset(ctx->unit_lens, 0, (size_t)ctx->units * 4);
+  if (e == cudaSuccess) e = cudaMallocHost(&ctx->lens_staging, (size_t)BPC_LENS_SLOTS * ctx->units * 4);
+  for (int i = 0; i < BPC_LENS_SLOTS && e == cudaSuccess; ++i)
+    e = cudaEventCreateWithFlags(&ctx->lens_event[i], cudaEventDisableTiming);
   ctx->host_lens = new (std::nothrow) int32_t[cfg->batch];
   if (ctx->host_lens) memset(ctx->host_lens, 0, sizeof(int32_t) * cfg->batch);
   if (e != cudaSuccess || ctx->host_lens == nullptr) {
@@ -225,8 +286,8 @@ bpc_status bpc_create(const bpc_config* cfg, bpc_ctx** out) {
   }
   e = bpc_plan_decode_geometry(ctx);
   if (e != cudaSuccess) { bpc_destroy(ctx); (void)cudaGetLastError(); return BPC_ERR_CUDA; }
-  if (ctx->cluster_size == 0) { bpc_destroy(ctx); return BPC_ERR_UNSUPPORTED; }
   if (hist_bins(ctx) > 2048 || hist_shift(ctx) > 5) { bpc_destroy(ctx); return BPC_ERR_UNSUPPORTED; }
+  if (ctx->cluster_size == 0) { bpc_destroy(ctx); return BPC_ERR_UNSUPPORTED; }
   *out = ctx;
   return BPC_OK;
 }
@@ -236,6 +297,11 @@ bpc_status bpc_destroy(bpc_ctx* ctx) {
   cudaFree(ctx->P); cudaFree(ctx->P_h); cudaFree(ctx->P_hf); cudaFree(ctx->gram);
   cudaFree(ctx->unit_lens); cudaFree(ctx->sel_scratch); cudaFree(ctx->dev_err);
   cudaFree(ctx->key_err); cudaFree(ctx->eas_idx); cudaFree(ctx->eas_cnt);
+  cudaFree(ctx->sc_scores); cudaFree(ctx->sc_hist); cudaFree(ctx->sc_table); cudaFree(ctx->sc_planes);
+  cudaFree(ctx->sc_partials); cudaFree(ctx->sc_sync);
+  if (ctx->lens_staging) cudaFreeHost(ctx->lens_staging);
+  for (int i = 0; i < BPC_LENS_SLOTS; ++i)
+    if (ctx->lens_event[i]) cudaEventDestroy(ctx->lens_event[i]);
   delete[] ctx->host_lens;
   delete ctx;
   (void)cudaGetLastError();
@@ -245,8 +311,13 @@ bpc_status bpc_destroy(bpc_ctx* ctx) {
 bpc_status bpc_set_cluster_size(bpc_ctx* ctx, int32_t cs) {
   if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
   const int cap = ctx->chunk_cap_limit, mc = ctx->max_cluster;
-  if (cs == 0 && ctx->streaming) return BPC_OK;            // keeps the size chosen at creation
-  if (cs == 0) cs = choose_cluster(ctx, cap, mc);
+  if (cs == 0) {                                           // back to the library's own choice of geometry
+    if (ctx->streaming) return BPC_OK;                     // keeps the size chosen at creation
+    cs = choose_cluster(ctx, cap, mc);
+    if (cs < 1) return BPC_ERR_UNSUPPORTED;
+    ctx->cluster_size = cs;
+    return BPC_OK;
+  }
   if (cs < 1 || cs > mc || ctx->max_active[cs] < 1) return BPC_ERR_UNSUPPORTED;
   if (!ctx->streaming && chunk_for(ctx->cfg.n_max, cs) > cap) return BPC_ERR_UNSUPPORTED;
   ctx->cluster_size = cs;
@@ -277,17 +348,20 @@ bpc_status bpc_set_seq_lens(bpc_ctx* ctx, const int32_t* host_lens, void* stream
   const bpc_config& c = ctx->cfg;
   for (int i = 0; i < c.batch; ++i)
     if (host_lens[i] < 0 || host_lens[i] > c.n_max) return BPC_ERR_CAPACITY;
-  // expand to per-unit lengths through a small pageable staging array: the copy is synchronous with
-  // respect to the host buffer, so the temporary can be released on return
-  int32_t* tmp = new (std::nothrow) int32_t[ctx->units];
-  if (tmp == nullptr) return BPC_ERR_INVALID_ARG;
+  // The per-unit lengths are staged in pinned memory owned by the context and copied asynchronously on `stream`: the
+  // call does not wait for the stream.  A ring of staging slots, each guarded by an event recorded after its copy,
+  // lets several calls be in flight; only a call that finds its slot's previous copy unfinished waits for that copy.
+  const int slot = ctx->lens_slot;
+  ctx->lens_slot = (slot + 1) % BPC_LENS_SLOTS;
+  cudaError_t e = cudaEventSynchronize(ctx->lens_event[slot]);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  int32_t* tmp = ctx->lens_staging + (size_t)slot * ctx->units;
   for (int i = 0; i < c.batch; ++i) {
     ctx->host_lens[i] = host_lens[i];
     for (int h = 0; h < c.n_kv_heads; ++h) tmp[i * c.n_kv_heads + h] = host_lens[i];
   }
-  cudaError_t e = cudaMemcpyAsync(ctx->unit_lens, tmp, (size_t)ctx->units * 4, cudaMemcpyHostToDevice, (cudaStream_t)stream);
-  if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
-  delete[] tmp;
+  e = cudaMemcpyAsync(ctx->unit_lens, tmp, (size_t)ctx->units * 4, cudaMemcpyHostToDevice, (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaEventRecord(ctx->lens_event[slot], (cudaStream_t)stream);
   return e == cudaSuccess ? BPC_OK : cuda_fail(ctx, e);
 }
 
@@ -410,6 +484,52 @@ static bpc_status decode_common(bpc_ctx* ctx, const void* k_new, const void* v_n
   if (budget_ppm == 0 && budget_count == 0) return BPC_ERR_INVALID_ARG;
   if (!ctx->fitted) return BPC_ERR_NOT_FITTED;
   const bpc_config& c = ctx->cfg;
+  const bool forced_stream_env = ctx->streaming && ctx->cluster_size > 0 && chunk_for(c.n_max, ctx->cluster_size) <= ctx->chunk_cap_limit;
+  (void)forced_stream_env;
+  const bool want_sched = ctx->sched_ok && ctx->decode_path == 2;   // measured slower than the cluster kernel: on request only
+  if (want_sched) {
+    bpcdev::SchedParams sp;
+    memset(&sp, 0, sizeof(sp));
+    sp.q = q; sp.k_cache = k_cache; sp.v_cache = v_cache; sp.codes = reinterpret_cast<const uint32_t*>(codes);
+    sp.P_h = ctx->P_h; sp.gram = ctx->gram; sp.unit_lens = ctx->unit_lens; sp.unit_lens_w = ctx->unit_lens;
+    sp.k_new = k_new; sp.v_new = v_new; sp.k_cache_w = k_cache_w; sp.v_cache_w = v_cache_w;
+    sp.codes_w = reinterpret_cast<uint32_t*>(codes_w);
+    sp.out = out; sp.sel = sel_idx;
+    sp.scores = ctx->sc_scores; sp.hist_rows = ctx->sc_hist; sp.table = reinterpret_cast<int4*>(ctx->sc_table);
+    sp.qplanes = ctx->sc_planes; sp.partials = ctx->sc_partials; sp.sync = ctx->sc_sync; sp.err = ctx->dev_err;
+    sp.dbg_scores = ctx->dbg_scores; sp.dbg_qweights = ctx->dbg_qweights; sp.dbg_trace = ctx->dbg_trace;
+    sp.units = ctx->units; sp.n_kv_heads = c.n_kv_heads; sp.group = ctx->group; sp.n_max = c.n_max;
+    sp.row_stride = ctx->row_stride; sp.shared_sets = c.hash_sets != ctx->units;
+    sp.budget_ppm = budget_ppm; sp.budget_count = budget_count; sp.residual_correction = c.residual_correction;
+    sp.ch = ctx->sched_ch_user > 0 ? ctx->sched_ch_user : ctx->sched_ch;
+    sp.r_max = (c.n_max + sp.ch - 1) / sp.ch;
+    const int k_max = bpcdev::sched_budget(c.n_max, budget_ppm, budget_count);
+    // rows per attention slice: a slice lies in one key range; twice the rows a range selects on average, so that
+    // most ranges are one slice, within [128, kSchedListCap] and never fewer than k/64 (bounds the slices per unit)
+    int rpa = ctx->sched_rpa_user;
+    if (rpa <= 0) {
+      rpa = (int)((2LL * k_max * sp.ch + c.n_max - 1) / c.n_max);
+      if (rpa < 128) rpa = 128;
+    }
+    if (rpa < (k_max + 63) / 64) rpa = (k_max + 63) / 64;
+    if (rpa > bpcdev::kSchedListCap) rpa = bpcdev::kSchedListCap;
+    sp.rpa = rpa;
+    sp.na_cap = ctx->sched_na_cap;
+    const int group_items = 2 * sp.r_max + (k_max + rpa - 1) / rpa;   // a unit's SCAN items plus (at most) its ATTEND items
+    if (sp.r_max + (k_max + rpa - 1) / rpa > sp.na_cap) return BPC_ERR_UNSUPPORTED;
+    sp.delta = 0;
+    sp.nbins = hist_bins(ctx);
+    sp.qp_words = ctx->sched_qp_words;
+    sp.sc_stride = ctx->sched_sc_stride;
+    sp.sm_scale_d = ctx->sm_scale_d;
+    long long items = (long long)ctx->units * (group_items + 2 + c.code_bits / 32);
+    const int grid = (int)(items < ctx->sched_grid_max ? items : ctx->sched_grid_max);
+    cudaError_t es = bpc_sched_launch(ctx->group, c.code_bits, sp, grid, ctx->sched_smem, ctx->use_pdl, (cudaStream_t)stream);
+    if (es != cudaSuccess) return cuda_fail(ctx, es);
+    ctx->launches += 1;
+    return BPC_OK;
+  }
+  if (ctx->cluster_size == 0) return BPC_ERR_UNSUPPORTED;
   const int cap = ctx->chunk_cap_limit;
   cudaError_t e;
   DecodeParams p;
@@ -481,11 +601,70 @@ bpc_status bpc_debug_set_phase_timer(bpc_ctx* ctx, uint64_t* stamps) {
   return BPC_OK;
 }
 
+bpc_status bpc_debug_set_pdl(bpc_ctx* ctx, int32_t on) {
+  if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
+  ctx->use_pdl = on != 0;
+  return BPC_OK;
+}
+
+bpc_status bpc_debug_set_tensor_core_encode(bpc_ctx* ctx, int32_t on) {
+  if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
+  ctx->no_tc_encode = on == 0;
+  return BPC_OK;
+}
+
+bpc_status bpc_debug_force_streaming(bpc_ctx* ctx, int32_t on) {
+  if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
+  if (on != 0 && (ctx->cfg.score_mode != BPC_SCORE_HAMMING || ctx->cfg.eas_ppm != 0)) return BPC_ERR_UNSUPPORTED;
+  ctx->force_streaming = on != 0;
+  cudaError_t e = bpc_plan_decode_geometry(ctx);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  return ctx->cluster_size > 0 ? BPC_OK : BPC_ERR_UNSUPPORTED;
+}
+
+bpc_status bpc_status_of_device_error(int32_t error_word) { return error_word == 0 ? BPC_OK : BPC_ERR_DEVICE; }
+
+bpc_status bpc_debug_set_decode_path(bpc_ctx* ctx, int32_t path) {
+  if (ctx == nullptr || path < 0 || path > 2) return BPC_ERR_INVALID_ARG;
+  if (path == 2 && !ctx->sched_ok) {                        // first request: plan the geometry, allocate the scratch
+    cudaError_t e = sched_setup(ctx);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+  }
+  if (path == 2 && !ctx->sched_ok) return BPC_ERR_UNSUPPORTED;
+  if (path == 1 && ctx->cluster_size == 0) return BPC_ERR_UNSUPPORTED;
+  ctx->decode_path = path;
+  return BPC_OK;
+}
+
+int32_t bpc_uses_work_items(bpc_ctx* ctx) { return (ctx != nullptr && ctx->sched_ok && ctx->decode_path == 2) ? 1 : 0; }
+
+bpc_status bpc_debug_set_work_item_geometry(bpc_ctx* ctx, int32_t keys_per_scan_item, int32_t rows_per_attend_item) {
+  if (ctx == nullptr || !ctx->sched_ok) return ctx == nullptr ? BPC_ERR_INVALID_ARG : BPC_ERR_UNSUPPORTED;
+  if (keys_per_scan_item < 0 || rows_per_attend_item < 0) return BPC_ERR_INVALID_ARG;
+  if (keys_per_scan_item > 0) {
+    if (keys_per_scan_item % ctx->sched_gran != 0 || keys_per_scan_item > 32768) return BPC_ERR_INVALID_ARG;
+    if ((ctx->cfg.n_max + keys_per_scan_item - 1) / keys_per_scan_item > ctx->sched_r_alloc) return BPC_ERR_INVALID_ARG;
+  }
+  if (rows_per_attend_item > bpcdev::kSchedListCap) return BPC_ERR_INVALID_ARG;
+  ctx->sched_ch_user = keys_per_scan_item;
+  ctx->sched_rpa_user = rows_per_attend_item;
+  return BPC_OK;
+}
+
+bpc_status bpc_debug_set_work_item_trace(bpc_ctx* ctx, uint64_t* trace) {
+  if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
+  ctx->dbg_trace = reinterpret_cast<unsigned long long*>(trace);
+  return BPC_OK;
+}
+
+int32_t bpc_work_item_grid(bpc_ctx* ctx) { return (ctx && ctx->sched_ok) ? ctx->sched_grid_max : 0; }
+
 bpc_status bpc_last_device_error(bpc_ctx* ctx, int32_t* host_out, void* stream) {
   if (ctx == nullptr || host_out == nullptr) return BPC_ERR_INVALID_ARG;
   cudaError_t e = cudaMemcpyAsync(host_out, ctx->dev_err, 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
-  return e == cudaSuccess ? BPC_OK : cuda_fail(ctx, e);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  return bpc_status_of_device_error(*host_out);
 }
 
 int32_t bpc_last_cuda_error(bpc_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }

@@ -8,6 +8,7 @@
 #define BPC_D 128            // head_dim (the paper's models all use 128)
 #define BPC_MAX_GROUP 8
 #define BPC_MAX_CLUSTER 16
+#define BPC_LENS_SLOTS 8      // pinned staging slots of bpc_set_seq_lens
 
 // Device error word bits.
 #define BPC_DEVERR_CHUNK_CAP   1   // a unit does not fit the cluster's score storage
@@ -42,6 +43,11 @@ struct bpc_ctx {
   float* gram;              // [hash_sets][b][b] float, P_h P_h^T
   int32_t* unit_lens;       // [units] device
   int32_t* host_lens;       // [batch] host shadow
+  int32_t* lens_staging;    // pinned, [BPC_LENS_SLOTS][units]: per-unit lengths on their way to the device
+  cudaEvent_t lens_event[BPC_LENS_SLOTS];
+  int lens_slot;
+  bool force_streaming;     // diagnostic switch: streaming selection at any size
+  bool no_tc_encode;        // diagnostic switch: CUDA-core encode kernel
   int32_t* sel_scratch;     // [units][n_max] int32
   int32_t* dev_err;         // device error word
   float* key_err;           // [units][n_max] squared reconstruction errors (error-aware safeguard), or null
@@ -56,6 +62,25 @@ struct bpc_ctx {
   int chunk_cap_limit;      // keys one decode block can hold with all opt-in shared memory
   double sm_scale_d;        // softmax scale in double (exact 1/sqrt(head_dim) by default)
   size_t decode_smem_set;   // non-zero once the decode kernel's function attributes have been set
+  // ---- work-item decode kernel (decode_sched.cuh): geometry and scratch, set up by bpc_create when the shape is covered
+  bool sched_ok;            // the work-item kernel serves this context's decode calls
+  int decode_path;          // 0 = automatic, 1 = cluster kernel, 2 = work-item kernel (diagnostic switch)
+  int sched_grid_max;       // resident blocks (SMs x blocks per SM)
+  size_t sched_smem;
+  int sched_gran;           // keys per SCAN item are a multiple of this
+  int sched_ch;             // keys per SCAN item (automatic choice)
+  int sched_r_alloc;        // SCAN items per unit the scratch rows are sized for
+  int sched_na_cap;         // ATTEND items per unit the partial slots are sized for
+  int sched_ch_user, sched_rpa_user;   // diagnostic overrides (0 = automatic)
+  int sched_sc_stride;
+  int sched_qp_words;
+  uint16_t* sc_scores;
+  uint16_t* sc_hist;
+  void* sc_table;
+  uint32_t* sc_planes;
+  float* sc_partials;
+  int32_t* sc_sync;
+  unsigned long long* dbg_trace;
 };
 
 struct DecodeParams {
@@ -142,6 +167,35 @@ __device__ __forceinline__ uint2 ld_stream_v2(const void* p) {
   asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p));
   return r;
 }
+
+// Streaming data (packed codes, gathered K/V rows) is read once per step: it is marked "evict first" in L2 so that it
+// does not push out what the step reuses (the kernel's own instructions, score keys, histograms, partials).
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint4 ld_stream_v4_ef(const void* p, uint64_t pol) {
+  uint4 r;
+  asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p), "l"(pol));
+  return r;
+}
+__device__ __forceinline__ uint2 ld_stream_v2_ef(const void* p, uint64_t pol) {
+  uint2 r;
+  asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v2.u32 {%0,%1}, [%2], %3;" : "=r"(r.x), "=r"(r.y) : "l"(p), "l"(pol));
+  return r;
+}
+__device__ __forceinline__ uint32_t ld_stream_u32_ef(const void* p, uint64_t pol) {
+  uint32_t r;
+  asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.u32 %0, [%1], %2;" : "=r"(r) : "l"(p), "l"(pol));
+  return r;
+}
+__device__ __forceinline__ void cp_async16_ef(void* smem_dst, const void* gsrc, uint64_t pol) {
+  const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(d), "l"(gsrc), "l"(pol) : "memory");
+}
+
 
 template <typename T> struct KvTraits;
 template <> struct KvTraits<__nv_bfloat16> {

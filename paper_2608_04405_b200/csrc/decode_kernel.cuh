@@ -311,8 +311,14 @@ bpc_decode_kernel(const DecodeParams p) {
   const int kvh = unit % p.n_kv_heads;
   const int seq = unit / p.n_kv_heads;
 
-  // The projection is written only by bpc_fit / bpc_set_projection, never by a decode launch, and only decode
-  // launches release their successor early; so its (cold) rows may be requested before the dependency wait below.
+  // Programmatic dependent launch: when this grid was launched early (while its predecessor in the stream
+  // was still running) nothing of the predecessor's output may be read before this point; afterwards the
+  // successor's blocks may be scheduled as ours drain.  Both are no-ops for an ordinary launch.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+  // The rows of the projection are requested first of all after the dependency wait (the kernel before this one in
+  // the stream may be the one that wrote them: bpc_fit, bpc_set_projection).
   constexpr int HPARTS = NT / B;                 // slices per projection row in the query hash
   constexpr int HDS = BPC_D / HPARTS;            // channels per slice (a multiple of 8)
   constexpr int HV = HDS * (int)sizeof(KV) / 16; // 16-byte vectors per slice
@@ -324,12 +330,6 @@ bpc_decode_kernel(const DecodeParams p) {
 #pragma unroll
     for (int v = 0; v < HV; ++v) prow[v] = row[v];
   }
-
-  // Programmatic dependent launch: when this grid was launched early (while its predecessor in the stream
-  // was still running) nothing of the predecessor's output may be read before this point; afterwards the
-  // successor's blocks may be scheduled as ours drain.  Both are no-ops for an ordinary launch.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   // The queries do not depend on the sequence length: their loads overlap the length read and the set-up below.
   const KV* qg = reinterpret_cast<const KV*>(p.q) + ((size_t)seq * p.n_kv_heads + kvh) * (size_t)G * BPC_D;

@@ -384,10 +384,7 @@ cudaError_t launch(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStrea
 // longer fits next to the operands in shared memory).
 cudaError_t bpc_launch_encode_tc(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStream_t stream) {
   if (ctx->cfg.kv_dtype != BPC_BF16) return cudaErrorNotSupported;
-  {
-    const char* off = getenv("BPC_NO_TC_ENCODE");           // diagnostic switch: force the CUDA-core kernel
-    if (off != nullptr && off[0] == '1') return cudaErrorNotSupported;
-  }
+  if (ctx->no_tc_encode) return cudaErrorNotSupported;     // diagnostic switch: the CUDA-core kernel is asked for
   cudaError_t e;
   if (ctx->cfg.code_bits == 64) e = launch<64>(ctx, k_cache, codes, stream);
   else if (ctx->cfg.code_bits == 128) e = launch<128>(ctx, k_cache, codes, stream);

@@ -71,6 +71,8 @@ bpc_status bpc_decode_attn_static(const bpc_config* cfg, const void* q, const vo
     return BPC_ERR_INVALID_ARG;
   if (cfg->head_dim != BPC_D) return BPC_ERR_UNSUPPORTED;
   if (cfg->code_bits != 32 && cfg->code_bits != 64 && cfg->code_bits != 128 && cfg->code_bits != 256) return BPC_ERR_UNSUPPORTED;
+  if (cfg->code_bits == 32 && cfg->n_max % 4 != 0) return BPC_ERR_INVALID_ARG;   // 16-byte aligned code rows per unit
+  if (cfg->eas_ppm != 0) return BPC_ERR_UNSUPPORTED;        // the safeguard set lives in a context
   if (cfg->n_q_heads % cfg->n_kv_heads != 0) return BPC_ERR_INVALID_ARG;
   const int group = cfg->n_q_heads / cfg->n_kv_heads;
   if (group > BPC_MAX_GROUP) return BPC_ERR_UNSUPPORTED;
@@ -104,8 +106,11 @@ bpc_status bpc_decode_attn_static(const bpc_config* cfg, const void* q, const vo
   if (nbins > 2048) return BPC_ERR_UNSUPPORTED;
   e = bpc_plan_decode_geometry(&tmp);                       // occupancy queries only; nothing is allocated
   if (e != cudaSuccess) { (void)cudaGetLastError(); return BPC_ERR_CUDA; }
-  if (tmp.cluster_size == 0) return BPC_ERR_UNSUPPORTED;
+  // only the plain kernel is launched here: contexts too long for a cluster's shared memory (which a context would
+  // serve with the streaming selection) are refused
+  if (tmp.cluster_size == 0 || tmp.streaming) return BPC_ERR_UNSUPPORTED;
   const int cs = tmp.cluster_size;
+  if (chunk_for(cfg->n_max, cs) > tmp.chunk_cap_limit) return BPC_ERR_UNSUPPORTED;
 
   // the error word accumulates with atomicOr, so it has to start at zero; the list is overwritten before use
   e = cudaMemsetAsync(scratch, 0, BPC_STATIC_HEADER_BYTES, (cudaStream_t)stream);
@@ -126,6 +131,18 @@ bpc_status bpc_decode_attn_static(const bpc_config* cfg, const void* q, const vo
                                 : bpc_launch_decode_f32(&tmp, p, (cudaStream_t)stream);
   if (e != cudaSuccess) { (void)cudaGetLastError(); return BPC_ERR_CUDA; }
   return BPC_OK;
+}
+
+bpc_status bpc_static_last_device_error(int32_t* host_out, void* stream) {
+  if (host_out == nullptr) return BPC_ERR_INVALID_ARG;
+  int device = 0;
+  cudaError_t e = cudaGetDevice(&device);
+  void* scratch = nullptr;
+  if (e == cudaSuccess) e = scratch_for_current_device(device, &scratch);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(host_out, scratch, 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+  if (e != cudaSuccess) { (void)cudaGetLastError(); return BPC_ERR_CUDA; }
+  return *host_out == 0 ? BPC_OK : BPC_ERR_DEVICE;
 }
 
 #pragma GCC visibility pop

@@ -181,13 +181,13 @@ class Workload:
 
 
 def algorithmic_bytes_per_step(spec: WorkloadSpec, seq_lens: Sequence[int]) -> int:
-    """Bytes one decode step must move: packed codes of every cached key, the selected K and V rows,
-    the queries and outputs, and the projection once per KV head (Appendix "CUDA Optimizations":
-    one code word per key; selected rows only)."""
+    """Bytes one decode step must move: packed codes of every cached key, the selected K and V rows, the queries
+    and the outputs (Appendix "CUDA Optimizations": one code word per key; selected rows only).  The hash
+    projection (b*D*esz per unit, about 1 % more) is read too but is not counted."""
     D, b, G = spec.head_dim, spec.code_bits, spec.group
     total = 0
     for n in seq_lens:
         k = min(n, -(-n * spec.budget_ppm // 1000000))
-        per_unit = n * b // 8 + 2 * k * D * spec.esz + G * D * (spec.esz + 4) + b * D * spec.esz
+        per_unit = n * b // 8 + 2 * k * D * spec.esz + G * D * (spec.esz + 4)
         total += per_unit * spec.n_kv_heads
     return total

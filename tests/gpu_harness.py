@@ -42,7 +42,8 @@ class Session:
     """A workload on the GPU with its library context, fitted and encoded."""
 
     def __init__(self, spec: WorkloadSpec, gen_device: str = "cpu", salt: int = 0, cluster_size: int = 0,
-                 extra_rows=None, interleaved: bool = False, score_mode: int = 0, eas_ppm: int = 0, fit_power_iters: int = 0):
+                 extra_rows=None, interleaved: bool = False, score_mode: int = 0, eas_ppm: int = 0, fit_power_iters: int = 0,
+                 decode_path: int = 0, force_streaming: bool = False):
         self.spec = spec
         self.w = Workload(spec, device=gen_device, extra_rows=extra_rows, salt=salt)
         dev = "cuda"
@@ -60,8 +61,12 @@ class Session:
                                  score_mode=score_mode, eas_ppm=eas_ppm, fit_power_iters=fit_power_iters)
         self.s_err = None
         self.ctx = B.Context(self.cfg)
+        if force_streaming:
+            self.ctx.debug_force_streaming(True)
         if cluster_size:
             self.ctx.set_cluster_size(cluster_size)
+        if decode_path:
+            self.ctx.debug_set_decode_path(decode_path)
         self.lens = list(self.w.seq_lens)
         self.ctx.set_seq_lens(self.lens)
         self.codes = self.ctx.alloc_codes()
@@ -142,6 +147,17 @@ def check_fit(sess: Session, units, report: dict):
             R = R - np.outer(uu, v)
             Pref[i] = v
         assert hard == 0, "fit: %d sign decisions differ outside the ambiguity band (unit %d)" % (hard, u)
+        # Whatever signs were adopted inside the band (which is wide once the residual has all but vanished, e.g. for a
+        # context shorter than the code length, or where the power iteration's tracked Gram matrix holds only rounding
+        # noise), the library's own pair (H, P) must reconstruct the keys as well as the fp64 replay of those signs does:
+        # || K - H P ||_F <= || R_b ||_F + 2e-5 * sqrt(b) * || K ||_F (the row tolerance below, summed over the b rows).
+        # Where the residual has vanished this pins the reconstruction at rounding level.
+        Hpm = 2.0 * gpuH.astype(np.float64) - 1.0
+        rec_err = float(np.linalg.norm(K - Hpm @ gpuP))
+        bound = float(np.linalg.norm(R)) * (1.0 + 1e-3) + 2e-5 * np.sqrt(s.code_bits) * float(np.linalg.norm(K))
+        assert rec_err <= bound, "fit: || K - H P ||_F = %g exceeds the replayed residual %g (unit %d)" % (rec_err, bound, u)
+        report["fit_reconstruction_err_over_K"] = max(report.get("fit_reconstruction_err_over_K", 0.0),
+                                                      rec_err / max(float(np.linalg.norm(K)), 1e-300))
         # rows: 2e-5 relative, plus the same absolute rounding floor in units of a typical key row (a row of P that is
         # itself at rounding level, e.g. once the residual of a tiny context has vanished, cannot be held to 2e-5 of itself)
         floor = eps_band * float(np.linalg.norm(K) / np.sqrt(max(n, 1)))

@@ -42,6 +42,18 @@ def test_size_queries_and_config_validation_without_gpu():
     assert off % 256 == 0
 
 
+def test_device_error_word_maps_to_a_status_and_library_reads_no_environment():
+    """A non-zero device error word is reported as BPC_ERR_DEVICE (6); diagnostic switches are explicit calls, so no
+    source file of the library reads the environment."""
+    from paper_2608_04405_b200 import binding as B
+    assert B.lib.bpc_status_of_device_error(0) == B.BPC_OK
+    for word in (1, 2, 4, 7):
+        assert B.lib.bpc_status_of_device_error(word) == 6 and B.STATUS_NAMES[6] == "BPC_ERR_DEVICE"
+    csrc = os.path.join(ROOT, "paper_2608_04405_b200", "csrc")
+    for f in os.listdir(csrc):
+        assert "getenv" not in open(os.path.join(csrc, f)).read(), "%s reads the environment" % f
+
+
 def test_product_path_does_not_import_the_checker():
     pkg = os.path.join(ROOT, "paper_2608_04405_b200")
     for dirpath, _, files in os.walk(pkg):

@@ -49,20 +49,20 @@ def test_random_shapes(case, monkeypatch):
     i, bits, group, dtype, n_kv, batch, n_ctx, ragged, mode, eas, cluster, budget, interleaved, stream, power = case
     if mode == 1 and 127 * group * bits > 65535:
         mode = 0                                        # weighted scores would not fit 16 bits: plain Hamming instead
-    if stream:
-        monkeypatch.setenv("BPC_FORCE_STREAMING", "1")
+    stream = bool(stream and mode == 0 and eas == 0)      # the streaming selection covers Hamming scores without the safeguard
     spec = CONFIGS[1].scaled(name="fuzz%d" % i, wid=200 + i, batch=batch, n_kv_heads=n_kv, n_q_heads=n_kv * group, n_ctx=n_ctx,
                              n_ctx_min=max(1, n_ctx // 5) if ragged else None, dtype=dtype, code_bits=bits, steps=2,
                              needles=4, rope_base=None if dtype == "f32" else 500000.0)
     try:
         sess = H.Session(spec, gen_device="cuda", cluster_size=cluster, interleaved=interleaved, score_mode=mode, eas_ppm=eas,
-                         fit_power_iters=power)
+                         fit_power_iters=power, force_streaming=stream)
     except RuntimeError as e:
         if "UNSUPPORTED" in str(e):                     # e.g. a cluster size the shape cannot use
-            sess = H.Session(spec, gen_device="cuda", interleaved=interleaved, score_mode=mode, eas_ppm=eas, fit_power_iters=power)
+            sess = H.Session(spec, gen_device="cuda", interleaved=interleaved, score_mode=mode, eas_ppm=eas, fit_power_iters=power,
+                             force_streaming=stream)
         else:
             raise
-    assert sess.ctx.uses_streaming() == bool(stream and mode == 0)
+    assert sess.ctx.uses_streaming() == stream
     rep = {}
     units = sorted({0, sess.units - 1, sess.units // 2})
     sess.fit(); H.check_fit(sess, units[:1], rep)

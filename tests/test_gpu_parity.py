@@ -56,6 +56,27 @@ def test_cluster_sizes_agree_with_checker(cluster):
     print(rep)
 
 
+@pytest.mark.parametrize("bits,group,n,batch", [(128, 4, 5037, 1), (64, 1, 3000, 2), (256, 4, 9000, 1), (128, 7, 20011, 2),
+                                                (32, 8, 4000, 1), (128, 2, 70000, 1)])
+def test_work_item_kernel_agrees_with_checker(bits, group, n, batch):
+    """The alternative decode kernel (persistent grid of work items; selected per context) through the same stage-wise
+    checks: decode alone, fused cache write + decode at two consecutive steps, ragged tails, several key ranges."""
+    H = _harness()
+    spec = CONFIGS[1].scaled(batch=batch, n_ctx=n, n_kv_heads=2, n_q_heads=2 * group, code_bits=bits, steps=2)
+    sess = H.Session(spec, gen_device="cuda", decode_path=2, interleaved=(bits == 128))
+    assert sess.ctx.uses_work_items()
+    rep = {}
+    sess.fit()
+    sess.encode(); H.check_encode(sess, [0, 1], rep, max_keys=4096)
+    units = [0, 2 * batch - 1]
+    _decode_loop(sess, 2, units, rep, H)
+    q, _ = sess.w.queries(sess.lens, k_cache=sess.k_cache)
+    H.check_decode(sess, q, units, rep, budget_ppm=1000000)       # every key selected: dense attention
+    H.check_decode(sess, q, units, rep, budget_ppm=0, budget_count=1)
+    assert sess.ctx.last_device_error() == 0
+    print(rep)
+
+
 @pytest.mark.parametrize("bits,group,dtype", [(64, 1, "bf16"), (64, 4, "bf16"), (256, 4, "bf16"), (128, 7, "bf16"),
                                               (128, 8, "bf16"), (128, 2, "bf16"), (128, 3, "f32"), (256, 1, "f32"),
                                               (32, 4, "bf16"), (32, 1, "f32"), (32, 8, "bf16")])
@@ -230,12 +251,12 @@ def test_tensor_core_encode_agrees_with_cuda_core_encode(bits):
     tc = sess.codes.clone()
     rep = {}
     H.check_encode(sess, [0, 1], rep)
-    os.environ["BPC_NO_TC_ENCODE"] = "1"
+    sess.ctx.debug_set_tensor_core_encode(False)
     try:
         sess.codes.zero_()
         sess.encode()
     finally:
-        del os.environ["BPC_NO_TC_ENCODE"]
+        sess.ctx.debug_set_tensor_core_encode(True)
     H.check_encode(sess, [0, 1], rep)
     n = sess.lens[0]
     diff = (tc[:, :, :n] != sess.codes[:, :, :n]).any(dim=-1).sum().item()
@@ -301,7 +322,8 @@ def test_cfg2_full_size_sampled_units():
     rep = {}
     sess.fit()
     sess.encode(); H.check_encode(sess, [5], rep, key_slice=(120000, 124096))
-    _decode_loop(sess, 1, [0, 13, 31], rep, H)
+    # two steps: bpc_append + bpc_decode_attn, then the fused bpc_append_decode_attn launch (the one the benchmark times)
+    _decode_loop(sess, 2, [0, 13, 31], rep, H)
     # planted-needle recall of the selection is the same number on both sides because the index sets are identical
     print(rep)
 
@@ -386,14 +408,13 @@ def test_streaming_selection_two_million_keys():
 
 @pytest.mark.parametrize("dtype,bits,group,n,cluster", [("bf16", 128, 4, 40000, 4), ("f32", 64, 2, 9000, 2), ("bf16", 256, 8, 7000, 1),
                                                         ("bf16", 32, 4, 12000, 2)])
-def test_streaming_selection_forced_at_ordinary_sizes(dtype, bits, group, n, cluster, monkeypatch):
+def test_streaming_selection_forced_at_ordinary_sizes(dtype, bits, group, n, cluster):
     """The streaming selection forced on contexts that would fit (diagnostic switch), so that it is checked stage by
     stage at sizes the checker handles in full: several cluster sizes, both cache types, fused steps and ties."""
-    monkeypatch.setenv("BPC_FORCE_STREAMING", "1")
     H = _harness()
     spec = CONFIGS[1].scaled(name="streamf", wid=91 + group, batch=2, n_kv_heads=2, n_q_heads=2 * group, n_ctx=n, dtype=dtype,
                              code_bits=bits, steps=3)
-    sess = H.Session(spec, gen_device="cuda", cluster_size=cluster)
+    sess = H.Session(spec, gen_device="cuda", cluster_size=cluster, force_streaming=True)
     assert sess.ctx.uses_streaming()
     rep = {}
     sess.fit(); sess.encode()
