@@ -360,7 +360,7 @@ def run_ours(args):
     ms_app = _time_graph(g_app, barrier) / K
     # --- the paper's weighted score (sign + 7 magnitude planes) on the same workload, where 16-bit keys suffice
     ms_w7 = None
-    if 127 * spec.group * spec.code_bits <= 65535:
+    if True:
         for ly, c in zip(layers, per_layer_w):
             ly.make_weighted_twin(B)
             ly.ctx_w7.set_seq_lens([n + c for n in ly.lens0])

@@ -280,9 +280,13 @@ bpc_status bpc_debug_set_work_item_trace(bpc_ctx* ctx, uint64_t* trace);
  * Diagnostic switches (explicit calls; the library reads no environment variable): bpc_debug_set_pdl(ctx, 0) launches
  * the decode kernel without programmatic dependent launch; bpc_debug_set_tensor_core_encode(ctx, 0) makes
  * bpc_encode_keys take the CUDA-core kernel; bpc_debug_force_streaming(ctx, 1) selects the streaming selection at any
- * context length (Hamming scores without the safeguard only) and re-plans the launch geometry. */
+ * context length (Hamming scores without the safeguard only) and re-plans the launch geometry;
+ * bpc_debug_force_key_shift(ctx, s) with s in 0..2 stores weighted score keys shifted right by at least s bits (the
+ * library does that by itself only when a query's largest possible score exceeds 16 bits), so that the exact
+ * re-scoring of the keys at the threshold can be exercised at any shape. */
 bpc_status bpc_status_of_device_error(int32_t error_word);
 bpc_status bpc_debug_set_pdl(bpc_ctx* ctx, int32_t on);
+bpc_status bpc_debug_force_key_shift(bpc_ctx* ctx, int32_t shift);
 bpc_status bpc_debug_set_tensor_core_encode(bpc_ctx* ctx, int32_t on);
 bpc_status bpc_debug_force_streaming(bpc_ctx* ctx, int32_t on);
 bpc_status bpc_last_device_error(bpc_ctx* ctx, int32_t* host_out, void* stream);

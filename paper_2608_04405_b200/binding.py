@@ -73,6 +73,7 @@ def _load() -> ctypes.CDLL:
         "bpc_uses_streaming": (i32, [vp]),
         "bpc_status_of_device_error": (i32, [i32]),
         "bpc_debug_set_pdl": (i32, [vp, i32]),
+        "bpc_debug_force_key_shift": (i32, [vp, i32]),
         "bpc_debug_set_tensor_core_encode": (i32, [vp, i32]),
         "bpc_debug_force_streaming": (i32, [vp, i32]),
         "bpc_uses_work_items": (i32, [vp]),
@@ -99,7 +100,7 @@ EXPORTS = ["bpc_create", "bpc_destroy", "bpc_codes_bytes", "bpc_fit_workspace_by
            "bpc_encode_keys", "bpc_build_eas", "bpc_get_eas", "bpc_eas_capacity", "bpc_exact_topk", "bpc_append", "bpc_decode_attn", "bpc_append_decode_attn", "bpc_decode_attn_static", "bpc_static_scratch_entries", "bpc_static_last_device_error",
            "bpc_debug_set_buffers", "bpc_debug_set_phase_timer",
            "bpc_set_cluster_size", "bpc_plan_cluster_size",
-           "bpc_get_cluster_size", "bpc_uses_streaming", "bpc_status_of_device_error", "bpc_debug_set_pdl",
+           "bpc_get_cluster_size", "bpc_uses_streaming", "bpc_status_of_device_error", "bpc_debug_set_pdl", "bpc_debug_force_key_shift",
            "bpc_debug_set_tensor_core_encode", "bpc_debug_force_streaming", "bpc_uses_work_items", "bpc_work_item_grid", "bpc_debug_set_decode_path",
            "bpc_debug_set_work_item_geometry", "bpc_debug_set_work_item_trace", "bpc_last_device_error", "bpc_last_cuda_error", "bpc_launch_count", "bpc_version"]
 
@@ -316,6 +317,9 @@ class Context:
 
     def debug_set_pdl(self, on: bool) -> None:
         _check(lib.bpc_debug_set_pdl(self._h, 1 if on else 0), "bpc_debug_set_pdl")
+
+    def debug_force_key_shift(self, shift: int) -> None:
+        _check(lib.bpc_debug_force_key_shift(self._h, shift), "bpc_debug_force_key_shift")
 
     def debug_set_tensor_core_encode(self, on: bool) -> None:
         _check(lib.bpc_debug_set_tensor_core_encode(self._h, 1 if on else 0), "bpc_debug_set_tensor_core_encode")

@@ -34,8 +34,9 @@ bpc_status check_cfg(const bpc_config* c) {
   if (c->n_q_heads / c->n_kv_heads > BPC_MAX_GROUP) return BPC_ERR_UNSUPPORTED;
   if (c->kv_dtype != BPC_BF16 && c->kv_dtype != BPC_F32) return BPC_ERR_UNSUPPORTED;
   if (c->score_mode != BPC_SCORE_HAMMING && c->score_mode != BPC_SCORE_WEIGHTED7) return BPC_ERR_INVALID_ARG;
-  // weighted scores are kept as 16-bit keys: the largest possible score 127 * G * b must fit
-  if (c->score_mode == BPC_SCORE_WEIGHTED7 && 127LL * (c->n_q_heads / c->n_kv_heads) * c->code_bits > 65535) return BPC_ERR_UNSUPPORTED;
+  // weighted scores are kept as 16-bit keys, shifted right by up to two bits when the largest possible score
+  // 127 * G * b needs more (the dropped bits are recovered for the keys at the threshold)
+  if (c->score_mode == BPC_SCORE_WEIGHTED7 && 127LL * (c->n_q_heads / c->n_kv_heads) * c->code_bits > 4LL * 65535) return BPC_ERR_UNSUPPORTED;
   const long long units = (long long)c->batch * c->n_kv_heads;
   if (c->hash_sets != units && c->hash_sets != c->n_kv_heads) return BPC_ERR_INVALID_ARG;
   if (c->residual_correction != 0 && c->residual_correction != 1) return BPC_ERR_INVALID_ARG;
@@ -63,12 +64,14 @@ int max_score_key(const bpc_ctx* ctx) {
   if (ctx->cfg.score_mode == BPC_SCORE_WEIGHTED7) return 127 * G * b;
   return (G * b) >> ((G % 2 == 0) ? 1 : 0);
 }
+// (the histogram is taken over the stored keys, which are at most 16 bits wide)
+int max_stored_key(const bpc_ctx* ctx) { const int m = max_score_key(ctx); return m > 65535 ? 65535 : m; }
 int hist_shift(const bpc_ctx* ctx) {
   int s = 0;
-  while ((max_score_key(ctx) >> s) >= 2048) ++s;
+  while ((max_stored_key(ctx) >> s) >= 2048) ++s;
   return s;
 }
-int hist_bins(const bpc_ctx* ctx) { return (max_score_key(ctx) >> hist_shift(ctx)) + 1; }
+int hist_bins(const bpc_ctx* ctx) { return (max_stored_key(ctx) >> hist_shift(ctx)) + 1; }
 
 cudaError_t decode_limits(const bpc_ctx* ctx, int /*unused*/, int* max_cluster, int* chunk_cap, size_t* smem) {
   const int nbins = hist_bins(ctx);
@@ -550,6 +553,7 @@ static bpc_status decode_common(bpc_ctx* ctx, const void* k_new, const void* v_n
   p.chunk_cap = ctx->streaming ? 0 : chunk;               // shared memory is sized for the largest possible unit
   p.nbins = hist_bins(ctx);
   p.hist_shift = hist_shift(ctx);
+  p.key_shift_min = ctx->key_shift_min;
   if (ctx->streaming)
     e = c.kv_dtype == BPC_BF16 ? bpc_launch_decode_bf16_stream(ctx, p, (cudaStream_t)stream)
                                : bpc_launch_decode_f32_stream(ctx, p, (cudaStream_t)stream);
@@ -604,6 +608,13 @@ bpc_status bpc_debug_set_phase_timer(bpc_ctx* ctx, uint64_t* stamps) {
 bpc_status bpc_debug_set_pdl(bpc_ctx* ctx, int32_t on) {
   if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
   ctx->use_pdl = on != 0;
+  return BPC_OK;
+}
+
+bpc_status bpc_debug_force_key_shift(bpc_ctx* ctx, int32_t shift) {
+  if (ctx == nullptr || shift < 0 || shift > 2) return BPC_ERR_INVALID_ARG;
+  if (ctx->cfg.score_mode != BPC_SCORE_WEIGHTED7) return BPC_ERR_UNSUPPORTED;
+  ctx->key_shift_min = shift;
   return BPC_OK;
 }
 

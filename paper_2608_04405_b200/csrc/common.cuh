@@ -48,6 +48,7 @@ struct bpc_ctx {
   int lens_slot;
   bool force_streaming;     // diagnostic switch: streaming selection at any size
   bool no_tc_encode;        // diagnostic switch: CUDA-core encode kernel
+  int key_shift_min;        // diagnostic switch: weighted scores stored with at least this right shift
   int32_t* sel_scratch;     // [units][n_max] int32
   int32_t* dev_err;         // device error word
   float* key_err;           // [units][n_max] squared reconstruction errors (error-aware safeguard), or null
@@ -119,7 +120,8 @@ struct DecodeParams {
   int stages;                // gather ring depth (2 or 3)
   int chunk_cap;             // keys whose scores one thread block can hold
   int nbins;                 // histogram bins
-  int hist_shift;            // histogram bin = score key >> hist_shift
+  int hist_shift;            // histogram bin = stored score key >> hist_shift
+  int key_shift_min;         // weighted scores: smallest right shift of the stored 16-bit keys (diagnostic; normally 0)
 };
 
 // ---- launchers implemented in the per-dtype translation units

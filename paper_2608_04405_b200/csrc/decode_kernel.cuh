@@ -284,6 +284,21 @@ struct RowFragF32 {
   }
 };
 
+// Exact score key of one code from the query planes kept in shared memory (sign words, then mask planes).  Used
+// only for the few keys whose stored 16-bit key equals the threshold when weighted scores need more than 16 bits;
+// kept out of line so that its registers do not weigh on the loops that call it.
+template <int W32, int NP>
+__device__ __noinline__ int rescore_key(const uint32_t* code, const uint32_t* signw, const uint32_t (*mask)[8]) {
+  uint32_t h[W32], sg[W32], mk[NP][W32];
+#pragma unroll
+  for (int w = 0; w < W32; ++w) {
+    h[w] = code[w]; sg[w] = signw[w];
+#pragma unroll
+    for (int pl = 0; pl < NP; ++pl) mk[pl][w] = mask[pl][w];
+  }
+  return score_key<W32, NP>(h, sg, mk);
+}
+
 // VAR selects what is compiled in besides the plain path (VAR = 0): 1 = the error-aware safeguard (a static
 // hard-to-hash set that is always attended); 2 = the streaming selection for units whose scores do not fit the
 // cluster's shared memory (no score is stored: the scan keeps one histogram per warp over that warp's contiguous key
@@ -575,6 +590,16 @@ bpc_decode_kernel(const DecodeParams p) {
   }
   cp_async_wait<0>();                                        // Gram staging (appending block only) has landed
   __syncthreads();
+  // Weighted scores reach sum_j |A_j| <= 127 G b, which can exceed 16 bits (seven or eight query heads per KV head at
+  // 128 bits, 256-bit codes).  The stored key is then the score key shifted right by ksh (0, 1 or 2, from this query's
+  // own sum), the selection runs on the stored keys as before, and the keys whose stored key equals the threshold are
+  // scored again from their codes to order them by the bits the shift dropped.
+  int ksh = 0;
+  if (MODE == 1) {
+    const int rs = st->rsum;
+    ksh = rs > 0xffff ? (rs > 0x1ffff ? 2 : 1) : 0;
+    ksh = max(ksh, p.key_shift_min);
+  }
   if (eas_local && (tid == 0 || tid == 32)) {                // lower bounds of the block's two range ends in the set
     const int lo_key = min(n, rank * chunk);
     const int bound = tid == 0 ? lo_key : min(n, lo_key + chunk);
@@ -601,8 +626,8 @@ bpc_decode_kernel(const DecodeParams p) {
 #pragma unroll
       for (int u = 0; u < U; ++u) {
         const int key = score_key<W32, NP>(h[u], sg, mk);
-        sc[score_slot(base - c0 + u * nts + tid)] = (uint16_t)key;
-        atomicAdd(&hist[key >> hsh], 1u);
+        sc[score_slot(base - c0 + u * nts + tid)] = (uint16_t)(key >> ksh);
+        atomicAdd(&hist[(key >> ksh) >> hsh], 1u);
       }
     };
     [[maybe_unused]] const int STEP = nts * U;
@@ -682,8 +707,8 @@ bpc_decode_kernel(const DecodeParams p) {
         const int i = i0 + u * nts + tid;
         if (i < c1s) {
           const int key = score_key<W32, NP>(h[u], sg, mk);
-          sc[score_slot(i - c0)] = (uint16_t)key;
-          atomicAdd(&hist[key >> hsh], 1u);
+          sc[score_slot(i - c0)] = (uint16_t)(key >> ksh);
+          atomicAdd(&hist[(key >> ksh) >> hsh], 1u);
         }
       }
     }
@@ -809,8 +834,8 @@ bpc_decode_kernel(const DecodeParams p) {
         for (int pl = 0; pl < NP; ++pl) mk[pl][w] = st->mask[pl][w];
       }
       const int key = score_key<W32, NP>(h, sg, mk);
-      sc[score_slot(n - 1 - c0)] = (uint16_t)key;
-      atomicAdd(&hist[key >> hsh], 1u);
+      sc[score_slot(n - 1 - c0)] = (uint16_t)(key >> ksh);
+      atomicAdd(&hist[(key >> ksh) >> hsh], 1u);
       if (p.dbg_scores != nullptr) p.dbg_scores[(size_t)unit * p.n_max + (n - 1)] = ((2 * key) << cs) - (st->rsum << cs);
     }
   }
@@ -1001,6 +1026,63 @@ bpc_decode_kernel(const DecodeParams p) {
     __syncthreads();
     T_exact = st->T;
   }
+  // exact key of key i of this block's range (weighted scores with shifted keys only)
+  auto exact_key = [&](int i) -> int {
+    const bool is_new = fused && c0 + i == n - 1;            // the key appended by this launch: its code is in shared memory
+    const uint32_t* code = is_new ? st->newcode : cu + (size_t)(c0 + i) * W32;
+    return rescore_key<W32, NP>(code, st->signw, st->mask);
+  };
+  int T_low = 0;
+  if (MODE == 1 && ksh > 0 && kh > 0) {
+    // Stored keys are score keys shifted right by ksh: the class of stored keys equal to the threshold found above is
+    // split once more by the dropped bits (2 or 4 values), from exact scores recomputed for the members of the class
+    // (a handful of keys per block).  Same procedure as for the coarse bin: counts summed across the cluster, the
+    // exact threshold, and the per-block numbers of keys above it and at it.
+    const int FB = 1 << ksh;
+    uint32_t* fine = st->wgt;                                // (32 words the weighted mode does not use otherwise; the array of the
+                                                             //  previous level may still be read by a peer)
+    if (tid < 32) fine[tid] = 0u;
+    __syncthreads();
+    {
+      const int len = c1 - c0;
+      for (int i = tid; i < len; i += NT)
+        if ((int)sc[score_slot(i)] == T_exact) atomicAdd(&fine[exact_key(i) & (FB - 1)], 1u);
+    }
+    cluster.sync();
+    if (warp == 0) {
+      uint32_t fr[BPC_MAX_CLUSTER];
+      uint32_t f = 0;
+#pragma unroll
+      for (int r = 0; r < BPC_MAX_CLUSTER; ++r) {
+        fr[r] = (r < CS && lane < FB) ? cluster.map_shared_rank(fine, r)[lane] : 0u;
+        f += fr[r];
+      }
+      uint32_t incl = f;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_down_sync(0xffffffffu, incl, o);
+        if (lane + o < 32) incl += v;
+      }
+      const uint32_t above = incl - f;
+      const uint32_t need_c = (uint32_t)(kh - st->cnt_gt);    // keys still to take from the class (>= 1)
+      const bool mine = above < need_c && above + f >= need_c;
+      const int vstar = __ffs(__ballot_sync(0xffffffffu, mine)) - 1;
+      const uint32_t above_star = __shfl_sync(0xffffffffu, above, vstar);
+#pragma unroll
+      for (int r = 0; r < BPC_MAX_CLUSTER; ++r) {
+        if (r < CS) {
+          uint32_t g = lane > vstar ? fr[r] : 0u;
+#pragma unroll
+          for (int o = 16; o >= 1; o >>= 1) g += __shfl_xor_sync(0xffffffffu, g, o);
+          const uint32_t e = __shfl_sync(0xffffffffu, fr[r], vstar);
+          if (lane == 0) { st->gt[r] += g; st->eq[r] = e; }
+        }
+      }
+      if (lane == 0) { st->e0 = vstar; st->cnt_gt += (int)above_star; }   // (e0 is free here: the safeguard is Hamming-only)
+    }
+    __syncthreads();
+    T_low = st->e0;
+  }
   if (!kFastOnly && !fast_sel && tid == 0) {
     const int need = kh - st->cnt_gt;                        // ties to take, cluster-wide (>= 1)
     int tie_base = 0, out_base = 0;
@@ -1129,6 +1211,11 @@ bpc_decode_kernel(const DecodeParams p) {
             const int j = __ffs(rem) - 1;
             rem &= rem - 1;
             if ((int)sc[(size_t)seg * kSegSlots + j] > T) mg |= 1u << j;
+            else if (MODE == 1 && ksh > 0) {                 // stored key == threshold: the dropped bits decide
+              const int low = exact_key(seg * kSegKeys + j) & ((1 << ksh) - 1);
+              if (low > T_low) mg |= 1u << j;
+              else if (low < T_low) m &= ~(1u << j);
+            }
           }
           M[q] = m; Mgt[q] = mg;
           cgt += __popc(mg);

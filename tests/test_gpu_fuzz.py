@@ -47,8 +47,6 @@ def test_random_shapes(case, monkeypatch):
     from paper_2608_04405_b200 import binding as B
     H = _harness()
     i, bits, group, dtype, n_kv, batch, n_ctx, ragged, mode, eas, cluster, budget, interleaved, stream, power = case
-    if mode == 1 and 127 * group * bits > 65535:
-        mode = 0                                        # weighted scores would not fit 16 bits: plain Hamming instead
     stream = bool(stream and mode == 0 and eas == 0)      # the streaming selection covers Hamming scores without the safeguard
     spec = CONFIGS[1].scaled(name="fuzz%d" % i, wid=200 + i, batch=batch, n_kv_heads=n_kv, n_q_heads=n_kv * group, n_ctx=n_ctx,
                              n_ctx_min=max(1, n_ctx // 5) if ragged else None, dtype=dtype, code_bits=bits, steps=2,

@@ -231,11 +231,43 @@ def test_weighted_scores_seven_magnitude_planes(bits, group, dtype, n):
     print(rep)
 
 
-def test_weighted_scores_reject_shapes_whose_scores_exceed_16_bits():
+@pytest.mark.parametrize("bits,group,n,shift,cluster", [(128, 7, 9000, 0, 0), (128, 8, 20000, 0, 3), (256, 4, 6000, 0, 0),
+                                                        (256, 8, 12000, 0, 2), (128, 4, 9000, 2, 0), (64, 8, 7000, 1, 4),
+                                                        (128, 7, 40000, 2, 5)])
+def test_weighted_scores_wider_than_16_bits(bits, group, n, shift, cluster):
+    """Algorithm 3's score where 127 * G * b exceeds 16 bits (seven or eight query heads per KV head at 128 bits: the
+    28/4 and 70B-style head layouts; 256-bit codes): the stored keys are shifted right and the keys at the threshold are
+    re-scored exactly, so scores, index sets (lowest-index ties) and outputs must equal the checker's as for any other
+    shape.  The shift is also forced (diagnostic switch) on shapes that would not need it, where many more keys share a
+    stored key and the re-scoring decides most of the ties; several cluster sizes; separate calls and the fused call;
+    a dense budget and a single key."""
+    H = _harness()
     from paper_2608_04405_b200 import binding as B
-    with pytest.raises(B.BpcError) as e:
-        B.Context(B.make_config(1, 28, 4, 4096, 128, torch.bfloat16, score_mode=B.BPC_SCORE_WEIGHTED7))   # 127*7*128
-    assert e.value.status == 2
+    spec = CONFIGS[1].scaled(name="w7wide", wid=70 + group, n_ctx=n, n_kv_heads=2, n_q_heads=2 * group, code_bits=bits, steps=2)
+    sess = H.Session(spec, gen_device="cuda", score_mode=B.BPC_SCORE_WEIGHTED7, cluster_size=cluster)
+    if shift:
+        sess.ctx.debug_force_key_shift(shift)
+    rep = {}
+    sess.fit(); sess.encode()
+    _decode_loop(sess, 2, [0, 1], rep, H)
+    q, _ = sess.w.queries(sess.lens)
+    for ppm in (1000, 100000, 1000000):
+        H.check_decode(sess, q.cuda(), [0, 1], rep, budget_ppm=ppm)
+    H.check_decode(sess, q.cuda(), [1], rep, budget_ppm=0, budget_count=1)
+    print(rep)
+
+
+def test_weighted_scores_config4_head_layout_full_size():
+    """Configuration 4's shape (28/4 heads: seven query heads per KV head, 128-bit codes, 131072 keys) with the paper's
+    weighted score: 127 * 7 * 128 needs 17 bits.  One sequence of the batch at full length, sampled units."""
+    H = _harness()
+    from paper_2608_04405_b200 import binding as B
+    spec = CONFIGS[4].scaled(batch=1, steps=2)
+    sess = H.Session(spec, gen_device="cuda", score_mode=B.BPC_SCORE_WEIGHTED7)
+    rep = {}
+    sess.fit(); sess.encode()
+    _decode_loop(sess, 2, [0, 3], rep, H)
+    print(rep)
 
 
 @pytest.mark.parametrize("bits", [64, 128])
