@@ -1,18 +1,24 @@
 // Tensor-core encode: Algorithm 2 for all cached keys of bf16 caches.
 //
 // The decision values before any correction are a dense contraction T = K P_h^T (keys x channels times
-// channels x bits).  It runs on the 5th-generation tensor cores: per block, tiles of 128 keys (M = 128) against
-// the unit's b projection rows (N = b, 64 or 128) over the 128 channels (eight tcgen05.mma steps of K = 16), bf16
+// channels x bits).  It runs on the 5th-generation tensor cores: per warpgroup, tiles of 128 keys (M = 128) against
+// the unit's b projection rows (N = b: 32, 64 or 128) over the 128 channels (eight tcgen05.mma steps of K = 16), bf16
 // operands in shared memory in the 128-byte-swizzled K-major layout, fp32 accumulator in tensor memory with one
-// key per TMEM lane.  Each of the 128 threads of a warpgroup then pulls its key's b decision values out of tensor
-// memory (tcgen05.ld) into registers and runs the greedy sweep of Algorithm 2 in its Gram form
+// key per TMEM lane.  Algorithm 2's greedy sweep in its Gram form,
 //     u_i = sign(t_i);  t_j -= u_i * G_ij  (j > i),   G = P_h P_h^T,
-// which equals updating the residual r <- r - u_i P_i and testing r . P_{i+1}.  While the threads sweep tile i,
-// the asynchronous copy of tile i+1 is already in flight.  A block holds two such warpgroups, which share the
-// projection rows and the Gram matrix in shared memory and otherwise run independent pipelines, and every warpgroup
-// works on two key tiles at once, one key of each per thread: the sweep is a chain of dependent FMAs per key fed by
-// broadcast reads of the Gram matrix, so one warp per scheduler cannot keep the FP32 pipe busy, and with one key per
-// thread the shared-memory reads (one 16-byte read per four FMAs) bound it.
+// (equal to updating the residual r <- r - u_i P_i and testing r . P_{i+1}) is blocked by 32 bits.  Inside a block the
+// 32 sign decisions are sequential: each thread pulls its key's 32 decision values out of tensor memory (tcgen05.ld)
+// and sweeps them in registers (496 FMAs).  The corrections of all LATER blocks by those 32 signs are again a dense
+// contraction, T[:, later] -= U (128 keys x 32 signs) G[block, later], and go to the tensor cores too: the signs are
+// written to shared memory as a bf16 operand (+-1 is exact), the Gram rows are kept as three bf16 terms whose sum
+// carries 24 mantissa bits (so the products are exact and the fp32 accumulation in tensor memory sees what an fp32
+// FMA chain would see up to rounding), and six small MMAs (three terms x two K = 16 steps) accumulate straight into
+// the accumulator columns that still wait for their decisions.  That leaves 1 984 of the 8 128 sign-dependent FMAs per
+// key (128 bits) on the CUDA cores.  The small operands use the K-major layout without swizzle (8-row x 16-byte core
+// matrices; leading-dimension offset = distance between core matrices along K, stride offset = 128 bytes along M/N).
+// A block holds two warpgroups, which share the projection rows and the Gram operands in shared memory and otherwise
+// run independent pipelines (own key tile, own accumulator columns, own mbarrier, own hardware barrier), so one
+// warpgroup's sweep covers the other's MMA round trips; the next key tile of a warpgroup is copied in while it sweeps.
 //
 // Waits on the MMA-completion mbarrier are bounded: on expiry the block raises the device error word, still
 // releases its tensor memory and returns.
@@ -24,8 +30,7 @@ namespace {
 constexpr int kTileKeys = 128;
 constexpr int kGroupThreads = 128;   // one warpgroup sweeps one key tile (a TMEM lane per thread)
 constexpr int kGroups = 2;           // warpgroups per block, each with its own tiles, accumulator columns and barrier
-constexpr int kPair = 2;             // key tiles a warpgroup sweeps together, one key of each per thread: every Gram
-                                     // value read from shared memory then feeds two FMAs (the loads bound the sweep)
+constexpr int kPair = 1;             // key tiles a warpgroup sweeps together (one key of each per thread)
 constexpr int kThreads = kGroupThreads * kGroups;
 
 __device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
@@ -47,6 +52,19 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(const void* smem_ptr) {
   d |= (uint64_t)1 << 46;                  // bits [46,48): descriptor version of this architecture
   d |= (uint64_t)2 << 61;                  // bits [61,64): 128-byte swizzle
   return d;
+}
+// Shared-memory operand descriptor: K-major without swizzle.  Core matrices are 8 rows x 16 bytes, stored contiguously
+// (128 bytes); lbo = bytes between core matrices adjacent along K, sbo = bytes between core matrices adjacent along M/N.
+__device__ __forceinline__ uint64_t umma_desc_nosw(const void* smem_ptr, unsigned lbo, unsigned sbo) {
+  uint64_t d = (uint64_t)(smem_u32(smem_ptr) & 0x3FFFF) >> 4;
+  d |= (uint64_t)(lbo >> 4) << 16;
+  d |= (uint64_t)(sbo >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  return d;
+}
+// byte offset of element (row r, k) of an [R x 32] bf16 operand in that layout (core matrices of one K chunk contiguous)
+__device__ __forceinline__ size_t nosw_offset(int R, int r, int k) {
+  return (size_t)(k >> 3) * ((size_t)(R >> 3) * 128) + (size_t)(r >> 3) * 128 + (size_t)(r & 7) * 16 + (size_t)(k & 7) * 2;
 }
 // Instruction descriptor: D fp32, A and B bf16, both K-major, N and M.
 __device__ __forceinline__ uint32_t umma_idesc_bf16(int m, int n) {
@@ -137,18 +155,25 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
   extern __shared__ __align__(16) unsigned char smem_raw[];
   // the swizzled operand tiles need 1024-byte alignment in the shared address space
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  constexpr int NB = NBITS / 32;                           // 32-bit column blocks
   constexpr int A_BYTES = kTileKeys * 256;                 // one key tile (128 rows x 128 bf16)
   constexpr int B_BYTES = NBITS * 256;                     // the projection rows
+  constexpr int GD_BYTES = NB * 32 * 32 * 4;               // diagonal 32 x 32 blocks of the Gram matrix, fp32
+  constexpr int U_BYTES = kTileKeys * 64;                  // the 32 signs of one block for 128 keys, bf16 operand [128 x 32]
+  constexpr int GB_PART = NBITS * 64;                      // one bf16 term of -G[block rows][all columns], operand [NBITS x 32]
+  constexpr unsigned U_LBO = (kTileKeys / 8) * 128, GB_LBO = (NBITS / 8) * 128;   // bytes between core matrices along K
   const int tid = threadIdx.x, warp = tid >> 5;
   const int grp = tid / kGroupThreads, gtid = tid % kGroupThreads;   // warpgroup and thread within it
-  unsigned char* a_t = smem + (size_t)(grp * kPair) * A_BYTES;   // this warpgroup's kPair key tiles (one buffer each: see the loop)
-  unsigned char* b_s = smem + kGroups * kPair * A_BYTES;
-  float* g_s = reinterpret_cast<float*>(smem + kGroups * kPair * A_BYTES + B_BYTES);   // [NBITS][NBITS]
+  unsigned char* a_t = smem + (size_t)grp * A_BYTES;       // this warpgroup's key tile (one buffer: see the loop)
+  unsigned char* b_s = smem + kGroups * A_BYTES;
+  float* gd_s = reinterpret_cast<float*>(b_s + B_BYTES);   // [NB][32][32]
+  unsigned char* u_s = reinterpret_cast<unsigned char*>(gd_s) + GD_BYTES + (size_t)grp * U_BYTES;
+  unsigned char* gb_s = reinterpret_cast<unsigned char*>(gd_s) + GD_BYTES + kGroups * U_BYTES;   // [NB-1][3][NBITS x 32]
   __shared__ unsigned long long mma_bar_s[kGroups];
   __shared__ uint32_t tmem_base_s;
   __shared__ int timed_out_g[kGroups];
   unsigned long long* mma_bar = &mma_bar_s[grp];
-  constexpr int kAccCols = kGroups * kPair * NBITS;        // fp32 accumulator columns of all tiles in flight
+  constexpr int kAccCols = kGroups * NBITS;                // fp32 accumulator columns of the tiles in flight
   constexpr int kTmemCols = kAccCols <= 32 ? 32 : kAccCols <= 64 ? 64 : kAccCols <= 128 ? 128 : kAccCols <= 256 ? 256 : 512;   // a power of two >= 32
   static_assert(kAccCols <= 512, "accumulators exceed tensor memory");
 
@@ -157,7 +182,7 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
   const int ntiles = (n + kTileKeys - 1) / kTileKeys;
   const int set = shared_sets ? unit % n_kv_heads : unit;
 
-  // ---- one-time set-up: barrier, tensor memory, projection and Gram matrix in shared memory
+  // ---- one-time set-up: barrier, tensor memory, projection and Gram operands in shared memory
   if (tid == 0) {
     for (int g = 0; g < kGroups; ++g) { mbar_init(&mma_bar_s[g], 1); timed_out_g[g] = 0; }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -172,173 +197,173 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
       const int r = c >> 4, ch = c & 15;
       *reinterpret_cast<uint4*>(b_s + sw128_offset(NBITS, r, ch)) = *reinterpret_cast<const uint4*>(psrc + (size_t)r * 256 + ch * 16);
     }
-    const float4* gsrc = reinterpret_cast<const float4*>(gram + (size_t)set * NBITS * NBITS);
-    for (int c = tid; c < NBITS * NBITS / 4; c += kThreads) reinterpret_cast<float4*>(g_s)[c] = gsrc[c];
+    const float* gsrc = gram + (size_t)set * NBITS * NBITS;
+    for (int c = tid; c < NB * 32 * 32; c += kThreads) {     // diagonal blocks, kept in fp32 for the in-register sweep
+      const int d = c >> 10, i = (c >> 5) & 31, j = c & 31;
+      gd_s[c] = gsrc[(size_t)(32 * d + i) * NBITS + 32 * d + j];
+    }
+    // -G[32 pb + i][j] as three bf16 terms (g = t1 + t2 + t3 up to 2^-24 |g|), operand rows j, K index i
+    for (int c = tid; c < (NB - 1) * 32 * NBITS; c += kThreads) {
+      const int pb = c / (32 * NBITS), i = (c / NBITS) & 31, j = c % NBITS;
+      const float g = -gsrc[(size_t)(32 * pb + i) * NBITS + j];
+      const __nv_bfloat16 t1 = __float2bfloat16_rn(g);
+      const float r1 = g - __bfloat162float(t1);
+      const __nv_bfloat16 t2 = __float2bfloat16_rn(r1);
+      const __nv_bfloat16 t3 = __float2bfloat16_rn(r1 - __bfloat162float(t2));
+      unsigned char* base = gb_s + (size_t)pb * 3 * GB_PART + nosw_offset(NBITS, j, i);
+      *reinterpret_cast<__nv_bfloat16*>(base) = t1;
+      *reinterpret_cast<__nv_bfloat16*>(base + GB_PART) = t2;
+      *reinterpret_cast<__nv_bfloat16*>(base + 2 * GB_PART) = t3;
+    }
   }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the tensor core
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_all = tmem_base_s;
-  const uint32_t tmem_base = tmem_all + (uint32_t)(grp * kPair * NBITS);   // this warpgroup's accumulator columns (tile q at + q * NBITS)
+  const uint32_t tmem_base = tmem_all + (uint32_t)(grp * NBITS);   // this warpgroup's accumulator columns
   float trace_g = 0.f;
   if (key_err != nullptr)
-    for (int i = 0; i < NBITS; ++i) trace_g += g_s[i * NBITS + i];
+    for (int i = 0; i < NBITS; ++i) trace_g += gd_s[(i >> 5) * 1024 + (i & 31) * 33];
 
   const unsigned char* kbase = reinterpret_cast<const unsigned char*>(k_cache) + (size_t)unit * n_max * (size_t)row_stride * 2;
-  auto load_tile = [&](int tile, unsigned char* dst) {
+  auto load_tile = [&](int tile) {                           // rows past n are zero-filled
     const int r0 = tile * kTileKeys;
     for (int c = gtid; c < kTileKeys * 16; c += kGroupThreads) {
       const int r = c >> 4, ch = c & 15;
-      unsigned char* d = dst + sw128_offset(kTileKeys, r, ch);
+      unsigned char* d = a_t + sw128_offset(kTileKeys, r, ch);
       if (r0 + r < n) cp_async16(d, kbase + (size_t)(r0 + r) * row_stride * 2 + ch * 16);
       else *reinterpret_cast<uint4*>(d) = make_uint4(0u, 0u, 0u, 0u);
     }
     cp_async_commit();
   };
   const uint32_t idesc = umma_idesc_bf16(kTileKeys, NBITS);
-  auto issue_mma = [&]() {                                  // one thread: per tile 8 steps of K = 16 over the 128 channels
+  auto issue_gemm = [&]() {                                 // one thread: 8 steps of K = 16 over the 128 channels
 #pragma unroll
-    for (int q = 0; q < kPair; ++q) {
-#pragma unroll
-      for (int ks = 0; ks < 8; ++ks) {
-        const size_t aoff = (size_t)q * A_BYTES + (size_t)(ks >> 2) * (kTileKeys * 128) + (size_t)(ks & 3) * 32;
-        const size_t boff = (size_t)(ks >> 2) * (NBITS * 128) + (size_t)(ks & 3) * 32;
-        umma_bf16(tmem_base + (uint32_t)(q * NBITS), umma_desc_sw128(a_t + aoff), umma_desc_sw128(b_s + boff), idesc, ks > 0 ? 1u : 0u);
-      }
+    for (int ks = 0; ks < 8; ++ks) {
+      const size_t aoff = (size_t)(ks >> 2) * (kTileKeys * 128) + (size_t)(ks & 3) * 32;
+      const size_t boff = (size_t)(ks >> 2) * (NBITS * 128) + (size_t)(ks & 3) * 32;
+      umma_bf16(tmem_base, umma_desc_sw128(a_t + aoff), umma_desc_sw128(b_s + boff), idesc, ks > 0 ? 1u : 0u);
     }
     umma_commit(mma_bar);                                    // arrives when all MMAs issued so far have completed
   };
-  auto load_pair = [&](int pr) {                             // tiles kPair * pr + q; rows past n are zero-filled
+  // corrections of the columns after block pb by the block's 32 signs: T[:, j0..] += U x (-G[block rows, j0..]),
+  // three bf16 terms x two K steps, accumulated into the columns that still wait for their decisions
+  auto issue_corrections = [&](int pb) {
+    const int j0 = 32 * (pb + 1);
+    const uint32_t idc = umma_idesc_bf16(kTileKeys, NBITS - j0);
 #pragma unroll
-    for (int q = 0; q < kPair; ++q) load_tile(kPair * pr + q, a_t + (size_t)q * A_BYTES);
+    for (int part = 0; part < 3; ++part) {
+#pragma unroll
+      for (int ks = 0; ks < 2; ++ks) {
+        const unsigned char* ap = u_s + (size_t)ks * 2 * U_LBO;
+        const unsigned char* bp = gb_s + (size_t)(pb * 3 + part) * GB_PART + (size_t)(j0 >> 3) * 128 + (size_t)ks * 2 * GB_LBO;
+        umma_bf16(tmem_base + (uint32_t)j0, umma_desc_nosw(ap, U_LBO, 128), umma_desc_nosw(bp, GB_LBO, 128), idc, 1u);
+      }
+    }
+    umma_commit(mma_bar);
   };
 
-  // Tile pairs of this warpgroup: kGroups * blockIdx.x + grp, then every kGroups * blocks_per_unit-th.  The warpgroups
-  // run independent pipelines (own tiles, own accumulator columns, own MMA barrier, own hardware barrier); all threads
+  // Tiles of this warpgroup: kGroups * blockIdx.x + grp, then every kGroups * blocks_per_unit-th.  The warpgroups
+  // run independent pipelines (own tile, own accumulator columns, own MMA barrier, own hardware barrier); all threads
   // of a warpgroup take the same branches, so its barrier is always reached by all 128 of them.
-  const int npairs = (ntiles + kPair - 1) / kPair;
-  const int pair_step = kGroups * blocks_per_unit;
-  int pr = kGroups * blockIdx.x + grp;
-  int it = 0;
-  if (pr < npairs) {
-    load_pair(pr);
+  const int tile_step = kGroups * blocks_per_unit;
+  int tl = kGroups * blockIdx.x + grp;
+  unsigned ph = 0;                                           // phase of the MMA barrier the next wait refers to
+  if (tl < ntiles) {
+    load_tile(tl);
     cp_async_wait_all();
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the tensor core
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     group_sync(grp);
     if (gtid == 0) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      issue_mma();
+      issue_gemm();
     }
   }
-  for (; pr < npairs; pr += pair_step, ++it) {
-    const int next = pr + pair_step;
-    // decision values of these tiles: wait for the MMAs, then one TMEM lane (one key of each tile) per thread
-    bool ok = mbar_wait(mma_bar, (unsigned)(it & 1));
-    if (!ok) timed_out_g[grp] = 1;
+  for (; tl < ntiles; tl += tile_step) {
+    const int next = tl + tile_step;
+    // decision values of this tile: wait for the MMAs, then one TMEM lane (one key) per thread
+    if (!mbar_wait(mma_bar, ph)) timed_out_g[grp] = 1;
+    ph ^= 1u;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    // The MMAs are the only readers of the key tiles (besides the key norms below), and they have completed: the
-    // buffers are refilled with the warpgroup's next tiles right away, under the sweep, which is many times longer
-    // than the copy.
-    int key[kPair];
-    float k2[kPair];
+    // The MMAs are the only readers of the key tile (besides the key norms below), and they have completed: the
+    // buffer is refilled with the warpgroup's next tile right away, under the sweep.
+    const int key = tl * kTileKeys + gtid;
+    float k2 = 0.f;
+    if (key_err != nullptr) {                                // squared norm of this thread's key, from the operand tile
+      if (key < n) {
 #pragma unroll
-    for (int q = 0; q < kPair; ++q) { key[q] = (kPair * pr + q) * kTileKeys + gtid; k2[q] = 0.f; }
-    if (key_err != nullptr) {                                // squared norms of this thread's keys, from the operand tiles
-#pragma unroll
-      for (int q = 0; q < kPair; ++q) {
-        if (key[q] < n) {
-#pragma unroll
-          for (int ch = 0; ch < 16; ++ch) {
-            const uint4 w = *reinterpret_cast<const uint4*>(a_t + (size_t)q * A_BYTES + sw128_offset(kTileKeys, gtid, ch));
-            const float f0 = bf16_lo(w.x), f1 = bf16_hi(w.x), f2 = bf16_lo(w.y), f3 = bf16_hi(w.y);
-            const float f4 = bf16_lo(w.z), f5 = bf16_hi(w.z), f6 = bf16_lo(w.w), f7 = bf16_hi(w.w);
-            k2[q] += (f0 * f0 + f1 * f1) + (f2 * f2 + f3 * f3) + (f4 * f4 + f5 * f5) + (f6 * f6 + f7 * f7);
-          }
+        for (int ch = 0; ch < 16; ++ch) {
+          const uint4 w = *reinterpret_cast<const uint4*>(a_t + sw128_offset(kTileKeys, gtid, ch));
+          const float f0 = bf16_lo(w.x), f1 = bf16_hi(w.x), f2 = bf16_lo(w.y), f3 = bf16_hi(w.y);
+          const float f4 = bf16_lo(w.z), f5 = bf16_hi(w.z), f6 = bf16_lo(w.w), f7 = bf16_hi(w.w);
+          k2 += (f0 * f0 + f1 * f1) + (f2 * f2 + f3 * f3) + (f4 * f4 + f5 * f5) + (f6 * f6 + f7 * f7);
         }
       }
-      group_sync(grp);                                       // every thread has read its rows before the refill starts
+      group_sync(grp);                                       // every thread has read its row before the refill starts
     }
-    if (next < npairs) load_pair(next);
+    if (next < ntiles) load_tile(next);
     const uint32_t taddr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);   // a warp reaches the lanes of its quarter
-    // Column blocks of 32 bits: pull the block out of tensor memory, apply the corrections of all earlier
-    // bits (t_j -= u_i G_ij, G rows are broadcast reads from shared memory), then sweep the block itself.
-    uint32_t words[kPair][NBITS / 32];
-    float abs_sum[kPair];                                    // sum of |t_i| at decision time (for Eq. 8)
+    uint32_t words[NB];
+    float abs_sum[kPair] = {0.f};                            // sum of |t_i| at decision time (for Eq. 8)
 #pragma unroll
-    for (int q = 0; q < kPair; ++q) {
-      abs_sum[q] = 0.f;
-#pragma unroll
-      for (int w = 0; w < NBITS / 32; ++w) words[q][w] = 0u;
-    }
-#pragma unroll 1
-    for (int cb = 0; cb < NBITS / 32; ++cb) {
-      float t[kPair][32];
-#pragma unroll
-      for (int q = 0; q < kPair; ++q) tmem_ld32<0>(taddr + (uint32_t)(q * NBITS + 32 * cb), t[q]);
-      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-      if (residual_correction) {
-#pragma unroll 1
-        for (int pb = 0; pb < cb; ++pb) {
-          uint32_t wprev[kPair];                             // words[q][pb], selected without indexing registers
-#pragma unroll
-          for (int q = 0; q < kPair; ++q) {
-            wprev[q] = words[q][0];
-#pragma unroll
-            for (int w = 1; w < NBITS / 32; ++w) wprev[q] = pb == w ? words[q][w] : wprev[q];
-          }
-#pragma unroll 4
-          for (int i = 0; i < 32; ++i) {
-            float mu[kPair];                                 // minus the sign of bit 32 pb + i
-#pragma unroll
-            for (int q = 0; q < kPair; ++q) mu[q] = ((wprev[q] >> i) & 1u) ? -1.f : 1.f;
-            const float4* gi = reinterpret_cast<const float4*>(g_s + (size_t)(32 * pb + i) * NBITS + 32 * cb);
-#pragma unroll
-            for (int j4 = 0; j4 < 8; ++j4) {
-              const float4 gv = gi[j4];
-#pragma unroll
-              for (int q = 0; q < kPair; ++q) {
-                t[q][4 * j4] = fmaf(mu[q], gv.x, t[q][4 * j4]);
-                t[q][4 * j4 + 1] = fmaf(mu[q], gv.y, t[q][4 * j4 + 1]);
-                t[q][4 * j4 + 2] = fmaf(mu[q], gv.z, t[q][4 * j4 + 2]);
-                t[q][4 * j4 + 3] = fmaf(mu[q], gv.w, t[q][4 * j4 + 3]);
-              }
-            }
-          }
-        }
+    for (int cb = 0; cb < NB; ++cb) {
+      if (cb > 0 && residual_correction) {                   // the corrections by block cb - 1 (and all before it) have landed
+        if (!mbar_wait(mma_bar, ph)) timed_out_g[grp] = 1;
+        ph ^= 1u;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       }
-      uint32_t word[kPair];
+      float t[kPair][32];
+      tmem_ld32<0>(taddr + (uint32_t)(32 * cb), t[0]);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      uint32_t word[kPair] = {0u};
+      DiagSweep<0>::run(t, word, abs_sum, gd_s + (size_t)cb * 1024, 32, residual_correction);
+      words[cb] = word[0];
+      if (cb + 1 < NB && residual_correction) {
+        // this key's 32 signs as a row of the bf16 operand U (+1 = 0x3F80, -1 = 0xBF80), 8 per 16-byte chunk
 #pragma unroll
-      for (int q = 0; q < kPair; ++q) word[q] = 0u;
-      DiagSweep<0>::run(t, word, abs_sum, g_s + (size_t)(32 * cb) * NBITS + 32 * cb, NBITS, residual_correction);
+        for (int c = 0; c < 4; ++c) {
+          uint32_t h[4];
 #pragma unroll
-      for (int q = 0; q < kPair; ++q) {
-#pragma unroll
-        for (int w = 0; w < NBITS / 32; ++w) words[q][w] = cb == w ? word[q] : words[q][w];
+          for (int e = 0; e < 4; ++e) {
+            const uint32_t lo = ((word[0] >> (8 * c + 2 * e)) & 1u) ? 0x3F80u : 0xBF80u;
+            const uint32_t hi = ((word[0] >> (8 * c + 2 * e + 1)) & 1u) ? 0x3F80u : 0xBF80u;
+            h[e] = lo | (hi << 16);
+          }
+          *reinterpret_cast<uint4*>(u_s + (size_t)c * U_LBO + (size_t)(gtid >> 3) * 128 + (size_t)(gtid & 7) * 16) =
+              make_uint4(h[0], h[1], h[2], h[3]);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        group_sync(grp);                                     // all 128 rows of U are written (and the block's TMEM reads are done)
+        if (gtid == 0) {
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          issue_corrections(cb);
+        }
       }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    if (next < npairs) {
+    if (next < ntiles) {
       cp_async_wait_all();
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    group_sync(grp);                                         // the accumulators have been read by the whole warpgroup; its next tiles have landed
+    group_sync(grp);                                         // the accumulators have been read by the whole warpgroup; its next tile has landed
     if (timed_out_g[grp]) break;                             // (written only by this warpgroup, before the barrier)
-    if (next < npairs && gtid == 0) {
+    if (next < ntiles && gtid == 0) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      issue_mma();
+      issue_gemm();
     }
+    // squared reconstruction error (Eq. 8) from the sweep: ||k - hP||^2 = ||k||^2 - 2 sum|t_i| + trace(G)
+    if (key_err != nullptr && key < n) key_err[(size_t)unit * n_max + key] = fmaxf(0.f, k2 - 2.f * abs_sum[0] + trace_g);
+    if (key < n) {
+      uint32_t* dst = reinterpret_cast<uint32_t*>(codes) + ((size_t)unit * n_max + key) * NB;
+      if (NB == 1) {
+        dst[0] = words[0];
+      } else if (NB == 2) {
+        *reinterpret_cast<uint2*>(dst) = make_uint2(words[0], words[1]);
+      } else {
 #pragma unroll
-    for (int q = 0; q < kPair; ++q) {
-      // squared reconstruction error (Eq. 8) from the sweep: ||k - hP||^2 = ||k||^2 - 2 sum|t_i| + trace(G)
-      if (key_err != nullptr && key[q] < n) key_err[(size_t)unit * n_max + key[q]] = fmaxf(0.f, k2[q] - 2.f * abs_sum[q] + trace_g);
-      if (key[q] < n) {
-        uint32_t* dst = reinterpret_cast<uint32_t*>(codes + ((size_t)unit * n_max + key[q]) * (NBITS / 64));
-        if (NBITS == 64) {
-          *reinterpret_cast<uint2*>(dst) = make_uint2(words[q][0], words[q][1]);
-        } else {
-#pragma unroll
-          for (int w = 0; w < NBITS / 32; w += 4) *reinterpret_cast<uint4*>(dst + w) = make_uint4(words[q][w], words[q][w + 1], words[q][w + 2], words[q][w + 3]);
-        }
+        for (int w = 0; w + 3 < NB; w += 4) *reinterpret_cast<uint4*>(dst + w) = make_uint4(words[w], words[w + 1], words[w + 2], words[w + 3]);
       }
     }
   }
@@ -354,14 +379,15 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
 template <int NBITS>
 cudaError_t launch(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStream_t stream) {
   const bpc_config& c = ctx->cfg;
-  const size_t smem = (size_t)kGroups * kPair * kTileKeys * 256 + (size_t)NBITS * 256 + (size_t)NBITS * NBITS * 4 + 1024;
+  constexpr int NB = NBITS / 32;
+  const size_t smem = (size_t)kGroups * kTileKeys * 256 + (size_t)NBITS * 256 + (size_t)NB * 4096 + (size_t)kGroups * kTileKeys * 64 +
+                      (size_t)(NB - 1) * 3 * NBITS * 64 + 1024;
   cudaError_t e = cudaFuncSetAttribute(encode_tc_kernel<NBITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  const int tiles_max = ((c.n_max + kTileKeys - 1) / kTileKeys + kGroups * kPair - 1) / (kGroups * kPair);   // a block takes kGroups * kPair tiles at a time
+  const int tiles_max = ((c.n_max + kTileKeys - 1) / kTileKeys + kGroups - 1) / kGroups;   // a block takes kGroups tiles at a time
   // Blocks per unit.  One block fits an SM (shared memory), so the grid runs in waves of sm_count blocks and a last,
   // partly filled wave costs as much as a full one: starting from about four waves, take the first count whose last
-  // wave is at least 90 % full (32 units on 148 SMs: 23 blocks per unit = 736 blocks = 4.97 waves; the 10 used before
-  // gave 2.16 waves, i.e. three rounds for two rounds' worth of work).
+  // wave is at least 90 % full (32 units on 148 SMs: 23 blocks per unit = 736 blocks = 4.97 waves).
   int bpu = (4 * ctx->sm_count + ctx->units - 1) / ctx->units;
   if (bpu < 1) bpu = 1;
   for (int tries = 0; tries < 16; ++tries) {
@@ -379,14 +405,15 @@ cudaError_t launch(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStrea
 
 }  // namespace
 
-// bf16 caches with 64- or 128-bit codes run on the tensor cores; other shapes report "not supported" and the
-// caller falls back to the CUDA-core kernel (fp32 caches have no bf16 operands; at 256 bits the Gram matrix no
-// longer fits next to the operands in shared memory).
+// bf16 caches with 32-, 64- or 128-bit codes run on the tensor cores; other shapes report "not supported" and the
+// caller falls back to the CUDA-core kernel (fp32 caches have no bf16 operands; at 256 bits the bf16 terms of the Gram
+// matrix, 336 KB, do not fit shared memory next to the operands).
 cudaError_t bpc_launch_encode_tc(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStream_t stream) {
   if (ctx->cfg.kv_dtype != BPC_BF16) return cudaErrorNotSupported;
   if (ctx->no_tc_encode) return cudaErrorNotSupported;     // diagnostic switch: the CUDA-core kernel is asked for
   cudaError_t e;
-  if (ctx->cfg.code_bits == 64) e = launch<64>(ctx, k_cache, codes, stream);
+  if (ctx->cfg.code_bits == 32) e = launch<32>(ctx, k_cache, codes, stream);
+  else if (ctx->cfg.code_bits == 64) e = launch<64>(ctx, k_cache, codes, stream);
   else if (ctx->cfg.code_bits == 128) e = launch<128>(ctx, k_cache, codes, stream);
   else return cudaErrorNotSupported;
   if (e == cudaSuccess) ctx->launches += 1;
