@@ -548,7 +548,11 @@ def run_ours(args):
                          "fused_step_with_error_aware_safeguard": ms_eas * 1e3},
         "prefill": {"fit_ms": fit_ms, "fit_power2_ms": fit_power2_ms, "encode_ms": enc_ms, "encode_keys_per_s": n_keys / (enc_ms * 1e-3),
                     "encode_gemm_tflops": enc_flops / (enc_ms * 1e-3) / 1e12,
-                    "encode_frac_of_bf16_peak": enc_flops / (enc_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]},
+                    "encode_frac_of_bf16_peak": enc_flops / (enc_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                    # the encode reads every key row once and writes one code per key
+                    "encode_algorithmic_bytes": n_keys * (spec.head_dim * spec.esz + spec.code_bits // 8),
+                    "encode_hbm_gbs": n_keys * (spec.head_dim * spec.esz + spec.code_bits // 8) / (enc_ms * 1e-3) / 1e9,
+                    "encode_frac_of_hbm_peak": n_keys * (spec.head_dim * spec.esz + spec.code_bits // 8) / (enc_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
         "device_error_word": err,
         "needle_recall": hits / max(1, total_needles),
         "paper_context": "paper reports up to 3.56x end-to-end decode speed-up over FlashAttention-2 on 8 data-center GPUs "

@@ -29,7 +29,7 @@ namespace {
 
 constexpr int kTileKeys = 128;
 constexpr int kGroupThreads = 128;   // one warpgroup sweeps one key tile (a TMEM lane per thread)
-constexpr int kGroups = 2;           // warpgroups per block, each with its own tiles, accumulator columns and barrier
+constexpr int kGroups = 3;           // warpgroups per block, each with its own tile, accumulator columns and barrier
 constexpr int kPair = 1;             // key tiles a warpgroup sweeps together (one key of each per thread)
 constexpr int kThreads = kGroupThreads * kGroups;
 
@@ -124,12 +124,19 @@ struct DiagSweep {
       u[q] = pos ? 1.f : -1.f;
     }
     if (rc) {
-      const float* gi = g_diag + I * ld;
+      // row I of the diagonal block, columns after I: 16-byte broadcast reads (the reads, not the FMAs, bound the sweep)
+      const float4* gi4 = reinterpret_cast<const float4*>(g_diag + I * ld);
 #pragma unroll
-      for (int j = I + 1; j < 32; ++j) {
-        const float g = gi[j];
+      for (int j4 = (I + 1) / 4; j4 < 8; ++j4) {
+        const float4 gv = gi4[j4];
+        const float ge[4] = {gv.x, gv.y, gv.z, gv.w};
 #pragma unroll
-        for (int q = 0; q < kPair; ++q) t[q][j] = fmaf(-u[q], g, t[q][j]);
+        for (int e = 0; e < 4; ++e) {
+          if (4 * j4 + e > I) {
+#pragma unroll
+            for (int q = 0; q < kPair; ++q) t[q][4 * j4 + e] = fmaf(-u[q], ge[e], t[q][4 * j4 + e]);
+          }
+        }
       }
     }
     DiagSweep<I + 1>::run(t, word, abs_sum, g_diag, ld, rc);
@@ -160,15 +167,18 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
   constexpr int B_BYTES = NBITS * 256;                     // the projection rows
   constexpr int GD_BYTES = NB * 32 * 32 * 4;               // diagonal 32 x 32 blocks of the Gram matrix, fp32
   constexpr int U_BYTES = kTileKeys * 64;                  // the 32 signs of one block for 128 keys, bf16 operand [128 x 32]
-  constexpr int GB_PART = NBITS * 64;                      // one bf16 term of -G[block rows][all columns], operand [NBITS x 32]
-  constexpr unsigned U_LBO = (kTileKeys / 8) * 128, GB_LBO = (NBITS / 8) * 128;   // bytes between core matrices along K
+  // one bf16 term of -G[rows of block pb][columns after block pb] is an operand [NBITS - 32 (pb + 1) x 32]; the three
+  // terms of block pb start at gb_off(pb)
+  constexpr unsigned U_LBO = (kTileKeys / 8) * 128;        // bytes between core matrices along K
   const int tid = threadIdx.x, warp = tid >> 5;
   const int grp = tid / kGroupThreads, gtid = tid % kGroupThreads;   // warpgroup and thread within it
   unsigned char* a_t = smem + (size_t)grp * A_BYTES;       // this warpgroup's key tile (one buffer: see the loop)
   unsigned char* b_s = smem + kGroups * A_BYTES;
   float* gd_s = reinterpret_cast<float*>(b_s + B_BYTES);   // [NB][32][32]
   unsigned char* u_s = reinterpret_cast<unsigned char*>(gd_s) + GD_BYTES + (size_t)grp * U_BYTES;
-  unsigned char* gb_s = reinterpret_cast<unsigned char*>(gd_s) + GD_BYTES + kGroups * U_BYTES;   // [NB-1][3][NBITS x 32]
+  unsigned char* gb_s = reinterpret_cast<unsigned char*>(gd_s) + GD_BYTES + kGroups * U_BYTES;
+  auto gb_cols = [](int pb) { return NBITS - 32 * (pb + 1); };                     // columns after block pb
+  auto gb_off = [](int pb) { return (size_t)3 * 64 * (size_t)(pb * NBITS - 16 * pb * (pb + 1)); };   // 3 * 64 * sum_{p<pb} cols(p)
   __shared__ unsigned long long mma_bar_s[kGroups];
   __shared__ uint32_t tmem_base_s;
   __shared__ int timed_out_g[kGroups];
@@ -202,18 +212,21 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
       const int d = c >> 10, i = (c >> 5) & 31, j = c & 31;
       gd_s[c] = gsrc[(size_t)(32 * d + i) * NBITS + 32 * d + j];
     }
-    // -G[32 pb + i][j] as three bf16 terms (g = t1 + t2 + t3 up to 2^-24 |g|), operand rows j, K index i
+    // -G[32 pb + i][j], j after block pb, as three bf16 terms (g = t1 + t2 + t3 up to 2^-24 |g|); operand rows j, K index i
     for (int c = tid; c < (NB - 1) * 32 * NBITS; c += kThreads) {
       const int pb = c / (32 * NBITS), i = (c / NBITS) & 31, j = c % NBITS;
+      const int j0 = 32 * (pb + 1);
+      if (j < j0) continue;
       const float g = -gsrc[(size_t)(32 * pb + i) * NBITS + j];
       const __nv_bfloat16 t1 = __float2bfloat16_rn(g);
       const float r1 = g - __bfloat162float(t1);
       const __nv_bfloat16 t2 = __float2bfloat16_rn(r1);
       const __nv_bfloat16 t3 = __float2bfloat16_rn(r1 - __bfloat162float(t2));
-      unsigned char* base = gb_s + (size_t)pb * 3 * GB_PART + nosw_offset(NBITS, j, i);
+      const size_t part = (size_t)gb_cols(pb) * 64;
+      unsigned char* base = gb_s + gb_off(pb) + nosw_offset(gb_cols(pb), j - j0, i);
       *reinterpret_cast<__nv_bfloat16*>(base) = t1;
-      *reinterpret_cast<__nv_bfloat16*>(base + GB_PART) = t2;
-      *reinterpret_cast<__nv_bfloat16*>(base + 2 * GB_PART) = t3;
+      *reinterpret_cast<__nv_bfloat16*>(base + part) = t2;
+      *reinterpret_cast<__nv_bfloat16*>(base + 2 * part) = t3;
     }
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the tensor core
@@ -256,9 +269,10 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
     for (int part = 0; part < 3; ++part) {
 #pragma unroll
       for (int ks = 0; ks < 2; ++ks) {
+        const unsigned lbo = (unsigned)(gb_cols(pb) >> 3) * 128;
         const unsigned char* ap = u_s + (size_t)ks * 2 * U_LBO;
-        const unsigned char* bp = gb_s + (size_t)(pb * 3 + part) * GB_PART + (size_t)(j0 >> 3) * 128 + (size_t)ks * 2 * GB_LBO;
-        umma_bf16(tmem_base + (uint32_t)j0, umma_desc_nosw(ap, U_LBO, 128), umma_desc_nosw(bp, GB_LBO, 128), idc, 1u);
+        const unsigned char* bp = gb_s + gb_off(pb) + (size_t)part * gb_cols(pb) * 64 + (size_t)ks * 2 * lbo;
+        umma_bf16(tmem_base + (uint32_t)j0, umma_desc_nosw(ap, U_LBO, 128), umma_desc_nosw(bp, lbo, 128), idc, 1u);
       }
     }
     umma_commit(mma_bar);
@@ -381,7 +395,7 @@ cudaError_t launch(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStrea
   const bpc_config& c = ctx->cfg;
   constexpr int NB = NBITS / 32;
   const size_t smem = (size_t)kGroups * kTileKeys * 256 + (size_t)NBITS * 256 + (size_t)NB * 4096 + (size_t)kGroups * kTileKeys * 64 +
-                      (size_t)(NB - 1) * 3 * NBITS * 64 + 1024;
+                      (size_t)3 * 64 * ((NB - 1) * NBITS - 16 * (NB - 1) * NB) + 1024;   // (Gram terms: columns after each block)
   cudaError_t e = cudaFuncSetAttribute(encode_tc_kernel<NBITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const int tiles_max = ((c.n_max + kTileKeys - 1) / kTileKeys + kGroups - 1) / kGroups;   // a block takes kGroups tiles at a time
