@@ -129,7 +129,9 @@ append_kernel(const KV* __restrict__ k_new, const KV* __restrict__ v_new, KV* __
               int32_t* __restrict__ unit_lens, int32_t* __restrict__ err, int n_kv_heads, int n_max, int row_stride,
               int b, int shared_sets, int residual_correction) {
   extern __shared__ __align__(16) unsigned char smem[];
-  float* gs = reinterpret_cast<float*>(smem);                        // [b][b] when b <= 128
+  // the 32 x 32 blocks of the Gram matrix on and to the right of the diagonal (the only ones the sweep reads), block
+  // (r, c) at slot r * nb - r (r - 1) / 2 + (c - r): 144 KB at 256 bits
+  float* gs = reinterpret_cast<float*>(smem);
   __shared__ float t_s[256];
   __shared__ float k_s[BPC_D];
   __shared__ uint32_t ubits_s[8];
@@ -142,11 +144,16 @@ append_kernel(const KV* __restrict__ k_new, const KV* __restrict__ v_new, KV* __
   }
   const int set = shared_sets ? unit % n_kv_heads : unit;
   const float* Gset = gram + (size_t)set * b * b;
-  const bool g_in_smem = b <= 128;
-  if (g_in_smem && residual_correction) {
-    const float4* src = reinterpret_cast<const float4*>(Gset);
+  const int nb = b / 32;
+  if (residual_correction) {
     float4* dst = reinterpret_cast<float4*>(gs);
-    for (int i = tid; i < b * b / 4; i += kAppThreads) dst[i] = src[i];
+    int slot = 0;
+    for (int r = 0; r < nb; ++r) {
+      for (int c = r; c < nb; ++c, ++slot) {                         // one block per pass of the 256 threads: row tid / 8, four columns
+        const int i = tid >> 3, l4 = tid & 7;
+        dst[slot * 256 + tid] = *reinterpret_cast<const float4*>(Gset + (size_t)(32 * r + i) * b + 32 * c + 4 * l4);
+      }
+    }
   }
   const KV* kn = k_new + (size_t)unit * BPC_D;
   const KV* vn = v_new + (size_t)unit * BPC_D;
@@ -175,13 +182,13 @@ append_kernel(const KV* __restrict__ k_new, const KV* __restrict__ v_new, KV* __
     }
   }
   __syncthreads();
-  const int nb = b / 32;
-  const float* Gp = g_in_smem ? gs : Gset;
+  auto gblock = [&](int r, int c) { return gs + (size_t)(r * nb - r * (r - 1) / 2 + (c - r)) * 1024; };
   float t = warp < nb ? t_s[32 * warp + lane] : 0.f;
   float gd[32];                                                      // diagonal block column of this lane
   if (warp < nb && residual_correction) {
+    const float* gb = gblock(warp, warp);
 #pragma unroll
-    for (int i = 0; i < 32; ++i) gd[i] = Gp[(size_t)(32 * warp + i) * b + 32 * warp + lane];
+    for (int i = 0; i < 32; ++i) gd[i] = gb[32 * i + lane];
   }
   for (int blk = 0; blk < nb; ++blk) {
     if (warp == blk) {
@@ -201,11 +208,11 @@ append_kernel(const KV* __restrict__ k_new, const KV* __restrict__ v_new, KV* __
     __syncthreads();
     if (residual_correction && warp > blk && warp < nb) {
       const uint32_t bits = ubits_s[blk];
-      const float* gcol = Gp + (size_t)(32 * blk) * b + 32 * warp + lane;
+      const float* gcol = gblock(blk, warp) + lane;
       float a = 0.f;
 #pragma unroll 8
       for (int i = 0; i < 32; ++i) {
-        const float g = gcol[(size_t)i * b];
+        const float g = gcol[32 * i];
         a += ((bits >> i) & 1u) ? g : -g;
       }
       t -= a;
@@ -679,7 +686,7 @@ cudaError_t bpc_launch_append(bpc_ctx* ctx, const void* k_new, const void* v_new
                               uint64_t* codes, cudaStream_t stream) {
   const bpc_config& c = ctx->cfg;
   const int b = c.code_bits;
-  const size_t smem = b <= 128 ? (size_t)b * b * 4 : 16;
+  const size_t smem = (size_t)(b / 32) * (b / 32 + 1) / 2 * 4096;   // Gram blocks on and right of the diagonal
   const int shared_sets = c.hash_sets != ctx->units;
   cudaError_t e;
   if (c.kv_dtype == BPC_BF16) {
