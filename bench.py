@@ -290,6 +290,11 @@ def run_ours(args):
         layers[s % L].step()
     torch.cuda.synchronize()
     if args.profile:                      # plain eager steps for a profiler to capture; no graphs, no other legs
+        if args.profile_leg == "work_items":
+            for ly in layers:
+                ly.ctx.debug_set_decode_path(2)
+            for s in range(W):
+                layers[s % L].step()
         if args.profile_leg == "weighted7":
             for ly in layers:
                 ly.make_weighted_twin(B)
@@ -358,7 +363,28 @@ def run_ours(args):
     torch.cuda.synchronize()
     reset_after_warmup()
     ms_app = _time_graph(g_app, barrier) / K
-    # --- the paper's weighted score (sign + 7 magnitude planes) on the same workload, where 16-bit keys suffice
+    # --- the same fused step through the library's second decode kernel ((unit, key range) work items on a persistent
+    # grid; opt-in, never chosen by the library itself), for comparison
+    ms_items = None
+    if spec.dtype == "bf16":
+        for ly in layers:
+            ly.ctx.debug_set_decode_path(2)
+        if all(ly.ctx.uses_work_items() for ly in layers):
+            reset_after_warmup()
+            for s in range(min(W, 8)):
+                layers[(W + s) % L].step()
+            torch.cuda.synchronize()
+            reset_after_warmup()
+            g_items = _graph_of(lambda: [layers[(W + s) % L].step() for s in range(K)])
+            reset_after_warmup()
+            g_items.replay()
+            torch.cuda.synchronize()
+            reset_after_warmup()
+            ms_items = _time_graph(g_items, barrier) / K
+        for ly in layers:
+            ly.ctx.debug_set_decode_path(0)                 # back to the library's own choice
+        reset_after_warmup()
+    # --- the paper's weighted score (sign + 7 magnitude planes) on the same workload
     ms_w7 = None
     if True:
         for ly, c in zip(layers, per_layer_w):
@@ -536,7 +562,7 @@ def run_ours(args):
         "roofline": _roofline(spec, lens_now, ms_step, peaks,
                               # dram__bytes_read.sum + dram__bytes_write.sum of one launch: not measured by this run, quoted
                               # from the committed profiler capture of this workload
-                              traffic=116.8e6 if (args.workload == 2 and not args.separate_kv) else None,
+                              traffic=116.5e6 if (args.workload == 2 and not args.separate_kv) else None,
                               traffic_source="ncu capture of one launch, profiles/decode_fused_cfg2_ncu.md (not measured in this run)"
                               if (args.workload == 2 and not args.separate_kv) else None),
         "timing": {"reps": args.reps, "us_per_step_median": ms_step * 1e3, "us_per_step_min": min(rep_ms) / K * 1e3,
@@ -545,6 +571,7 @@ def run_ours(args):
         "breakdown_us": {"fused_step": ms_step * 1e3, "decode_attn_only": ms_dec * 1e3, "append_only": ms_app * 1e3,
                          "append_then_decode_two_launches": ms_two * 1e3,
                          "fused_step_weighted7_scores": None if ms_w7 is None else ms_w7 * 1e3,
+                         "fused_step_work_item_kernel_opt_in": None if ms_items is None else ms_items * 1e3,
                          "fused_step_with_error_aware_safeguard": ms_eas * 1e3},
         "prefill": {"fit_ms": fit_ms, "fit_power2_ms": fit_power2_ms, "encode_ms": enc_ms, "encode_keys_per_s": n_keys / (enc_ms * 1e-3),
                     "encode_gemm_tflops": enc_flops / (enc_ms * 1e-3) / 1e12,
@@ -846,7 +873,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--separate-kv", action="store_true", help="separate K and V arrays instead of interleaved rows")
     ap.add_argument("--profile", action="store_true", help="warm-up plus K eager steps only (for ncu captures)")
-    ap.add_argument("--profile-leg", choices=("fused", "weighted7"), default="fused",
+    ap.add_argument("--profile-leg", choices=("fused", "weighted7", "work_items"), default="fused",
                     help="with --profile: the fused step with Hamming scores (default) or with the weighted score")
     ap.add_argument("--sweep", action="store_true", help="second workload: latency over contexts and batch sizes, 64-bit codes, 1K/2K budgets")
     ap.add_argument("--quality", action="store_true", help="selection quality yard-sticks (recall vs exact top-k, cosine vs dense) for 32/64/128/256-bit codes")
