@@ -85,9 +85,9 @@ def fit(K: np.ndarray, v_star: np.ndarray, power_iters: int = 0):
             if nw > 0.0:
                 w = w / nw
             w = R @ (R.T @ w)
-        u = sign_pm1(w)                                              # u <- sign(...)
-        v = (u @ R) / N                                              # v <- u R / N
-        R = R - np.outer(u, v)                                       # R <- R - u^T v
+        u = sign_pm1(w)                                              # binary component of this iteration
+        v = (u @ R) / N                                              # its least-squares row of P
+        R = R - np.outer(u, v)                                       # what the component explains is removed
         H[:, i] = u
         P[i, :] = v
         trace.append(np.linalg.norm(R))
@@ -280,7 +280,9 @@ def decode_unit(q_group, K, V, bits, P_h, ppm, count=0, mode=HAMMING, sm_scale=0
 
     With an error-aware safeguard set s_err (ascending indices), the budget k is split: the first min(|s_err|, k)
     safeguard keys are always attended and the hash search fills the remaining k - min(|s_err|, k) places
-    (it competes over all keys, so a key may be chosen twice; the union removes it).
+    (it competes over all keys, so a key may be chosen twice; the union removes it).  When the set is larger than
+    the budget (the paper sizes it at a tenth of the budget, so this is a degenerate case it never meets) "the first"
+    means the lowest indices: the set is static and kept in index order, its members are not ranked again by error.
     Returns dict(out [G, D], idx [<= k] (attended keys, ascending), hash_idx, scores [n], s, a).
     """
     _, s, a = query_hash(q_group, P_h, mode)
