@@ -272,6 +272,59 @@ __device__ __forceinline__ int score_key<4, 2>(const uint32_t (&h)[4], const uin
   return __popc(s0) + __popc(x0[3]) + 2 * __popc(s2) + 4 * (__popc(c1) + __popc(c2));
 }
 
+// Weighted scores of U codes at once, planes in the outer loop.  The plane masks (up to ten planes of W32 words) are
+// read from shared memory one plane at a time (the whole warp reads one address: a broadcast) instead of living in
+// registers, which leaves the registers to the U codes and their carry words: U independent dependency chains per
+// thread instead of two, so that the logic and population-count pipes stay busy.  Same arithmetic as score_key.
+template <int W32, int NP, int U>
+__device__ __forceinline__ void score_keys_plane_outer(const uint32_t (&h)[U][W32], const uint32_t (&sg)[W32],
+                                                       const uint32_t (*mask)[8], int (&key)[U]) {
+  static_assert(W32 >= 2 && W32 % 2 == 0, "pairs of words");
+  constexpr int C = W32 / 2;
+  uint32_t x[U][W32], cy[U][C];
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    key[u] = 0;
+#pragma unroll
+    for (int f = 0; f < C; ++f) cy[u][f] = 0u;
+#pragma unroll
+    for (int w = 0; w < W32; ++w) x[u][w] = ~(h[u][w] ^ sg[w]);
+  }
+#pragma unroll
+  for (int pl = 0; pl < NP; ++pl) {
+    uint32_t m[W32];
+    if constexpr (W32 % 4 == 0) {
+#pragma unroll
+      for (int w = 0; w < W32; w += 4) {
+        const uint4 v = *reinterpret_cast<const uint4*>(&mask[pl][w]);
+        m[w] = v.x; m[w + 1] = v.y; m[w + 2] = v.z; m[w + 3] = v.w;
+      }
+    } else {
+      const uint2 v = *reinterpret_cast<const uint2*>(&mask[pl][0]);
+      m[0] = v.x; m[1] = v.y;
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      int c = 0;
+#pragma unroll
+      for (int f = 0; f < C; ++f) {
+        const uint32_t t = (x[u][2 * f] & m[2 * f]) ^ cy[u][f];
+        const uint32_t s2 = (x[u][2 * f + 1] & m[2 * f + 1]) ^ t;
+        cy[u][f] = cy[u][f] ^ (t & (s2 ^ t ^ cy[u][f]));
+        c += __popc(s2);
+      }
+      key[u] += c << pl;
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    int c = 0;
+#pragma unroll
+    for (int f = 0; f < C; ++f) c += __popc(cy[u][f]);
+    key[u] += c << NP;
+  }
+}
+
 // K/V row fragment of 8 consecutive dims held by one lane (fp32 caches; read from the staging ring)
 struct RowFragF32 {
   uint4 a, b;
@@ -444,8 +497,9 @@ bpc_decode_kernel(const DecodeParams p) {
   const uint32_t* cu = reinterpret_cast<const uint32_t*>(p.codes) + (size_t)unit * (size_t)p.n_max * W32;
   int32_t* dbg = p.dbg_scores != nullptr ? p.dbg_scores + (size_t)unit * p.n_max : nullptr;
   // codes in flight per thread and buffer: the Hamming scan is bound by memory latency and wants many; the weighted
-  // scan is bound by its arithmetic and wants the registers for the plane masks instead
-  constexpr int U = MODE == 1 ? (W32 <= 2 ? 4 : 2) : (W32 <= 4 ? 8 : 4);
+  // scan is bound by its arithmetic and scores a whole batch plane by plane (masks read from shared memory), so its
+  // batch is as large as the registers for the codes and their carry words allow
+  constexpr int U = MODE == 1 ? (W32 <= 1 ? 4 : W32 == 2 ? 8 : W32 == 4 ? 4 : 2) : (W32 <= 4 ? 8 : 4);
   auto load_code = [&](uint32_t (&h)[W32], int i) {
     const uint32_t* src = cu + (size_t)i * W32;
     if (W32 == 1) {
@@ -614,20 +668,38 @@ bpc_decode_kernel(const DecodeParams p) {
   BPC_STAMP(1);
   // ------------------------------------------------------------------ phase 1: scan
   if (tid < nts) {
-    uint32_t sg[W32], mk[NP][W32];
+    // weighted scores of codes of two or more words: the plane masks stay in shared memory (score_keys_plane_outer)
+    constexpr bool kPlaneOuter = MODE == 1 && W32 >= 2;
+    uint32_t sg[W32], mk[kPlaneOuter ? 1 : NP][W32];
 #pragma unroll
     for (int w = 0; w < W32; ++w) {
       sg[w] = st->signw[w];
+      if constexpr (!kPlaneOuter) {
 #pragma unroll
-      for (int pl = 0; pl < NP; ++pl) mk[pl][w] = st->mask[pl][w];
+        for (int pl = 0; pl < NP; ++pl) mk[pl][w] = st->mask[pl][w];
+      }
     }
     const int rfull = st->rsum << cs;                       // sum_j |A_j|
+    auto score_one = [&](const uint32_t (&h)[W32]) -> int {
+      if constexpr (kPlaneOuter) return rescore_key<W32, NP>(h, st->signw, st->mask);
+      else return score_key<W32, NP>(h, sg, mk);
+    };
     auto score_batch = [&](const uint32_t (&h)[U][W32], int base) {
+      if constexpr (kPlaneOuter) {
+        int keys[U];
+        score_keys_plane_outer<W32, NP, U>(h, sg, st->mask, keys);
 #pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int key = score_key<W32, NP>(h[u], sg, mk);
-        sc[score_slot(base - c0 + u * nts + tid)] = (uint16_t)(key >> ksh);
-        atomicAdd(&hist[(key >> ksh) >> hsh], 1u);
+        for (int u = 0; u < U; ++u) {
+          sc[score_slot(base - c0 + u * nts + tid)] = (uint16_t)(keys[u] >> ksh);
+          atomicAdd(&hist[(keys[u] >> ksh) >> hsh], 1u);
+        }
+      } else {
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const int key = score_key<W32, NP>(h[u], sg, mk);
+          sc[score_slot(base - c0 + u * nts + tid)] = (uint16_t)(key >> ksh);
+          atomicAdd(&hist[(key >> ksh) >> hsh], 1u);
+        }
       }
     };
     [[maybe_unused]] const int STEP = nts * U;
@@ -636,7 +708,7 @@ bpc_decode_kernel(const DecodeParams p) {
       for (int i = c0 + tid; i < c1s; i += nts) {
         uint32_t h[W32];
         load_code(h, i);
-        dbg[i] = ((2 * score_key<W32, NP>(h, sg, mk)) << cs) - rfull;
+        dbg[i] = ((2 * score_one(h)) << cs) - rfull;
       }
     }
     if constexpr (STREAM) {
@@ -702,13 +774,19 @@ bpc_decode_kernel(const DecodeParams p) {
           for (int w = 0; w < W32; ++w) h[u][w] = 0u;
         }
       }
+      int keys[U];
+      if constexpr (kPlaneOuter) {
+        score_keys_plane_outer<W32, NP, U>(h, sg, st->mask, keys);
+      } else {
+#pragma unroll
+        for (int u = 0; u < U; ++u) keys[u] = score_key<W32, NP>(h[u], sg, mk);
+      }
 #pragma unroll
       for (int u = 0; u < U; ++u) {
         const int i = i0 + u * nts + tid;
         if (i < c1s) {
-          const int key = score_key<W32, NP>(h[u], sg, mk);
-          sc[score_slot(i - c0)] = (uint16_t)(key >> ksh);
-          atomicAdd(&hist[(key >> ksh) >> hsh], 1u);
+          sc[score_slot(i - c0)] = (uint16_t)(keys[u] >> ksh);
+          atomicAdd(&hist[(keys[u] >> ksh) >> hsh], 1u);
         }
       }
     }

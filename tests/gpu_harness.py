@@ -229,12 +229,14 @@ def check_eas(sess: Session, units, report: dict):
         report["eas_keys"] = report.get("eas_keys", 0) + m
 
 
-def check_decode(sess: Session, q: torch.Tensor, units, report: dict, budget_ppm=None, budget_count=0, append=None):
+def check_decode(sess: Session, q: torch.Tensor, units, report: dict, budget_ppm=None, budget_count=0, append=None,
+                 before_decode=None):
     """One decode step through the library, checked stage by stage for the given units.
 
     With append=(k_new, v_new) the step goes through the fused bpc_append_decode_attn call; the cache rows, the
     new key's code and the advanced lengths are checked as for bpc_append, and the plain decode call that
-    follows must reproduce the fused call's output bit for bit."""
+    follows must reproduce the fused call's output bit for bit.  before_decode, if given, is called right before the
+    decode call with no host synchronisation in between (work it queues on the stream precedes the decode launch)."""
     s = sess.spec
     ppm = s.budget_ppm if budget_ppm is None else budget_ppm
     n_max = sess.w.n_max
@@ -242,6 +244,8 @@ def check_decode(sess: Session, q: torch.Tensor, units, report: dict, budget_ppm
     dbg_qw = torch.zeros(sess.units, s.code_bits, dtype=torch.int32, device="cuda")
     sel = torch.full((sess.units, n_max), -1, dtype=torch.int32, device="cuda")
     sess.ctx.debug_set_buffers(dbg_scores, dbg_qw)
+    if before_decode is not None:
+        before_decode()
     if append is None:
         out = sess.ctx.decode_attn(q, sess.k_cache, sess.v_cache, sess.codes, budget_ppm=ppm, budget_count=budget_count,
                                    sel_idx=sel)

@@ -165,6 +165,35 @@ def test_shared_projection_per_kv_head():
     H.check_decode(sess, q.cuda(), [0, 3], rep)
 
 
+def test_projection_update_then_decode_without_host_sync():
+    """bpc_set_projection and bpc_decode_attn queued back to back on one stream, no host synchronisation between them:
+    the decode launch may start early (programmatic dependent launch), but it must hash with the new projection.  The
+    context holds another projection until then, so a decode that read P_h too early would select other keys."""
+    H = _harness()
+    spec = CONFIGS[1].scaled(name="pdl", wid=73, batch=2, n_ctx=6000, n_kv_heads=2, n_q_heads=8, steps=1)
+    sess = H.Session(spec)
+    sess.fit()
+    P1 = sess.P.clone()
+    P2 = torch.flip(P1, dims=[1]).neg().contiguous()          # the same components, reversed and negated: another valid P
+    sess.ctx.set_projection(P2)
+    sess.P, sess.Ph, sess.gram = sess.ctx.get_projection()
+    sess.encode()                                             # cache codes under P2
+    rep = {}
+    H.check_encode(sess, [0, 3], rep)
+    q, _ = sess.w.queries(sess.lens)
+    q = q.cuda()
+    filler = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for trial in range(3):
+        sess.ctx.set_projection(P1)                           # the context hashes with P1 ...
+        torch.cuda.synchronize()
+
+        def switch():
+            filler.fill_(trial)                               # (keeps the GPU busy so that the next launches queue up behind it)
+            sess.ctx.set_projection(P2)                       # ... until this call, which the decode launch follows directly
+
+        H.check_decode(sess, q, [0, 3], rep, before_decode=switch)
+
+
 def test_offline_projection_calibration_on_aggregated_keys():
     """Offline Projection Calibration (Section 3.2): Algorithm 1 runs once, ahead of serving, on keys aggregated over
     several sequences (here with two power iterations), one projection per KV head; the serving context takes that
