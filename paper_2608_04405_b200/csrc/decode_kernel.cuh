@@ -680,10 +680,6 @@ bpc_decode_kernel(const DecodeParams p) {
       }
     }
     const int rfull = st->rsum << cs;                       // sum_j |A_j|
-    auto score_one = [&](const uint32_t (&h)[W32]) -> int {
-      if constexpr (kPlaneOuter) return rescore_key<W32, NP>(h, st->signw, st->mask);
-      else return score_key<W32, NP>(h, sg, mk);
-    };
     auto score_batch = [&](const uint32_t (&h)[U][W32], int base) {
       if constexpr (kPlaneOuter) {
         int keys[U];
@@ -708,7 +704,8 @@ bpc_decode_kernel(const DecodeParams p) {
       for (int i = c0 + tid; i < c1s; i += nts) {
         uint32_t h[W32];
         load_code(h, i);
-        dbg[i] = ((2 * score_one(h)) << cs) - rfull;
+        if constexpr (kPlaneOuter) dbg[i] = ((2 * rescore_key<W32, NP>(h, st->signw, st->mask)) << cs) - rfull;
+        else dbg[i] = ((2 * score_key<W32, NP>(h, sg, mk)) << cs) - rfull;
       }
     }
     if constexpr (STREAM) {
@@ -774,19 +771,26 @@ bpc_decode_kernel(const DecodeParams p) {
           for (int w = 0; w < W32; ++w) h[u][w] = 0u;
         }
       }
-      int keys[U];
       if constexpr (kPlaneOuter) {
+        int keys[U];
         score_keys_plane_outer<W32, NP, U>(h, sg, st->mask, keys);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const int i = i0 + u * nts + tid;
+          if (i < c1s) {
+            sc[score_slot(i - c0)] = (uint16_t)(keys[u] >> ksh);
+            atomicAdd(&hist[(keys[u] >> ksh) >> hsh], 1u);
+          }
+        }
       } else {
 #pragma unroll
-        for (int u = 0; u < U; ++u) keys[u] = score_key<W32, NP>(h[u], sg, mk);
-      }
-#pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int i = i0 + u * nts + tid;
-        if (i < c1s) {
-          sc[score_slot(i - c0)] = (uint16_t)(keys[u] >> ksh);
-          atomicAdd(&hist[(keys[u] >> ksh) >> hsh], 1u);
+        for (int u = 0; u < U; ++u) {
+          const int i = i0 + u * nts + tid;
+          if (i < c1s) {
+            const int key = score_key<W32, NP>(h[u], sg, mk);
+            sc[score_slot(i - c0)] = (uint16_t)(key >> ksh);
+            atomicAdd(&hist[(key >> ksh) >> hsh], 1u);
+          }
         }
       }
     }
