@@ -31,7 +31,12 @@ constexpr int kTileKeys = 128;
 constexpr int kGroupThreads = 128;   // one warpgroup sweeps one key tile (a TMEM lane per thread)
 constexpr int kGroups = 3;           // warpgroups per block, each with its own tile, accumulator columns and barrier
 constexpr int kPair = 1;             // key tiles a warpgroup sweeps together (one key of each per thread)
-constexpr int kThreads = kGroupThreads * kGroups;
+// 256-bit codes run as two launches over 128 bits each.  HALF = 0: the code is NBITS long.  HALF = 1: bits 0..127 of a
+// 256-bit code (projection rows 0..127, Gram block G[0:128, 0:128], code words 0..3 of 8).  HALF = 2: bits 128..255; their
+// decision values start from P_h[128 + j] . k - sum_{i < 128} u_i G[i][128 + j], and that sum over the first half's signs
+// (read back from the code words the first launch wrote) is one more contraction on the tensor cores, U1 (128 keys x
+// 128 signs) times -G[0:128, 128:256] as three bf16 terms (96 KB of shared memory: one warpgroup per block then).
+constexpr int kCrossBytes = 3 * 128 * 128 * 2;
 
 __device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
 
@@ -153,8 +158,8 @@ __device__ __forceinline__ size_t sw128_offset(int rows, int r, int ch) {
   return (size_t)(ch >> 3) * ((size_t)rows * 128) + (size_t)r * 128 + (size_t)(((ch & 7) ^ (r & 7)) << 4);
 }
 
-template <int NBITS>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int NBITS, int GROUPS, int HALF>
+__global__ void __launch_bounds__(kGroupThreads * GROUPS, 1)
 encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16* __restrict__ Ph, const float* __restrict__ gram,
                  const int32_t* __restrict__ unit_lens, uint64_t* __restrict__ codes, int32_t* __restrict__ err,
                  int n_kv_heads, int n_max, int row_stride, int shared_sets, int residual_correction, int blocks_per_unit,
@@ -162,7 +167,13 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
   extern __shared__ __align__(16) unsigned char smem_raw[];
   // the swizzled operand tiles need 1024-byte alignment in the shared address space
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-  constexpr int NB = NBITS / 32;                           // 32-bit column blocks
+  constexpr int kGroups = GROUPS;                          // (shadows the default of the single-launch code lengths)
+  constexpr int kThreads = kGroupThreads * GROUPS;
+  static_assert(HALF == 0 || NBITS == 128, "the two-launch form is for 256-bit codes");
+  constexpr int TOTAL = HALF == 0 ? NBITS : 256;           // bits of a whole code
+  constexpr int ROW0 = HALF == 2 ? 128 : 0;                // first projection row (= first bit) of this launch
+  constexpr int NB = NBITS / 32;                           // 32-bit column blocks of this launch
+  constexpr int NWK = TOTAL / 32;                          // code words per key
   constexpr int A_BYTES = kTileKeys * 256;                 // one key tile (128 rows x 128 bf16)
   constexpr int B_BYTES = NBITS * 256;                     // the projection rows
   constexpr int GD_BYTES = NB * 32 * 32 * 4;               // diagonal 32 x 32 blocks of the Gram matrix, fp32
@@ -177,6 +188,8 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
   float* gd_s = reinterpret_cast<float*>(b_s + B_BYTES);   // [NB][32][32]
   unsigned char* u_s = reinterpret_cast<unsigned char*>(gd_s) + GD_BYTES + (size_t)grp * U_BYTES;
   unsigned char* gb_s = reinterpret_cast<unsigned char*>(gd_s) + GD_BYTES + kGroups * U_BYTES;
+  constexpr size_t GB_BYTES = (size_t)3 * 64 * ((NB - 1) * NBITS - 16 * (NB - 1) * NB);
+  unsigned char* x_s = gb_s + GB_BYTES;                    // HALF == 2: the three bf16 terms of -G[0:128, 128:256], operands [128 x 128]
   auto gb_cols = [](int pb) { return NBITS - 32 * (pb + 1); };                     // columns after block pb
   auto gb_off = [](int pb) { return (size_t)3 * 64 * (size_t)(pb * NBITS - 16 * pb * (pb + 1)); };   // 3 * 64 * sum_{p<pb} cols(p)
   __shared__ unsigned long long mma_bar_s[kGroups];
@@ -202,22 +215,38 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   {
-    const unsigned char* psrc = reinterpret_cast<const unsigned char*>(Ph + (size_t)set * NBITS * BPC_D);
+    const unsigned char* psrc = reinterpret_cast<const unsigned char*>(Ph + ((size_t)set * TOTAL + ROW0) * BPC_D);
     for (int c = tid; c < NBITS * 16; c += kThreads) {
       const int r = c >> 4, ch = c & 15;
       *reinterpret_cast<uint4*>(b_s + sw128_offset(NBITS, r, ch)) = *reinterpret_cast<const uint4*>(psrc + (size_t)r * 256 + ch * 16);
     }
-    const float* gsrc = gram + (size_t)set * NBITS * NBITS;
+    const float* gfull = gram + (size_t)set * TOTAL * TOTAL;
+    const float* gsrc = gfull + (size_t)ROW0 * TOTAL + ROW0;  // this launch's diagonal block of the Gram matrix, row stride TOTAL
     for (int c = tid; c < NB * 32 * 32; c += kThreads) {     // diagonal blocks, kept in fp32 for the in-register sweep
       const int d = c >> 10, i = (c >> 5) & 31, j = c & 31;
-      gd_s[c] = gsrc[(size_t)(32 * d + i) * NBITS + 32 * d + j];
+      gd_s[c] = gsrc[(size_t)(32 * d + i) * TOTAL + 32 * d + j];
+    }
+    if constexpr (HALF == 2) {
+      // -G[i][128 + j] for the first half's bits i, as three bf16 terms; operand rows j, K index i, [128 x 128] each
+      for (int c = tid; c < 128 * 128; c += kThreads) {
+        const int i = c >> 7, j = c & 127;
+        const float g = -gfull[(size_t)i * TOTAL + 128 + j];
+        const __nv_bfloat16 t1 = __float2bfloat16_rn(g);
+        const float r1 = g - __bfloat162float(t1);
+        const __nv_bfloat16 t2 = __float2bfloat16_rn(r1);
+        const __nv_bfloat16 t3 = __float2bfloat16_rn(r1 - __bfloat162float(t2));
+        unsigned char* base = x_s + nosw_offset(128, j, i);
+        *reinterpret_cast<__nv_bfloat16*>(base) = t1;
+        *reinterpret_cast<__nv_bfloat16*>(base + 32768) = t2;
+        *reinterpret_cast<__nv_bfloat16*>(base + 65536) = t3;
+      }
     }
     // -G[32 pb + i][j], j after block pb, as three bf16 terms (g = t1 + t2 + t3 up to 2^-24 |g|); operand rows j, K index i
     for (int c = tid; c < (NB - 1) * 32 * NBITS; c += kThreads) {
       const int pb = c / (32 * NBITS), i = (c / NBITS) & 31, j = c % NBITS;
       const int j0 = 32 * (pb + 1);
       if (j < j0) continue;
-      const float g = -gsrc[(size_t)(32 * pb + i) * NBITS + j];
+      const float g = -gsrc[(size_t)(32 * pb + i) * TOTAL + j];
       const __nv_bfloat16 t1 = __float2bfloat16_rn(g);
       const float r1 = g - __bfloat162float(t1);
       const __nv_bfloat16 t2 = __float2bfloat16_rn(r1);
@@ -235,9 +264,12 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_all = tmem_base_s;
   const uint32_t tmem_base = tmem_all + (uint32_t)(grp * NBITS);   // this warpgroup's accumulator columns
-  float trace_g = 0.f;
-  if (key_err != nullptr)
+  float trace_g = 0.f;                                       // trace of the whole Gram matrix (added by the launch that finishes the code)
+  if (key_err != nullptr && HALF != 1) {
+    if constexpr (HALF == 2)
+      for (int i = 0; i < 128; ++i) trace_g += gram[(size_t)set * TOTAL * TOTAL + (size_t)i * TOTAL + i];
     for (int i = 0; i < NBITS; ++i) trace_g += gd_s[(i >> 5) * 1024 + (i & 31) * 33];
+  }
 
   const unsigned char* kbase = reinterpret_cast<const unsigned char*>(k_cache) + (size_t)unit * n_max * (size_t)row_stride * 2;
   auto load_tile = [&](int tile) {                           // rows past n are zero-filled
@@ -278,6 +310,21 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
     umma_commit(mma_bar);
   };
 
+  // HALF == 2: T[:, 0..127] += U1 x (-G[0:128, 128:256]); U1 sits in the key-tile buffer (the projection has completed),
+  // three bf16 terms x eight K steps
+  auto issue_cross = [&]() {
+#pragma unroll
+    for (int part = 0; part < 3; ++part) {
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        const unsigned char* ap = a_t + (size_t)ks * 2 * U_LBO;
+        const unsigned char* bp = x_s + (size_t)part * 32768 + (size_t)ks * 2 * U_LBO;
+        umma_bf16(tmem_base, umma_desc_nosw(ap, U_LBO, 128), umma_desc_nosw(bp, U_LBO, 128), idesc, 1u);
+      }
+    }
+    umma_commit(mma_bar);
+  };
+
   // Tiles of this warpgroup: kGroups * blockIdx.x + grp, then every kGroups * blocks_per_unit-th.  The warpgroups
   // run independent pipelines (own tile, own accumulator columns, own MMA barrier, own hardware barrier); all threads
   // of a warpgroup take the same branches, so its barrier is always reached by all 128 of them.
@@ -304,7 +351,7 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
     // buffer is refilled with the warpgroup's next tile right away, under the sweep.
     const int key = tl * kTileKeys + gtid;
     float k2 = 0.f;
-    if (key_err != nullptr) {                                // squared norm of this thread's key, from the operand tile
+    if (key_err != nullptr && HALF != 2) {                   // squared norm of this thread's key, from the operand tile
       if (key < n) {
 #pragma unroll
         for (int ch = 0; ch < 16; ++ch) {
@@ -315,6 +362,35 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
         }
       }
       group_sync(grp);                                       // every thread has read its row before the refill starts
+    }
+    const uint32_t* kwords = reinterpret_cast<const uint32_t*>(codes) + ((size_t)unit * n_max + (key < n ? key : 0)) * NWK;
+    if (HALF == 2 && residual_correction) {
+      // the first half's 128 signs of this thread's key as row gtid of the bf16 operand U1, written over the key tile
+      // (no reader of the tile is left: the MMAs have completed and this launch computes no key norms)
+      const uint4 cw = *reinterpret_cast<const uint4*>(kwords);
+      const uint32_t w4[4] = {cw.x, cw.y, cw.z, cw.w};
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {                         // chunk c: signs 8c .. 8c+7
+        uint32_t h[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const uint32_t lo = ((w4[c >> 2] >> (8 * (c & 3) + 2 * e)) & 1u) ? 0x3F80u : 0xBF80u;
+          const uint32_t hi = ((w4[c >> 2] >> (8 * (c & 3) + 2 * e + 1)) & 1u) ? 0x3F80u : 0xBF80u;
+          h[e] = lo | (hi << 16);
+        }
+        *reinterpret_cast<uint4*>(a_t + (size_t)c * U_LBO + (size_t)(gtid >> 3) * 128 + (size_t)(gtid & 7) * 16) =
+            make_uint4(h[0], h[1], h[2], h[3]);
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      group_sync(grp);
+      if (gtid == 0) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        issue_cross();
+      }
+      if (!mbar_wait(mma_bar, ph)) timed_out_g[grp] = 1;     // the decision values now carry the first half's corrections
+      ph ^= 1u;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     }
     if (next < ntiles) load_tile(next);
     const uint32_t taddr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);   // a warp reaches the lanes of its quarter
@@ -368,9 +444,15 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
       issue_gemm();
     }
     // squared reconstruction error (Eq. 8) from the sweep: ||k - hP||^2 = ||k||^2 - 2 sum|t_i| + trace(G)
-    if (key_err != nullptr && key < n) key_err[(size_t)unit * n_max + key] = fmaxf(0.f, k2 - 2.f * abs_sum[0] + trace_g);
+    // (256-bit codes: the first launch leaves ||k||^2 - 2 sum|t_i| of its bits, the second adds its own sum and the trace)
+    if (key_err != nullptr && key < n) {
+      float* ke = key_err + (size_t)unit * n_max + key;
+      if (HALF == 0) *ke = fmaxf(0.f, k2 - 2.f * abs_sum[0] + trace_g);
+      else if (HALF == 1) *ke = k2 - 2.f * abs_sum[0];
+      else *ke = fmaxf(0.f, *ke - 2.f * abs_sum[0] + trace_g);
+    }
     if (key < n) {
-      uint32_t* dst = reinterpret_cast<uint32_t*>(codes) + ((size_t)unit * n_max + key) * NB;
+      uint32_t* dst = reinterpret_cast<uint32_t*>(codes) + ((size_t)unit * n_max + key) * NWK + (HALF == 2 ? 4 : 0);
       if (NB == 1) {
         dst[0] = words[0];
       } else if (NB == 2) {
@@ -390,15 +472,16 @@ encode_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16*
   }
 }
 
-template <int NBITS>
+template <int NBITS, int GROUPS, int HALF>
 cudaError_t launch(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStream_t stream) {
   const bpc_config& c = ctx->cfg;
   constexpr int NB = NBITS / 32;
-  const size_t smem = (size_t)kGroups * kTileKeys * 256 + (size_t)NBITS * 256 + (size_t)NB * 4096 + (size_t)kGroups * kTileKeys * 64 +
-                      (size_t)3 * 64 * ((NB - 1) * NBITS - 16 * (NB - 1) * NB) + 1024;   // (Gram terms: columns after each block)
-  cudaError_t e = cudaFuncSetAttribute(encode_tc_kernel<NBITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const size_t smem = (size_t)GROUPS * kTileKeys * 256 + (size_t)NBITS * 256 + (size_t)NB * 4096 + (size_t)GROUPS * kTileKeys * 64 +
+                      (size_t)3 * 64 * ((NB - 1) * NBITS - 16 * (NB - 1) * NB) +            // (Gram terms: columns after each block)
+                      (HALF == 2 ? (size_t)kCrossBytes : 0) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(encode_tc_kernel<NBITS, GROUPS, HALF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  const int tiles_max = ((c.n_max + kTileKeys - 1) / kTileKeys + kGroups - 1) / kGroups;   // a block takes kGroups tiles at a time
+  const int tiles_max = ((c.n_max + kTileKeys - 1) / kTileKeys + GROUPS - 1) / GROUPS;   // a block takes GROUPS tiles at a time
   // Blocks per unit.  One block fits an SM (shared memory), so the grid runs in waves of sm_count blocks and a last,
   // partly filled wave costs as much as a full one: starting from about four waves, take the first count whose last
   // wave is at least 90 % full (32 units on 148 SMs: 23 blocks per unit = 736 blocks = 4.97 waves).
@@ -411,7 +494,7 @@ cudaError_t launch(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStrea
   }
   if (bpu > tiles_max) bpu = tiles_max;
   const dim3 grid(bpu, ctx->units);
-  encode_tc_kernel<NBITS><<<grid, kThreads, smem, stream>>>(
+  encode_tc_kernel<NBITS, GROUPS, HALF><<<grid, kGroupThreads * GROUPS, smem, stream>>>(
       (const __nv_bfloat16*)k_cache, (const __nv_bfloat16*)ctx->P_h, ctx->gram, ctx->unit_lens, codes, ctx->dev_err,
       c.n_kv_heads, c.n_max, ctx->row_stride, c.hash_sets != ctx->units, c.residual_correction, bpu, ctx->key_err);
   return cudaGetLastError();
@@ -419,17 +502,23 @@ cudaError_t launch(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStrea
 
 }  // namespace
 
-// bf16 caches with 32-, 64- or 128-bit codes run on the tensor cores; other shapes report "not supported" and the
-// caller falls back to the CUDA-core kernel (fp32 caches have no bf16 operands; at 256 bits the bf16 terms of the Gram
-// matrix, 336 KB, do not fit shared memory next to the operands).
+// bf16 caches run on the tensor cores: 32-, 64- and 128-bit codes in one launch, 256-bit codes in two (the bf16 terms of
+// a 256 x 256 Gram matrix do not fit shared memory next to the operands, those of its 128 x 128 blocks do).  fp32 caches
+// report "not supported" and the caller falls back to the CUDA-core kernel (they have no bf16 operands).
 cudaError_t bpc_launch_encode_tc(bpc_ctx* ctx, const void* k_cache, uint64_t* codes, cudaStream_t stream) {
   if (ctx->cfg.kv_dtype != BPC_BF16) return cudaErrorNotSupported;
   if (ctx->no_tc_encode) return cudaErrorNotSupported;     // diagnostic switch: the CUDA-core kernel is asked for
   cudaError_t e;
-  if (ctx->cfg.code_bits == 32) e = launch<32>(ctx, k_cache, codes, stream);
-  else if (ctx->cfg.code_bits == 64) e = launch<64>(ctx, k_cache, codes, stream);
-  else if (ctx->cfg.code_bits == 128) e = launch<128>(ctx, k_cache, codes, stream);
-  else return cudaErrorNotSupported;
+  if (ctx->cfg.code_bits == 32) e = launch<32, kGroups, 0>(ctx, k_cache, codes, stream);
+  else if (ctx->cfg.code_bits == 64) e = launch<64, kGroups, 0>(ctx, k_cache, codes, stream);
+  else if (ctx->cfg.code_bits == 128) e = launch<128, kGroups, 0>(ctx, k_cache, codes, stream);
+  else if (ctx->cfg.code_bits == 256) {
+    e = launch<128, kGroups, 1>(ctx, k_cache, codes, stream);
+    if (e == cudaSuccess) {
+      ctx->launches += 1;
+      e = launch<128, 1, 2>(ctx, k_cache, codes, stream);
+    }
+  } else return cudaErrorNotSupported;
   if (e == cudaSuccess) ctx->launches += 1;
   return e;
 }

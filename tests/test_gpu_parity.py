@@ -299,7 +299,7 @@ def test_weighted_scores_config4_head_layout_full_size():
     print(rep)
 
 
-@pytest.mark.parametrize("bits", [32, 64, 128])
+@pytest.mark.parametrize("bits", [32, 64, 128, 256])
 def test_tensor_core_encode_agrees_with_cuda_core_encode(bits):
     """bpc_encode_keys on the tcgen05 path and on the CUDA-core path (diagnostic switch) against each other and
     against the checker: ragged length with a partial last tile, several tiles per block."""
@@ -308,7 +308,7 @@ def test_tensor_core_encode_agrees_with_cuda_core_encode(bits):
     spec = CONFIGS[1].scaled(n_ctx=128 * 37 + 5, n_kv_heads=2, n_q_heads=8, code_bits=bits, steps=1)
     sess = H.Session(spec)
     sess.fit()
-    sess.encode()                                   # tensor-core path (bf16; 32, 64 or 128 bits)
+    sess.encode()                                   # tensor-core path (bf16; 256 bits: two launches)
     tc = sess.codes.clone()
     rep = {}
     H.check_encode(sess, [0, 1], rep)
