@@ -657,6 +657,8 @@ def run_all_configs(args):
                            "cluster_size": layers[0].ctx.get_cluster_size(), "kv_layout": "interleaved k|v rows"},
                 "timing": {"reps": args.reps, "us_per_step_min": min(rep_ms) / K * 1e3, "us_per_step_max": max(rep_ms) / K * 1e3},
                 "clocks": clocks, "roofline": _roofline(spec, lens_now, ms_step, peaks),
+                "prefill_ms_per_layer": {"fit": layers[-1].fit_ms, "encode": layers[-1].encode_ms,
+                                         "keys": int(sum(layers[-1].lens0)) * spec.n_kv_heads},
                 "device_error_word": max(ly.ctx.last_device_error() for ly in layers)}
         try:                                       # the paper's own score (sign + 7 magnitude planes) on the same workload
             for ly in layers:
