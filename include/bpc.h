@@ -279,7 +279,7 @@ bpc_status bpc_debug_set_work_item_trace(bpc_ctx* ctx, uint64_t* trace);
  * context, number of kernels this context has launched so far.
  * Diagnostic switches (explicit calls; the library reads no environment variable): bpc_debug_set_pdl(ctx, 0) launches
  * the decode kernel without programmatic dependent launch; bpc_debug_set_tensor_core_encode(ctx, 0) makes
- * bpc_encode_keys take the CUDA-core kernel; bpc_debug_force_streaming(ctx, 1) selects the streaming selection at any
+ * bpc_encode_keys and the passes of bpc_fit take the CUDA-core kernels instead of the tensor-core ones; bpc_debug_force_streaming(ctx, 1) selects the streaming selection at any
  * context length (Hamming scores without the safeguard only) and re-plans the launch geometry;
  * bpc_debug_force_key_shift(ctx, s) with s in 0..2 stores weighted score keys shifted right by at least s bits (the
  * library does that by itself only when a query's largest possible score exceeds 16 bits), so that the exact

@@ -322,6 +322,7 @@ class Context:
         _check(lib.bpc_debug_force_key_shift(self._h, shift), "bpc_debug_force_key_shift")
 
     def debug_set_tensor_core_encode(self, on: bool) -> None:
+        """False: bpc_encode_keys and the passes of bpc_fit run their CUDA-core kernels (cross-checks)."""
         _check(lib.bpc_debug_set_tensor_core_encode(self._h, 1 if on else 0), "bpc_debug_set_tensor_core_encode")
 
     def debug_force_streaming(self, on: bool) -> None:

@@ -137,6 +137,11 @@ cudaError_t bpc_launch_append(bpc_ctx* ctx, const void* k_new, const void* v_new
 cudaError_t bpc_launch_fit(bpc_ctx* ctx, const void* k_cache, const float* v_star, void* workspace,
                            cudaStream_t stream, int* launches);
 size_t bpc_fit_workspace_bytes_impl(const bpc_config* cfg);
+// tensor-core pass of Algorithm 1 (fit_tc.cu)
+bool bpc_fit_tc_covers(const bpc_ctx* ctx);
+void bpc_fit_tc_geometry(const bpc_ctx* ctx, int* blocks_per_unit, int* rows_per_block);
+cudaError_t bpc_launch_fit_pass_tc(bpc_ctx* ctx, const void* k_cache, uint32_t* hfit, const float* dir, const float* dots,
+                                   float* partials, int32_t* agree, int it, cudaStream_t stream);
 size_t bpc_fit_codes_offset_impl(const bpc_config* cfg);
 
 // ---- error-aware safeguard set construction (prefill.cu)

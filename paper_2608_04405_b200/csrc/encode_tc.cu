@@ -24,8 +24,10 @@
 // releases its tensor memory and returns.
 #include <stdlib.h>
 #include "common.cuh"
+#include "umma.cuh"
 
 namespace {
+using namespace umma;
 
 constexpr int kTileKeys = 128;
 constexpr int kGroupThreads = 128;   // one warpgroup sweeps one key tile (a TMEM lane per thread)
@@ -38,65 +40,9 @@ constexpr int kPair = 1;             // key tiles a warpgroup sweeps together (o
 // 128 signs) times -G[0:128, 128:256] as three bf16 terms (96 KB of shared memory: one warpgroup per block then).
 constexpr int kCrossBytes = 3 * 128 * 128 * 2;
 
-__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 // barrier among the 128 threads of one warpgroup (hardware barriers 1 .. kGroups; 0 is __syncthreads)
 __device__ __forceinline__ void group_sync(int g) { asm volatile("bar.sync %0, %1;" ::"r"(1 + g), "r"(kGroupThreads) : "memory"); }
 
-// Shared-memory operand descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t umma_desc_sw128(const void* smem_ptr) {
-  const uint64_t addr = (uint64_t)(smem_u32(smem_ptr) & 0x3FFFF) >> 4;
-  uint64_t d = addr;                       // bits [0,14): start address / 16
-  d |= (uint64_t)1 << 16;                  // bits [16,30): leading-dimension byte offset (unused for swizzled K-major)
-  d |= (uint64_t)(1024 >> 4) << 32;        // bits [32,46): stride between 8-row groups / 16
-  d |= (uint64_t)1 << 46;                  // bits [46,48): descriptor version of this architecture
-  d |= (uint64_t)2 << 61;                  // bits [61,64): 128-byte swizzle
-  return d;
-}
-// Shared-memory operand descriptor: K-major without swizzle.  Core matrices are 8 rows x 16 bytes, stored contiguously
-// (128 bytes); lbo = bytes between core matrices adjacent along K, sbo = bytes between core matrices adjacent along M/N.
-__device__ __forceinline__ uint64_t umma_desc_nosw(const void* smem_ptr, unsigned lbo, unsigned sbo) {
-  uint64_t d = (uint64_t)(smem_u32(smem_ptr) & 0x3FFFF) >> 4;
-  d |= (uint64_t)(lbo >> 4) << 16;
-  d |= (uint64_t)(sbo >> 4) << 32;
-  d |= (uint64_t)1 << 46;
-  return d;
-}
-// byte offset of element (row r, k) of an [R x 32] bf16 operand in that layout (core matrices of one K chunk contiguous)
-__device__ __forceinline__ size_t nosw_offset(int R, int r, int k) {
-  return (size_t)(k >> 3) * ((size_t)(R >> 3) * 128) + (size_t)(r >> 3) * 128 + (size_t)(r & 7) * 16 + (size_t)(k & 7) * 2;
-}
-// Instruction descriptor: D fp32, A and B bf16, both K-major, N and M.
-__device__ __forceinline__ uint32_t umma_idesc_bf16(int m, int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
-}
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit(unsigned long long* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-// bounded wait on an mbarrier phase; false when the iteration budget runs out
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity) {
-  for (int it = 0; it < 20000000; ++it) {
-    unsigned ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
-                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    if (ok) return true;
-  }
-  return false;
-}
 // 32 consecutive accumulator columns of this thread's TMEM lane, into t[OFF .. OFF+31]
 template <int OFF, int N>
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[N]) {
@@ -151,12 +97,6 @@ template <>
 struct DiagSweep<32> {
   static __device__ __forceinline__ void run(float (&)[kPair][32], uint32_t (&)[kPair], float (&)[kPair], const float*, int, int) {}
 };
-
-// byte offset of 16-byte chunk `ch` (0..15) of row `r` inside a [rows x 128 channels] bf16 operand tile:
-// two column blocks of 64 channels (128 bytes per row each), chunks XOR-swizzled by the row number
-__device__ __forceinline__ size_t sw128_offset(int rows, int r, int ch) {
-  return (size_t)(ch >> 3) * ((size_t)rows * 128) + (size_t)r * 128 + (size_t)(((ch & 7) ^ (r & 7)) << 4);
-}
 
 template <int NBITS, int GROUPS, int HALF>
 __global__ void __launch_bounds__(kGroupThreads * GROUPS, 1)

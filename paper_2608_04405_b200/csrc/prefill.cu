@@ -419,10 +419,10 @@ fit_pass_kernel(const KV* __restrict__ k_cache, uint32_t* __restrict__ hfit, con
 constexpr int kRedGroups = 4;
 __global__ void __launch_bounds__(BPC_D * kRedGroups)
 fit_reduce_kernel(const float* __restrict__ partials, const int32_t* __restrict__ agree, float* __restrict__ P,
-                  const int32_t* __restrict__ unit_lens, int n_max, int b, int it, int blocks_per_unit) {
+                  const int32_t* __restrict__ unit_lens, int n_max, int b, int it, int blocks_per_unit, int rows_per_block) {
   const int unit = blockIdx.x, c = threadIdx.x & (BPC_D - 1), q = threadIdx.x / BPC_D;
   const int n = min(unit_lens[unit], n_max);
-  const int nblk = (n + kFitRowsPerBlock - 1) / kFitRowsPerBlock;
+  const int nblk = (n + rows_per_block - 1) / rows_per_block;
   __shared__ double corr[256];                               // u_i . u_j for j < it
   __shared__ double part[kRedGroups][BPC_D];
   __shared__ int agp[kRedGroups][256];
@@ -747,7 +747,12 @@ cudaError_t bpc_launch_fit(bpc_ctx* ctx, const void* k_cache, const float* v_sta
                            cudaStream_t stream, int* launches) {
   const bpc_config& c = ctx->cfg;
   const size_t units = (size_t)ctx->units;
-  const int bpu = (c.n_max + kFitRowsPerBlock - 1) / kFitRowsPerBlock;
+  int bpu = (c.n_max + kFitRowsPerBlock - 1) / kFitRowsPerBlock;
+  int rows_per_block = kFitRowsPerBlock;
+  // bf16 caches with codes of up to 128 bits: the pass runs on the tensor cores, with longer row ranges per block (never
+  // more blocks than the workspace was sized for)
+  const bool tc_pass = bpc_fit_tc_covers(ctx);
+  if (tc_pass) bpc_fit_tc_geometry(ctx, &bpu, &rows_per_block);
   unsigned char* ws = (unsigned char*)workspace;
   uint32_t* hfit = (uint32_t*)ws;
   float* partials = (float*)(ws + fit_off_partials(&c));
@@ -779,13 +784,16 @@ cudaError_t bpc_launch_fit(bpc_ctx* ctx, const void* k_cache, const float* v_sta
 #define BPC_FIT_PASS(KV, JPL)                                                                                          \
     fit_pass_kernel<KV, JPL><<<grid, kFitThreads, 0, stream>>>((const KV*)k_cache, hfit, dir, dots, partials, agree,   \
                                                                 ctx->unit_lens, c.n_max, ctx->row_stride, it, bpu)
-    if (c.kv_dtype == BPC_BF16) {
+    if (tc_pass) {
+      cudaError_t e = bpc_launch_fit_pass_tc(ctx, k_cache, hfit, dir, dots, partials, agree, it, stream);
+      if (e != cudaSuccess) return e;
+    } else if (c.kv_dtype == BPC_BF16) {
       if (c.code_bits == 32) BPC_FIT_PASS(__nv_bfloat16, 4); else if (c.code_bits == 64) BPC_FIT_PASS(__nv_bfloat16, 8); else if (c.code_bits == 128) BPC_FIT_PASS(__nv_bfloat16, 16); else BPC_FIT_PASS(__nv_bfloat16, 32);
     } else {
       if (c.code_bits == 32) BPC_FIT_PASS(float, 4); else if (c.code_bits == 64) BPC_FIT_PASS(float, 8); else if (c.code_bits == 128) BPC_FIT_PASS(float, 16); else BPC_FIT_PASS(float, 32);
     }
 #undef BPC_FIT_PASS
-    fit_reduce_kernel<<<ctx->units, BPC_D * kRedGroups, 0, stream>>>(partials, agree, ctx->P, ctx->unit_lens, c.n_max, c.code_bits, it, bpu);
+    fit_reduce_kernel<<<ctx->units, BPC_D * kRedGroups, 0, stream>>>(partials, agree, ctx->P, ctx->unit_lens, c.n_max, c.code_bits, it, bpu, rows_per_block);
     *launches += 3;
   }
   return cudaGetLastError();

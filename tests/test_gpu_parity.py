@@ -327,6 +327,38 @@ def test_tensor_core_encode_agrees_with_cuda_core_encode(bits):
     assert torch.count_nonzero(tc[:, :, n:]) == 0   # nothing written past the cached keys
 
 
+@pytest.mark.parametrize("bits,n", [(128, 70000), (64, 9001), (32, 40000)])
+def test_tensor_core_fit_pass_agrees_with_cuda_core_pass(bits, n):
+    """bpc_fit with the pass over the keys on the tensor cores (bf16 caches, codes of up to 128 bits) and on the CUDA
+    cores (diagnostic switch): each against the fp64 replay of Algorithm 1, and the two projections against each other.
+    Lengths that are no multiple of the 128-key tile, several blocks per unit, two units of different length."""
+    H = _harness()
+    spec = CONFIGS[1].scaled(name="fit_tc", wid=74, batch=2, n_ctx=n, n_ctx_min=max(1, n // 3), n_kv_heads=1, n_q_heads=4,
+                             code_bits=bits, steps=1)
+    sess = H.Session(spec, gen_device="cuda" if n > 20000 else "cpu")
+    rep = {}
+    sess.fit()                                                # tensor-core pass
+    H.check_fit(sess, [0, 1], rep)
+    P_tc, H_tc = sess.P.clone(), [sess.hfit_bits(u) for u in range(2)]
+    sess.ctx.debug_set_tensor_core_encode(False)
+    try:
+        sess.fit()                                            # CUDA-core pass
+    finally:
+        sess.ctx.debug_set_tensor_core_encode(True)
+    H.check_fit(sess, [0, 1], rep)
+    # Each run is Algorithm 1 within rounding (checked above), but the two need not agree sign for sign: a decision value
+    # inside the rounding band may come out either way, the flipped row moves v_i by 2 K_row / N, and later decisions near
+    # zero follow.  They must stay close: few rows with any differing bit, projections equal to a few per cent.
+    for u in range(2):
+        rows = int((H_tc[u] != sess.hfit_bits(u)).any(axis=1).sum())
+        rep["rows_differing_u%d" % u] = rows
+        assert rows <= H_tc[u].shape[0] // 10, "%d rows differ between the two passes" % rows
+    rel = ((P_tc - sess.P).norm() / sess.P.norm()).item()
+    rep["projection_rel_diff"] = rel
+    assert rel <= 0.01
+    print(rep)
+
+
 def test_error_paths_do_not_launch():
     from paper_2608_04405_b200 import binding as B
     cfg = B.make_config(1, 4, 1, 1024, 128, torch.bfloat16)
