@@ -17,7 +17,7 @@
 // What stays on the CUDA cores is per key, not per (key, channel): the table look-up of sum_j u_j (v_j . d) four bits
 // at a time (the same table as the CUDA-core pass), the sign, one code-word store, and the agreement counters (bit-sliced,
 // one key per thread and tile).  A block holds three warpgroups with their own double-buffered key tiles, accumulators
-// and barriers; blocks take long contiguous row ranges (about two blocks per SM in total), so the per-block sums and
+// and barriers; blocks take long contiguous row ranges (a few waves of blocks in total), so the per-block sums and
 // counts are few and the counters are reduced once per block.
 //
 // Waits on MMA-completion barriers are bounded; on expiry the block raises the device error word, still releases its
@@ -33,7 +33,8 @@ constexpr int kTileKeys = 128;
 constexpr int kGroupThreads = 128;
 constexpr int kGroups = 3;
 constexpr int kThreads = kGroupThreads * kGroups;
-constexpr int kFlushTiles = 8;       // tiles whose channel sums accumulate in tensor memory before moving to fp64
+constexpr int kFlushTiles = 8;  // tiles whose channel sums accumulate in tensor memory before moving to fp64
+constexpr int kPlanWaves = 1;        // waves of blocks the row ranges are planned from
 constexpr int kPlanes = 8;           // bit-sliced agreement counters: up to 255 tiles per warpgroup and block
 constexpr int kTileBytes = kTileKeys * 256;
 constexpr int kSmallOp = 16 * 128 * 2;   // a [16 x 128] bf16 operand (direction terms / new signs)
@@ -303,13 +304,14 @@ fit_pass_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, uint32_t* __restri
   }
 }
 
-// Row range of a block: about two blocks per SM over all units (one block fits an SM, so a last wave that is nearly
-// empty costs as much as a full one: take the first count from there whose last wave is at least 90 % full), never
+// Row range of a block: from about two blocks per SM over all units, the first count whose last wave of one-block-per-SM
+// is at least 90 % full (32 units on 148 SMs: 23 blocks per unit = 4.97 waves; fewer, longer blocks were measured slower,
+// above all on ragged batches where a block is the unit of balance), never
 // more tiles per warpgroup than the agreement counters hold and never fewer rows than the CUDA-core pass's blocks
 // (the workspace is sized for those).
 void plan(const bpc_ctx* ctx, int* bpu_out, int* rows_out) {
   const int n_max = ctx->cfg.n_max;
-  int bpu = (2 * ctx->sm_count + ctx->units - 1) / ctx->units;
+  int bpu = (kPlanWaves * ctx->sm_count + ctx->units - 1) / ctx->units;
   if (bpu < 1) bpu = 1;
   for (int tries = 0; tries < 16; ++tries) {
     const int rem = (int)(((long long)ctx->units * bpu) % ctx->sm_count);
