@@ -16,9 +16,9 @@
 // the accumulator columns that still wait for their decisions.  That leaves 1 984 of the 8 128 sign-dependent FMAs per
 // key (128 bits) on the CUDA cores.  The small operands use the K-major layout without swizzle (8-row x 16-byte core
 // matrices; leading-dimension offset = distance between core matrices along K, stride offset = 128 bytes along M/N).
-// A block holds two warpgroups, which share the projection rows and the Gram operands in shared memory and otherwise
+// A block holds three warpgroups, which share the projection rows and the Gram operands in shared memory and otherwise
 // run independent pipelines (own key tile, own accumulator columns, own mbarrier, own hardware barrier), so one
-// warpgroup's sweep covers the other's MMA round trips; the next key tile of a warpgroup is copied in while it sweeps.
+// warpgroup's sweep covers the others' MMA round trips; the next key tile of a warpgroup is copied in while it sweeps.
 //
 // Waits on the MMA-completion mbarrier are bounded: on expiry the block raises the device error word, still
 // releases its tensor memory and returns.
