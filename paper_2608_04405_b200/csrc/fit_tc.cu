@@ -207,6 +207,15 @@ fit_pass_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, uint32_t* __restri
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       issue_dot(a);
     }
+    // The channel-sum MMA of the previous tile runs ahead of this tile's dot product in the tensor pipe; once it has
+    // completed, its operands (the sign row and the other tile buffer) are free: the next tile's copy starts as early
+    // as possible, because the buffer count, not the arithmetic, bounds this kernel.
+    if (pend2) {
+      if (!mbar_wait(bar2, ph2)) timed_out_g[grp] = 1;
+      ph2 ^= 1u;
+      pend2 = false;
+    }
+    if (tl + kGroups < ntile) load_tile(tl + kGroups, buf ^ 1);
     // sum_j u_j (v_j . d) from the table, four partial sums in a fixed order
     float s4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -219,14 +228,6 @@ fit_pass_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, uint32_t* __restri
     tmem_ld16(tm_d1 + lane_off, d1);
     const float tk = (d1[0] + d1[1]) + d1[2];                        // K_row . d: the three terms of d
     const bool pos = (tk - tc) >= 0.f;
-    // The channel-sum MMA of the previous tile was issued before this tile's dot product, which has completed: its
-    // operands (the sign row and the other tile buffer) are free.
-    if (pend2) {
-      if (!mbar_wait(bar2, ph2)) timed_out_g[grp] = 1;
-      ph2 ^= 1u;
-      pend2 = false;
-    }
-    if (tl + kGroups < ntile) load_tile(tl + kGroups, buf ^ 1);
     *reinterpret_cast<uint16_t*>(bu_s + small_off(0, gtid)) = live ? (pos ? (uint16_t)0x3F80u : (uint16_t)0xBF80u) : (uint16_t)0u;
     if (live) {
       hrow[it >> 5] = mine[it >> 5] | ((pos ? 1u : 0u) << (it & 31));
