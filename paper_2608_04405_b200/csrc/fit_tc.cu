@@ -1,4 +1,4 @@
-// Tensor-core pass of Algorithm 1 (bf16 caches, codes of up to 128 bits): one pass over the keys per bit.
+// Tensor-core pass of Algorithm 1 (bf16 caches): one pass over the keys per bit.
 //
 // Per bit i the pass needs, for every key row, the decision value
 //     t = R_row . d = K_row . d - sum_{j<i} u_j (v_j . d)
@@ -180,7 +180,10 @@ fit_pass_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, uint32_t* __restri
     for (int w = 0; w < WORDS; ++w) v[w] = 0u;
     if (it > 0 && r < row_end) {
       const uint32_t* src = hfit + ((size_t)unit * n_max + r) * WORDS;
-      if constexpr (WORDS == 4) { const uint4 q = *reinterpret_cast<const uint4*>(src); v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w; }
+      if constexpr (WORDS == 8) {
+        const uint4 q = *reinterpret_cast<const uint4*>(src), q2 = *reinterpret_cast<const uint4*>(src + 4);
+        v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w; v[4] = q2.x; v[5] = q2.y; v[6] = q2.z; v[7] = q2.w;
+      } else if constexpr (WORDS == 4) { const uint4 q = *reinterpret_cast<const uint4*>(src); v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w; }
       else if constexpr (WORDS == 2) { const uint2 q = *reinterpret_cast<const uint2*>(src); v[0] = q.x; v[1] = q.y; }
       else v[0] = src[0];
     }
@@ -270,30 +273,25 @@ fit_pass_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, uint32_t* __restri
   // adds the totals of bits l, 32 + l, ... to the block's counters
   {
     constexpr int PT = kPlanes + 5;
-    uint32_t s[PT][WORDS];
 #pragma unroll
-    for (int k = 0; k < PT; ++k)
+    for (int w = 0; w < WORDS; ++w) {                                // one code word at a time (registers)
+      uint32_t s[PT];
 #pragma unroll
-      for (int w = 0; w < WORDS; ++w) s[k][w] = k < kPlanes ? pl[k][w] : 0u;
+      for (int k = 0; k < PT; ++k) s[k] = k < kPlanes ? pl[k][w] : 0u;
 #pragma unroll
-    for (int st = 0; st < 5; ++st) {
-#pragma unroll
-      for (int w = 0; w < WORDS; ++w) {
+      for (int st = 0; st < 5; ++st) {
         uint32_t carry = 0u;
 #pragma unroll
         for (int k = 0; k < kPlanes + st + 1; ++k) {
-          const uint32_t o = __shfl_xor_sync(0xffffffffu, s[k][w], 1 << st);
-          const uint32_t x = s[k][w];
-          s[k][w] = x ^ o ^ carry;
+          const uint32_t o = __shfl_xor_sync(0xffffffffu, s[k], 1 << st);
+          const uint32_t x = s[k];
+          s[k] = x ^ o ^ carry;
           carry = (x & o) | (carry & (x ^ o));
         }
       }
-    }
-#pragma unroll
-    for (int w = 0; w < WORDS; ++w) {
       int c = 0;
 #pragma unroll
-      for (int k = 0; k < PT; ++k) c += (int)((s[k][w] >> lane) & 1u) << k;
+      for (int k = 0; k < PT; ++k) c += (int)((s[k] >> lane) & 1u) << k;
       if (c) atomicAdd(&cnt_s[32 * w + lane], c);
     }
   }
@@ -330,7 +328,7 @@ void plan(const bpc_ctx* ctx, int* bpu_out, int* rows_out) {
 }  // namespace
 
 bool bpc_fit_tc_covers(const bpc_ctx* ctx) {
-  return ctx->cfg.kv_dtype == BPC_BF16 && ctx->cfg.code_bits <= 128 && !ctx->no_tc_encode;
+  return ctx->cfg.kv_dtype == BPC_BF16 && !ctx->no_tc_encode;
 }
 
 void bpc_fit_tc_geometry(const bpc_ctx* ctx, int* blocks_per_unit, int* rows_per_block) { plan(ctx, blocks_per_unit, rows_per_block); }
@@ -351,7 +349,7 @@ cudaError_t bpc_launch_fit_pass_tc(bpc_ctx* ctx, const void* k_cache, uint32_t* 
     fit_pass_tc_kernel<W><<<grid, kThreads, smem, stream>>>((const __nv_bfloat16*)k_cache, hfit, dir, dots, partials, agree, \
                                                             ctx->unit_lens, ctx->dev_err, c.n_max, ctx->row_stride, it, bpu, rows); \
   } while (0)
-  if (b == 32) BPC_FIT_TC(1); else if (b == 64) BPC_FIT_TC(2); else if (b == 128) BPC_FIT_TC(4); else return cudaErrorNotSupported;
+  if (b == 32) BPC_FIT_TC(1); else if (b == 64) BPC_FIT_TC(2); else if (b == 128) BPC_FIT_TC(4); else if (b == 256) BPC_FIT_TC(8); else return cudaErrorNotSupported;
 #undef BPC_FIT_TC
   return cudaGetLastError();
 }

