@@ -73,8 +73,9 @@ class Session:
         self.units = spec.batch * spec.n_kv_heads
         self.fit_ws = None
 
-    def fit(self):
-        self.fit_ws = torch.zeros(self.ctx.fit_workspace_bytes(), dtype=torch.uint8, device="cuda")
+    def fit(self, dirty_workspace: bool = False):
+        """dirty_workspace: hand bpc_fit a workspace full of ones (the library must not rely on its contents)."""
+        self.fit_ws = torch.full((self.ctx.fit_workspace_bytes(),), 255 if dirty_workspace else 0, dtype=torch.uint8, device="cuda")
         self.ctx.fit(self.k_cache, self.v_star, self.fit_ws)
         torch.cuda.synchronize()
         self.P, self.Ph, self.gram = self.ctx.get_projection()

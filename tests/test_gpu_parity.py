@@ -337,13 +337,13 @@ def test_tensor_core_fit_pass_agrees_with_cuda_core_pass(bits, n):
                              code_bits=bits, steps=1)
     sess = H.Session(spec, gen_device="cuda" if n > 20000 else "cpu")
     rep = {}
-    sess.fit()                                                # tensor-core pass
+    sess.fit(dirty_workspace=True)                            # tensor-core pass; the workspace holds leftovers
     H.check_fit(sess, [0, 1], rep)
     err_tc = rep["fit_reconstruction_err_over_K"]
     P_tc, H_tc = sess.P.clone(), [sess.hfit_bits(u) for u in range(2)]
     sess.ctx.debug_set_tensor_core_encode(False)
     try:
-        sess.fit()                                            # CUDA-core pass
+        sess.fit(dirty_workspace=True)                        # CUDA-core pass
     finally:
         sess.ctx.debug_set_tensor_core_encode(True)
     rep_cc = {}
