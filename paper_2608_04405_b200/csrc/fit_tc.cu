@@ -186,12 +186,6 @@ fit_pass_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, uint32_t* __restri
       } else if constexpr (WORDS == 4) { const uint4 q = *reinterpret_cast<const uint4*>(src); v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w; }
       else if constexpr (WORDS == 2) { const uint2 q = *reinterpret_cast<const uint2*>(src); v[0] = q.x; v[1] = q.y; }
       else v[0] = src[0];
-      // Only the bits decided so far count: the workspace may hold anything from an earlier fit (the pass of bit
-      // `it` is the first to write that bit, and it ORs it into the word).
-      const int wi = it >> 5;
-      const uint32_t below = (1u << (it & 31)) - 1u;
-#pragma unroll
-      for (int w = 0; w < WORDS; ++w) v[w] = w < wi ? v[w] : (w == wi ? (v[w] & below) : 0u);
     }
   };
   uint32_t nxt[WORDS];
@@ -204,7 +198,7 @@ fit_pass_tc_kernel(const __nv_bfloat16* __restrict__ k_cache, uint32_t* __restri
     const int row = row0_blk + tl * kTileKeys + gtid;
     const bool live = row < row_end;
     uint32_t* hrow = hfit + ((size_t)unit * n_max + (live ? row : row0_blk)) * WORDS;
-    uint32_t mine[WORDS];                                            // the key's earlier bits (bits >= it masked off)
+    uint32_t mine[WORDS];                                            // the key's earlier bits (bits >= it are zero: the fit clears the code words first)
 #pragma unroll
     for (int w = 0; w < WORDS; ++w) mine[w] = nxt[w];                // (requested one turn ago)
     load_words(nxt, row + kGroups * kTileKeys);
