@@ -153,6 +153,20 @@ class Layer:
         self.k_new, self.v_new = w.new_kv(self.lens0)
         self.out = torch.zeros(spec.batch, spec.n_q_heads, spec.head_dim, dtype=torch.float32, device="cuda")
 
+    def reconstruction_error(self, rows=16384):
+        """Sanity figure of the prefill side, computed with torch from what the library wrote: ||K - H P_h|| / ||K|| over
+        the first keys of unit 0 (H = the cache codes as +-1).  A fitted projection gives well below 1; anything else
+        means the fit or the encode went wrong, and the benchmark refuses to time that state."""
+        n = min(int(self.lens0[0]), rows)
+        _, Ph, _ = self.ctx.get_projection()
+        K = self.k_cache[0, 0, :n].float()
+        words = self.codes[0, 0, :n]
+        nbit = 32 if words.dtype == torch.int32 else 64
+        shifts = torch.arange(nbit, device=words.device, dtype=words.dtype)
+        bits = ((words.unsqueeze(-1) >> shifts) & 1).reshape(n, -1)[:, :self.w.spec.code_bits]
+        Hm = bits.float() * 2.0 - 1.0
+        return ((K - Hm @ Ph[0].float()).norm() / K.norm()).item()
+
     def step(self):
         """One decode step: cache write of the new (k, v) + decode, as the single fused launch."""
         self.ctx.append_decode_attn(self.k_new, self.v_new, self.k_cache, self.v_cache, self.codes, self.q,
@@ -262,6 +276,9 @@ def run_ours(args):
               for i in range(L)]
     fit_ws[0] = None
     torch.cuda.empty_cache()
+    recon = [ly.reconstruction_error() for ly in layers]
+    if not all(r < 1.0 for r in recon):
+        raise RuntimeError("prefill sanity check failed: ||K - H P_h|| / ||K|| per layer replica = %s" % recon)
     fit_power2_ms = None
     if not args.profile:
         # one more fit of layer 0's keys with two power iterations per bit (the variant of Algorithm 1's component search)
@@ -579,7 +596,8 @@ def run_ours(args):
                     # the encode reads every key row once and writes one code per key
                     "encode_algorithmic_bytes": n_keys * (spec.head_dim * spec.esz + spec.code_bits // 8),
                     "encode_hbm_gbs": n_keys * (spec.head_dim * spec.esz + spec.code_bits // 8) / (enc_ms * 1e-3) / 1e9,
-                    "encode_frac_of_hbm_peak": n_keys * (spec.head_dim * spec.esz + spec.code_bits // 8) / (enc_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+                    "encode_frac_of_hbm_peak": n_keys * (spec.head_dim * spec.esz + spec.code_bits // 8) / (enc_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                    "reconstruction_err_over_K_per_layer_replica": recon},
         "device_error_word": err,
         "needle_recall": hits / max(1, total_needles),
         "paper_context": "paper reports up to 3.56x end-to-end decode speed-up over FlashAttention-2 on 8 data-center GPUs "
@@ -658,7 +676,8 @@ def run_all_configs(args):
                 "timing": {"reps": args.reps, "us_per_step_min": min(rep_ms) / K * 1e3, "us_per_step_max": max(rep_ms) / K * 1e3},
                 "clocks": clocks, "roofline": _roofline(spec, lens_now, ms_step, peaks),
                 "prefill_ms_per_layer": {"fit": layers[-1].fit_ms, "encode": layers[-1].encode_ms,
-                                         "keys": int(sum(layers[-1].lens0)) * spec.n_kv_heads},
+                                         "keys": int(sum(layers[-1].lens0)) * spec.n_kv_heads,
+                                         "reconstruction_err_over_K": [ly.reconstruction_error() for ly in layers]},
                 "device_error_word": max(ly.ctx.last_device_error() for ly in layers)}
         try:                                       # the paper's own score (sign + 7 magnitude planes) on the same workload
             for ly in layers:
