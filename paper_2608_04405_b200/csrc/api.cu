@@ -628,6 +628,7 @@ bpc_status bpc_debug_force_streaming(bpc_ctx* ctx, int32_t on) {
   if (ctx == nullptr) return BPC_ERR_INVALID_ARG;
   if (on != 0 && (ctx->cfg.score_mode != BPC_SCORE_HAMMING || ctx->cfg.eas_ppm != 0)) return BPC_ERR_UNSUPPORTED;
   ctx->force_streaming = on != 0;
+  ctx->decode_smem_set = 0;                                 // another kernel variant: its function attributes are set at its first launch
   cudaError_t e = bpc_plan_decode_geometry(ctx);
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   return ctx->cluster_size > 0 ? BPC_OK : BPC_ERR_UNSUPPORTED;

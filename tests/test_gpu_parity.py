@@ -522,6 +522,23 @@ def test_streaming_selection_forced_at_ordinary_sizes(dtype, bits, group, n, clu
     print(rep)
 
 
+def test_selection_variant_switched_on_a_live_context():
+    """The diagnostic switch between the in-shared-memory and the streaming selection on a context that has already
+    launched the other variant (each variant is its own kernel, with function attributes of its own)."""
+    H = _harness()
+    spec = CONFIGS[1].scaled(name="switch", wid=75, n_ctx=30000, n_kv_heads=2, n_q_heads=8, steps=1)
+    sess = H.Session(spec)
+    rep = {}
+    sess.fit(); sess.encode()
+    q, _ = sess.w.queries(sess.lens)
+    q = q.cuda()
+    H.check_decode(sess, q, [0, 1], rep)
+    for on in (True, False, True):
+        sess.ctx.debug_force_streaming(on)
+        assert sess.ctx.uses_streaming() == on
+        H.check_decode(sess, q, [0, 1], rep)
+
+
 @pytest.mark.parametrize("dtype,bits,group,n", [("bf16", 128, 4, 9000), ("f32", 64, 2, 5000), ("bf16", 256, 8, 6000), ("bf16", 32, 4, 7000)])
 def test_quality_yardsticks(dtype, bits, group, n):
     """The TOPK (Oracle) selector and dense attention (appendix "Baseline Methods"; cosine-similarity table), and the two
