@@ -443,13 +443,17 @@ def test_cfg3_ragged_sweep_code_length_and_budget(bits):
     print(sess.lens, rep)
 
 
-def test_cfg3_full_batch_sampled_units():
-    """Config 3 at full size (batch 16, 128 units, one block per unit) in the benchmark's launch configuration."""
+@pytest.mark.parametrize("bits", [64, 128, 256])
+def test_cfg3_full_batch_sampled_units(bits):
+    """Config 3 at full size (batch 16, 128 units, one block per unit) in the benchmark's launch configuration, at the
+    three code lengths of its sweep: the fit and the encode of one unit each (at 256 bits the encode is two launches),
+    then fused decode steps."""
     H = _harness()
-    spec = CONFIGS[3]
+    spec = CONFIGS[3].scaled(code_bits=bits)
     sess = H.Session(spec, gen_device="cuda", interleaved=True)
     rep = {}
-    sess.fit(); sess.encode()
+    sess.fit(dirty_workspace=True); H.check_fit(sess, [41], rep)
+    sess.encode(); H.check_encode(sess, [100], rep, max_keys=4096)
     _decode_loop(sess, 2, [0, 77, 127], rep, H, fused=True)
     print(sess.ctx.get_cluster_size(), rep)
 
