@@ -299,6 +299,18 @@ def test_weighted_scores_config4_head_layout_full_size():
     print(rep)
 
 
+def test_weighted_scores_config2_full_size_fused():
+    """The weighted step the benchmark times next to the headline: config 2 at full size (batch 4, clusters of 4),
+    cache write fused into the launch, Algorithm 3's score; sampled units."""
+    H = _harness()
+    from paper_2608_04405_b200 import binding as B
+    sess = H.Session(CONFIGS[2].scaled(steps=2), gen_device="cuda", interleaved=True, score_mode=B.BPC_SCORE_WEIGHTED7)
+    rep = {}
+    sess.fit(); sess.encode()
+    _decode_loop(sess, 2, [0, 13, 31], rep, H, fused=True)
+    print(sess.ctx.get_cluster_size(), rep)
+
+
 @pytest.mark.parametrize("bits", [32, 64, 128, 256])
 def test_tensor_core_encode_agrees_with_cuda_core_encode(bits):
     """bpc_encode_keys on the tcgen05 path and on the CUDA-core path (diagnostic switch) against each other and
