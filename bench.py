@@ -741,7 +741,7 @@ def run_sweep(args):
             ms = _time_graph(g, lambda: None) / K
             err = max(ly.ctx.last_device_error() for ly in layers)
             rows.append({"context": n_ctx, "batch": batch, "budget": budget, "us_per_step": round(ms * 1e3, 2),
-                         "cluster_size": layers[0].ctx.get_cluster_size(), "streaming": layers[0].ctx.uses_streaming(), "layer_replicas": L,
+                         "cluster_size": layers[0].ctx.get_cluster_size(), "streaming": layers[0].ctx.uses_streaming(), "byte_keys": layers[0].ctx.uses_byte_keys(), "layer_replicas": L,
                          "algorithmic_GBps": round(step_bytes / ms / 1e6, 1), "device_error_word": err})
             layers = None
             g = None

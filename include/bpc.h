@@ -289,6 +289,14 @@ bpc_status bpc_debug_set_pdl(bpc_ctx* ctx, int32_t on);
 bpc_status bpc_debug_force_key_shift(bpc_ctx* ctx, int32_t shift);
 bpc_status bpc_debug_set_tensor_core_encode(bpc_ctx* ctx, int32_t on);
 bpc_status bpc_debug_force_streaming(bpc_ctx* ctx, int32_t on);
+/* Byte score keys.  Hamming scores with at most 256 distinct values (G*b/2 <= 255 for an even number G of query heads
+ * per KV head, G*b <= 255 for an odd one; no safeguard) can be kept one byte per key in shared memory, which lets a
+ * thread block hold 2.5 times as many keys.  The library takes that kernel variant by itself when the 16-bit keys
+ * would need the streaming selection or more waves of clusters (bpc_uses_byte_keys reports the choice); the result is
+ * the same bit for bit.  bpc_debug_force_byte_keys(ctx, 1) takes it wherever it is possible (BPC_ERR_UNSUPPORTED
+ * where it is not), -1 never, 0 leaves the choice to the library; each call re-plans the launch geometry. */
+int32_t bpc_uses_byte_keys(bpc_ctx* ctx);
+bpc_status bpc_debug_force_byte_keys(bpc_ctx* ctx, int32_t mode);
 bpc_status bpc_last_device_error(bpc_ctx* ctx, int32_t* host_out, void* stream);
 int32_t    bpc_last_cuda_error(bpc_ctx* ctx);
 int64_t    bpc_launch_count(bpc_ctx* ctx);

@@ -76,6 +76,8 @@ def _load() -> ctypes.CDLL:
         "bpc_debug_force_key_shift": (i32, [vp, i32]),
         "bpc_debug_set_tensor_core_encode": (i32, [vp, i32]),
         "bpc_debug_force_streaming": (i32, [vp, i32]),
+        "bpc_debug_force_byte_keys": (i32, [vp, i32]),
+        "bpc_uses_byte_keys": (i32, [vp]),
         "bpc_uses_work_items": (i32, [vp]),
         "bpc_work_item_grid": (i32, [vp]),
         "bpc_debug_set_decode_path": (i32, [vp, i32]),
@@ -101,7 +103,7 @@ EXPORTS = ["bpc_create", "bpc_destroy", "bpc_codes_bytes", "bpc_fit_workspace_by
            "bpc_debug_set_buffers", "bpc_debug_set_phase_timer",
            "bpc_set_cluster_size", "bpc_plan_cluster_size",
            "bpc_get_cluster_size", "bpc_uses_streaming", "bpc_status_of_device_error", "bpc_debug_set_pdl", "bpc_debug_force_key_shift",
-           "bpc_debug_set_tensor_core_encode", "bpc_debug_force_streaming", "bpc_uses_work_items", "bpc_work_item_grid", "bpc_debug_set_decode_path",
+           "bpc_debug_set_tensor_core_encode", "bpc_debug_force_streaming", "bpc_debug_force_byte_keys", "bpc_uses_byte_keys", "bpc_uses_work_items", "bpc_work_item_grid", "bpc_debug_set_decode_path",
            "bpc_debug_set_work_item_geometry", "bpc_debug_set_work_item_trace", "bpc_last_device_error", "bpc_last_cuda_error", "bpc_launch_count", "bpc_version"]
 
 
@@ -324,6 +326,13 @@ class Context:
     def debug_set_tensor_core_encode(self, on: bool) -> None:
         """False: bpc_encode_keys and the passes of bpc_fit run their CUDA-core kernels (cross-checks)."""
         _check(lib.bpc_debug_set_tensor_core_encode(self._h, 1 if on else 0), "bpc_debug_set_tensor_core_encode")
+
+    def uses_byte_keys(self) -> bool:
+        return bool(lib.bpc_uses_byte_keys(self._h))
+
+    def debug_force_byte_keys(self, mode: int) -> None:
+        """1 = byte score keys wherever possible, -1 = never, 0 = the library decides."""
+        _check(lib.bpc_debug_force_byte_keys(self._h, mode), "bpc_debug_force_byte_keys")
 
     def debug_force_streaming(self, on: bool) -> None:
         _check(lib.bpc_debug_force_streaming(self._h, 1 if on else 0), "bpc_debug_force_streaming")

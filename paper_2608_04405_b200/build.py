@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libbpc.so")
-SOURCES = ["api.cu", "prefill.cu", "decode_sched.cu", "decode_bf16.cu", "decode_f32.cu", "decode_bf16_w7.cu", "decode_f32_w7.cu", "decode_bf16_eas.cu", "decode_f32_eas.cu", "decode_bf16_stream.cu", "decode_f32_stream.cu", "encode_tc.cu", "fit_tc.cu", "noalloc.cu", "yardstick.cu"]
+SOURCES = ["api.cu", "prefill.cu", "decode_sched.cu", "decode_bf16.cu", "decode_f32.cu", "decode_bf16_w7.cu", "decode_f32_w7.cu", "decode_bf16_eas.cu", "decode_f32_eas.cu", "decode_bf16_stream.cu", "decode_f32_stream.cu", "decode_bf16_k8.cu", "decode_f32_k8.cu", "encode_tc.cu", "fit_tc.cu", "noalloc.cu", "yardstick.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]

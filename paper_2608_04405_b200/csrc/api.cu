@@ -15,6 +15,10 @@ cudaError_t bpc_decode_limits_bf16_eas(const bpc_ctx*, int, int*, int*, size_t*)
 cudaError_t bpc_decode_limits_f32_eas(const bpc_ctx*, int, int*, int*, size_t*);
 cudaError_t bpc_launch_decode_bf16_stream(bpc_ctx*, const DecodeParams&, cudaStream_t);
 cudaError_t bpc_launch_decode_f32_stream(bpc_ctx*, const DecodeParams&, cudaStream_t);
+cudaError_t bpc_launch_decode_bf16_k8(bpc_ctx*, const DecodeParams&, cudaStream_t);
+cudaError_t bpc_launch_decode_f32_k8(bpc_ctx*, const DecodeParams&, cudaStream_t);
+cudaError_t bpc_decode_limits_bf16_k8(const bpc_ctx*, int, int*, int*, size_t*);
+cudaError_t bpc_decode_limits_f32_k8(const bpc_ctx*, int, int*, int*, size_t*);
 cudaError_t bpc_launch_decode_bf16_w7(bpc_ctx*, const DecodeParams&, cudaStream_t);
 cudaError_t bpc_launch_decode_f32_w7(bpc_ctx*, const DecodeParams&, cudaStream_t);
 cudaError_t bpc_decode_limits_bf16_w7(const bpc_ctx*, int, int*, int*, size_t*);
@@ -197,6 +201,25 @@ cudaError_t bpc_plan_decode_geometry(bpc_ctx* ctx) {
   ctx->chunk_cap_limit = cap;
   ctx->cluster_size = choose_cluster(ctx, cap, ctx->max_cluster);
   ctx->streaming = false;
+  ctx->byte_keys = false;
+  // Byte score keys (Hamming scores with at most 256 distinct values, no safeguard): a block holds 2.5 times the keys,
+  // so contexts of a million keys and more fit clusters that are all resident at once.  Taken when the 16-bit plan
+  // would need the streaming selection or more waves of clusters than the byte plan (same kernel resources: the
+  // occupancy answers of the plain variant are reused).
+  if (ctx->cfg.score_mode == BPC_SCORE_HAMMING && ctx->cfg.eas_ppm == 0 && hist_shift(ctx) == 0 && hist_bins(ctx) <= 256 &&
+      ctx->force_byte_keys >= 0 && !ctx->force_streaming) {
+    int cap8 = 0;
+    e = ctx->cfg.kv_dtype == BPC_BF16 ? bpc_decode_limits_bf16_k8(ctx, hist_bins(ctx), nullptr, &cap8, nullptr)
+                                      : bpc_decode_limits_f32_k8(ctx, hist_bins(ctx), nullptr, &cap8, nullptr);
+    if (e != cudaSuccess) return e;
+    const int cs8 = choose_cluster(ctx, cap8, ctx->max_cluster);
+    auto waves = [&](int cs) { return (ctx->units + ctx->max_active[cs] - 1) / ctx->max_active[cs]; };
+    if (cs8 > 0 && (ctx->force_byte_keys > 0 || ctx->cluster_size == 0 || waves(cs8) < waves(ctx->cluster_size))) {
+      ctx->byte_keys = true;
+      ctx->cluster_size = cs8;
+      ctx->chunk_cap_limit = cap8;
+    }
+  }
   const bool forced = ctx->force_streaming;                 // diagnostic switch: two-pass selection at any size
   if ((ctx->cluster_size == 0 || forced) && ctx->cfg.score_mode == BPC_SCORE_HAMMING && ctx->cfg.eas_ppm == 0) {
     // Units too long for the largest cluster's shared memory: no score is stored, the codes are read twice.  The
@@ -557,6 +580,9 @@ static bpc_status decode_common(bpc_ctx* ctx, const void* k_new, const void* v_n
   if (ctx->streaming)
     e = c.kv_dtype == BPC_BF16 ? bpc_launch_decode_bf16_stream(ctx, p, (cudaStream_t)stream)
                                : bpc_launch_decode_f32_stream(ctx, p, (cudaStream_t)stream);
+  else if (ctx->byte_keys)
+    e = c.kv_dtype == BPC_BF16 ? bpc_launch_decode_bf16_k8(ctx, p, (cudaStream_t)stream)
+                               : bpc_launch_decode_f32_k8(ctx, p, (cudaStream_t)stream);
   else if (c.score_mode == BPC_SCORE_WEIGHTED7)
     e = c.kv_dtype == BPC_BF16 ? bpc_launch_decode_bf16_w7(ctx, p, (cudaStream_t)stream)
                                : bpc_launch_decode_f32_w7(ctx, p, (cudaStream_t)stream);
@@ -633,6 +659,18 @@ bpc_status bpc_debug_force_streaming(bpc_ctx* ctx, int32_t on) {
   if (e != cudaSuccess) return cuda_fail(ctx, e);
   return ctx->cluster_size > 0 ? BPC_OK : BPC_ERR_UNSUPPORTED;
 }
+
+bpc_status bpc_debug_force_byte_keys(bpc_ctx* ctx, int32_t mode) {
+  if (ctx == nullptr || mode < -1 || mode > 1) return BPC_ERR_INVALID_ARG;
+  ctx->force_byte_keys = mode;
+  ctx->decode_smem_set = 0;                                 // possibly another kernel variant: attributes at its first launch
+  cudaError_t e = bpc_plan_decode_geometry(ctx);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  if (ctx->cluster_size == 0) return BPC_ERR_UNSUPPORTED;
+  return (mode > 0 && !ctx->byte_keys) ? BPC_ERR_UNSUPPORTED : BPC_OK;
+}
+
+int32_t bpc_uses_byte_keys(bpc_ctx* ctx) { return (ctx != nullptr && ctx->byte_keys) ? 1 : 0; }
 
 bpc_status bpc_status_of_device_error(int32_t error_word) { return error_word == 0 ? BPC_OK : BPC_ERR_DEVICE; }
 

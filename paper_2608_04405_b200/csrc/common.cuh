@@ -46,6 +46,8 @@ struct bpc_ctx {
   int32_t* lens_staging;    // pinned, [BPC_LENS_SLOTS][units]: per-unit lengths on their way to the device
   cudaEvent_t lens_event[BPC_LENS_SLOTS];
   int lens_slot;
+  bool byte_keys;           // Hamming scores stored as byte keys (kernel variant 3): 2.5 times the keys per block
+  int force_byte_keys;      // diagnostic switch: 0 = the library decides, 1 = byte keys wherever they are possible, -1 = never
   bool force_streaming;     // diagnostic switch: streaming selection at any size
   bool no_tc_encode;        // diagnostic switch: CUDA-core encode kernel
   int key_shift_min;        // diagnostic switch: weighted scores stored with at least this right shift

@@ -79,7 +79,12 @@ struct DecodeSmem {
   __host__ __device__ static constexpr size_t hashpart_bytes() { return (size_t)NT * GV * 8; }
 
   size_t off_hist, off_tot, off_qf, off_pd, off_idx, off_cta, off_small, off_union, total;
-  __host__ __device__ DecodeSmem(int chunk_cap, int nbins, int stages) {
+  // bytes of the score keys of a block: 16-bit keys in padded 32-key segments, or (key_bytes == 1) plain bytes
+  __host__ __device__ static constexpr size_t score_bytes(int chunk_cap, int key_bytes) {
+    return key_bytes == 1 ? (size_t)((chunk_cap + kSegKeys - 1) / kSegKeys) * kSegKeys
+                          : (size_t)((chunk_cap + kSegKeys - 1) / kSegKeys) * kSegSlots * 2;
+  }
+  __host__ __device__ DecodeSmem(int chunk_cap, int nbins, int stages, int key_bytes = 2) {
     const size_t nb = a16((size_t)nbins * 4);
     off_hist = 0;
     off_tot = off_hist + nb;
@@ -89,7 +94,7 @@ struct DecodeSmem {
     off_cta = off_idx + kIdxTile * 4;                                // merge inbox: acc_t[GP * (128 + 2 * 16) + 16]
     off_small = a16(off_cta + ((size_t)GP * (BPC_D + 2 * BPC_MAX_CLUSTER) + BPC_MAX_CLUSTER) * sizeof(acc_t));
     off_union = a16(off_small + sizeof(SmallState));
-    size_t u = (size_t)((chunk_cap + kSegKeys - 1) / kSegKeys) * kSegSlots * 2;   // score keys
+    size_t u = score_bytes(chunk_cap, key_bytes);                                  // score keys
     if (u < part_bytes()) u = part_bytes();                                      // block-level merge
     if (u < hashpart_bytes()) u = hashpart_bytes();                              // query-hash partial sums
     if (u < (size_t)stages * kStageBytes) u = (size_t)stages * kStageBytes;      // gather ring
@@ -355,12 +360,16 @@ __device__ __noinline__ int rescore_key(const uint32_t* code, const uint32_t* si
 // VAR selects what is compiled in besides the plain path (VAR = 0): 1 = the error-aware safeguard (a static
 // hard-to-hash set that is always attended); 2 = the streaming selection for units whose scores do not fit the
 // cluster's shared memory (no score is stored: the scan keeps one histogram per warp over that warp's contiguous key
-// range, and after the threshold is known every warp reads its codes a second time and emits its selection in order).
+// range, and after the threshold is known every warp reads its codes a second time and emits its selection in order);
+// 3 = byte score keys: Hamming scores with at most 256 distinct keys are stored one byte per key, unpadded, so that a
+// block holds 2.5 times as many (contexts of a million keys and more in clusters that are all resident at once).
 template <typename KV, int GP, int W32, int MODE, int VAR>
 __global__ void __launch_bounds__((DecodeSmem<KV, GP, W32>::NT), 1)
 bpc_decode_kernel(const DecodeParams p) {
   constexpr int EAS = VAR == 1 ? 1 : 0;
   constexpr bool STREAM = VAR == 2;
+  constexpr bool K8 = VAR == 3;
+  static_assert(!K8 || MODE == 0, "byte keys are for Hamming scores");
   typedef DecodeSmem<KV, GP, W32> L;
   typedef typename L::acc_t acc_t;
   constexpr int NT = L::NT, NW = L::NW, B = L::B;
@@ -450,7 +459,7 @@ bpc_decode_kernel(const DecodeParams p) {
 
   const int nbins = p.nbins;
   const int hsh = p.hist_shift;                              // histogram bin = score key >> hsh (0 in Hamming mode)
-  const L plan(p.chunk_cap, nbins, p.stages);
+  const L plan(p.chunk_cap, nbins, p.stages, K8 ? 1 : 2);
   uint32_t* hist = reinterpret_cast<uint32_t*>(smem + plan.off_hist);
   uint32_t* tot = reinterpret_cast<uint32_t*>(smem + plan.off_tot);
   float* qf_s = reinterpret_cast<float*>(smem + plan.off_qf);
@@ -462,6 +471,7 @@ bpc_decode_kernel(const DecodeParams p) {
   SmallState* st = reinterpret_cast<SmallState*>(smem + plan.off_small);
   unsigned char* uni = smem + plan.off_union;
   uint16_t* sc = reinterpret_cast<uint16_t*>(uni);
+  [[maybe_unused]] uint8_t* sc8 = uni;                       // (byte-key variant: key i of the block at byte i)
   // Phase stamps (debug): slots 0 and 7 hold the global timer at block start and end, slots 15 and 14 the SM's cycle
   // counter at the same two points, every other slot the cycle counter (cheap to read) at that phase boundary.
 #define BPC_STAMP(i) do { if (p.dbg_times != nullptr && tid == 0) p.dbg_times[(size_t)blockIdx.x * 16 + (i)] = (unsigned long long)clock64(); } while (0)
@@ -477,7 +487,7 @@ bpc_decode_kernel(const DecodeParams p) {
   if (appender && p.residual_correction != 0) {
     const size_t union_bytes = plan.total - plan.off_union;
     const size_t score_bytes = STREAM ? (size_t)NW * nbins * 4      // (streaming: the per-warp histograms sit there)
-                                      : (size_t)((p.chunk_cap + kSegKeys - 1) / kSegKeys) * kSegSlots * 2;
+                                      : L::score_bytes(p.chunk_cap, K8 ? 1 : 2);
     constexpr size_t kGramPad = 0;
     if (score_bytes + (size_t)B * B * 4 + kGramPad <= union_bytes && L::hashpart_bytes() + (size_t)B * B * 4 + kGramPad <= union_bytes) {
       float* dstg = reinterpret_cast<float*>(uni + union_bytes - (size_t)B * B * 4 - kGramPad);
@@ -693,7 +703,8 @@ bpc_decode_kernel(const DecodeParams p) {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
           const int key = score_key<W32, NP>(h[u], sg, mk);
-          sc[score_slot(base - c0 + u * nts + tid)] = (uint16_t)(key >> ksh);
+          if constexpr (K8) sc8[base - c0 + u * nts + tid] = (uint8_t)key;
+          else sc[score_slot(base - c0 + u * nts + tid)] = (uint16_t)(key >> ksh);
           atomicAdd(&hist[(key >> ksh) >> hsh], 1u);
         }
       }
@@ -788,7 +799,8 @@ bpc_decode_kernel(const DecodeParams p) {
           const int i = i0 + u * nts + tid;
           if (i < c1s) {
             const int key = score_key<W32, NP>(h[u], sg, mk);
-            sc[score_slot(i - c0)] = (uint16_t)(key >> ksh);
+            if constexpr (K8) sc8[i - c0] = (uint8_t)key;
+            else sc[score_slot(i - c0)] = (uint16_t)(key >> ksh);
             atomicAdd(&hist[(key >> ksh) >> hsh], 1u);
           }
         }
@@ -916,7 +928,8 @@ bpc_decode_kernel(const DecodeParams p) {
         for (int pl = 0; pl < NP; ++pl) mk[pl][w] = st->mask[pl][w];
       }
       const int key = score_key<W32, NP>(h, sg, mk);
-      sc[score_slot(n - 1 - c0)] = (uint16_t)(key >> ksh);
+      if constexpr (K8) sc8[n - 1 - c0] = (uint8_t)key;
+      else sc[score_slot(n - 1 - c0)] = (uint16_t)(key >> ksh);
       atomicAdd(&hist[(key >> ksh) >> hsh], 1u);
       if (p.dbg_scores != nullptr) p.dbg_scores[(size_t)unit * p.n_max + (n - 1)] = ((2 * key) << cs) - (st->rsum << cs);
     }
@@ -930,7 +943,7 @@ bpc_decode_kernel(const DecodeParams p) {
   uint32_t* pushed = nullptr;
   {
     const size_t union_bytes = plan.total - plan.off_union;
-    size_t push_off = STREAM ? (size_t)NW * nbins * 4 : (size_t)((p.chunk_cap + kSegKeys - 1) / kSegKeys) * kSegSlots * 2;
+    size_t push_off = STREAM ? (size_t)NW * nbins * 4 : L::score_bytes(p.chunk_cap, K8 ? 1 : 2);
     if (push_off < L::hashpart_bytes()) push_off = L::hashpart_bytes();   // a peer may still be hashing
     push_off = (push_off + 15) & ~(size_t)15;
     if (fast_sel && CS > 1 && push_off + (size_t)CS * nbins * 4 + (size_t)B * B * 4 <= union_bytes)
@@ -1267,14 +1280,33 @@ bpc_decode_kernel(const DecodeParams p) {
         M[q] = 0u; Mgt[q] = 0u;
         const int seg = s0 + tid * spt + q;
         if (q < spt && seg < nseg) {
-          const uint4* src = reinterpret_cast<const uint4*>(sc + (size_t)seg * kSegSlots);
           uint32_t kw[16];
+          if constexpr (K8) {                                // 32 byte keys: two 16-byte reads
+            const uint4* src = reinterpret_cast<const uint4*>(sc8 + (size_t)seg * kSegKeys);
+#pragma unroll
+            for (int v = 0; v < 2; ++v) {
+              const uint4 x = src[v];
+              kw[4 * v] = x.x; kw[4 * v + 1] = x.y; kw[4 * v + 2] = x.z; kw[4 * v + 3] = x.w;
+            }
+          } else {
+          const uint4* src = reinterpret_cast<const uint4*>(sc + (size_t)seg * kSegSlots);
 #pragma unroll
           for (int v = 0; v < 4; ++v) {
             const uint4 x = src[v];
             kw[4 * v] = x.x; kw[4 * v + 1] = x.y; kw[4 * v + 2] = x.z; kw[4 * v + 3] = x.w;
           }
+          }
           uint32_t m = 0;
+          if constexpr (K8) {
+            // four keys per word: a per-byte unsigned compare leaves 0xFF where key >= T; one multiplication moves the
+            // four flags (bits 0, 8, 16, 24 after masking) next to each other: (y * 0x01020408) >> 24
+            const uint32_t T4 = (uint32_t)T * 0x01010101u;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) {
+              const uint32_t ge = __vcmpgeu4(kw[w], T4) & 0x01010101u;
+              m |= (((ge * 0x01020408u) >> 24) & 15u) << (4 * w);
+            }
+          } else {
 #pragma unroll
           for (int w = 0; w < 16; ++w) {
             if (MODE == 0) {                                 // keys < 2048: both halves compared with one addition
@@ -1286,12 +1318,16 @@ bpc_decode_kernel(const DecodeParams p) {
               m |= ((int)(kw[w] >> 16) >= T ? 2u : 0u) << (2 * w);
             }
           }
+          }
           const int valid = len - seg * kSegKeys;
           if (valid < kSegKeys) m &= (1u << valid) - 1u;     // slots past the end of the chunk hold stale bytes
           uint32_t rem = m, mg = 0;
           while (rem) {
             const int j = __ffs(rem) - 1;
             rem &= rem - 1;
+            if constexpr (K8) {
+              if ((int)sc8[(size_t)seg * kSegKeys + j] > T) mg |= 1u << j;
+            } else
             if ((int)sc[(size_t)seg * kSegSlots + j] > T) mg |= 1u << j;
             else if (MODE == 1 && ksh > 0) {                 // stored key == threshold: the dropped bits decide
               const int low = exact_key(seg * kSegKeys + j) & ((1 << ksh) - 1);

@@ -26,8 +26,9 @@ static cudaError_t launch_one(bpc_ctx* ctx, const DecodeParams& p_in, cudaStream
   int optin = 0;
   cudaError_t e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, ctx->device);
   if (e != cudaSuccess) return e;
-  p.stages = L(p.chunk_cap, p.nbins, 3).total <= (size_t)optin ? 3 : 2;
-  const size_t smem = L(p.chunk_cap, p.nbins, p.stages).total;
+  constexpr int kKeyBytes = EAS == 3 ? 1 : 2;               // (variant 3 stores byte score keys)
+  p.stages = L(p.chunk_cap, p.nbins, 3, kKeyBytes).total <= (size_t)optin ? 3 : 2;
+  const size_t smem = L(p.chunk_cap, p.nbins, p.stages, kKeyBytes).total;
   if (smem > (size_t)optin) return cudaErrorInvalidConfiguration;
   if (ctx->decode_smem_set == 0) {                          // function attributes are sticky: set them once
     e = configure_kernel<KV, GP, W32, MODE, EAS>(ctx->device);
@@ -63,9 +64,10 @@ static cudaError_t limits_one(const bpc_ctx* ctx, int nbins, int* max_cluster, i
   if (e != cudaSuccess) return e;
   const size_t fixed = L(0, nbins, 2).off_union;
   const size_t avail = (size_t)optin > fixed + 64 ? (size_t)optin - fixed - 64 : 0;
-  int cap = (int)((avail / (kSegSlots * 2)) * kSegKeys);
+  constexpr int kKeyBytes = EAS == 3 ? 1 : 2;
+  int cap = kKeyBytes == 1 ? (int)(avail > 0x3fffffff ? 0x3fffffff : avail) : (int)((avail / (kSegSlots * 2)) * kSegKeys);
   cap &= ~63;
-  if (L(cap, nbins, 2).total > (size_t)optin) cap = 0;
+  if (L(cap, nbins, 2, kKeyBytes).total > (size_t)optin) cap = 0;
   if (chunk_cap) *chunk_cap = cap;
   if (smem_bytes) *smem_bytes = (size_t)optin;
   if (max_cluster) {

@@ -104,11 +104,12 @@ bpc_status bpc_decode_attn_static(const bpc_config* cfg, const void* q, const vo
 
   const int nbins = ((group * cfg->code_bits) >> ((group % 2 == 0) ? 1 : 0)) + 1;
   if (nbins > 2048) return BPC_ERR_UNSUPPORTED;
+  tmp.force_byte_keys = -1;                                 // this entry point launches the 16-bit-key kernel only
   e = bpc_plan_decode_geometry(&tmp);                       // occupancy queries only; nothing is allocated
   if (e != cudaSuccess) { (void)cudaGetLastError(); return BPC_ERR_CUDA; }
   // only the plain kernel is launched here: contexts too long for a cluster's shared memory (which a context would
   // serve with the streaming selection) are refused
-  if (tmp.cluster_size == 0 || tmp.streaming) return BPC_ERR_UNSUPPORTED;
+  if (tmp.cluster_size == 0 || tmp.streaming || tmp.byte_keys) return BPC_ERR_UNSUPPORTED;
   const int cs = tmp.cluster_size;
   if (chunk_for(cfg->n_max, cs) > tmp.chunk_cap_limit) return BPC_ERR_UNSUPPORTED;
 

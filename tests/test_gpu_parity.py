@@ -501,14 +501,22 @@ def test_fit_with_power_iterations(dtype, bits, n, power):
 
 
 def test_streaming_selection_two_million_keys():
-    """A unit longer than the largest cluster's shared memory holds (the 2M-token point of the paper's latency-vs-context
-    study): the library switches to the streaming selection (per-warp histograms, codes read twice); same checks as
-    everywhere else, on a 2-KV-head model to bound memory: plain and fused steps, fixed budget of 2048 keys."""
+    """A unit longer than the largest cluster's shared memory holds with 16-bit score keys (the 2M-token point of the
+    paper's latency-vs-context study).  The library takes byte keys there when the scores allow it (checked first); with
+    those ruled out it switches to the streaming selection (per-warp histograms, codes read twice), which is what shapes
+    with more than 256 distinct scores get.  Same checks as everywhere else, on a 2-KV-head model to bound memory: plain
+    and fused steps, fixed budget of 2048 keys."""
     H = _harness()
     spec = CONFIGS[1].scaled(name="stream2m", wid=90, batch=1, n_kv_heads=2, n_q_heads=8, n_ctx=2097152, code_bits=64, steps=2)
     sess = H.Session(spec, gen_device="cuda", interleaved=True)
-    assert sess.ctx.uses_streaming()
+    assert sess.ctx.uses_byte_keys() and not sess.ctx.uses_streaming()
     rep = {}
+    sess.fit()
+    sess.encode()
+    q, _ = sess.w.queries(sess.lens)
+    H.check_decode(sess, q.cuda(), [0, 1], rep, budget_count=2048)              # byte keys, the library's own choice
+    sess.ctx.debug_force_byte_keys(-1)
+    assert sess.ctx.uses_streaming()
     sess.fit()
     sess.encode(); H.check_encode(sess, [1], rep, max_keys=4096)
     q, _ = sess.w.queries(sess.lens)
@@ -591,6 +599,64 @@ def test_sweep_shapes_single_word_codes_fixed_budgets(n_ctx, batch):
     q, _ = sess.w.queries(sess.lens)
     H.check_decode(sess, q.cuda(), units, rep, budget_count=2048, append=(k_new.cuda(), v_new.cuda()))
     print(rep)
+
+
+@pytest.mark.parametrize("dtype,bits,group,n,batch,cluster", [("bf16", 64, 4, 30011, 2, 0), ("bf16", 64, 1, 9000, 1, 3), ("bf16", 32, 4, 20000, 1, 0),
+                                                              ("bf16", 128, 2, 9000, 2, 1), ("f32", 64, 2, 6000, 1, 2), ("bf16", 32, 7, 4097, 1, 5)])
+def test_byte_score_keys_forced_at_ordinary_sizes(dtype, bits, group, n, batch, cluster):
+    """Kernel variant with byte score keys (Hamming scores with at most 256 distinct values), forced at ordinary sizes:
+    against the checker stage by stage, plain and fused steps, and bit for bit against the 16-bit-key variant."""
+    H = _harness()
+    spec = CONFIGS[1].scaled(name="k8", wid=76, batch=batch, n_ctx=n, n_ctx_min=max(1, n // 2) if batch > 1 else None, n_kv_heads=2,
+                             n_q_heads=2 * group, code_bits=bits, dtype=dtype, steps=2, rope_base=None if dtype == "f32" else 500000.0)
+    sess = H.Session(spec, cluster_size=cluster)
+    rep = {}
+    sess.fit(); sess.encode()
+    q, _ = sess.w.queries(sess.lens)
+    q = q.cuda()
+    units = [0, sess.units - 1]
+    ref = sess.ctx.decode_attn(q, sess.k_cache, sess.v_cache, sess.codes, budget_ppm=20000).clone()
+    sess.ctx.debug_force_byte_keys(1)
+    assert sess.ctx.uses_byte_keys()
+    if cluster:
+        sess.ctx.set_cluster_size(cluster)
+    for ppm, count in ((20000, 0), (1000000, 0), (0, 7)):
+        H.check_decode(sess, q, units, rep, budget_ppm=ppm, budget_count=count)
+    got = sess.ctx.decode_attn(q, sess.k_cache, sess.v_cache, sess.codes, budget_ppm=20000)
+    torch.cuda.synchronize()
+    assert torch.equal(got, ref), "byte keys and 16-bit keys select and attend the same rows"
+    k_new, v_new = sess.w.new_kv(sess.lens)
+    H.check_decode(sess, q, units, rep, append=(k_new.cuda(), v_new.cuda()))
+    sess.ctx.debug_force_byte_keys(-1)
+    assert not sess.ctx.uses_byte_keys()
+    print(rep)
+
+
+def test_byte_score_keys_are_refused_where_scores_need_more_than_a_byte():
+    H = _harness()
+    from paper_2608_04405_b200 import binding as B
+    spec = CONFIGS[1].scaled(name="k8no", wid=77, n_ctx=4000, n_kv_heads=2, n_q_heads=16, code_bits=64, steps=1)   # 8 heads x 64 bits / 2 = 256
+    sess = H.Session(spec)
+    with pytest.raises(B.BpcError) as e:
+        sess.ctx.debug_force_byte_keys(1)
+    assert e.value.status == 2                                   # BPC_ERR_UNSUPPORTED
+    assert not sess.ctx.uses_byte_keys()
+
+
+def test_million_key_context_takes_byte_keys_by_itself():
+    """One million keys per unit at batch 1 (8 units, 64-bit codes): with 16-bit keys a unit needs 16 blocks, of which
+    only 7 clusters are resident at once; the library takes byte keys and clusters that run in one wave."""
+    H = _harness()
+    spec = CONFIGS[1].scaled(name="mega", wid=78, batch=1, n_ctx=1048576, code_bits=64, steps=2)
+    sess = H.Session(spec, gen_device="cuda", interleaved=True)
+    assert sess.ctx.uses_byte_keys() and not sess.ctx.uses_streaming()
+    rep = {}
+    sess.fit(); sess.encode()
+    q, _ = sess.w.queries(sess.lens)
+    H.check_decode(sess, q.cuda(), [0, 7], rep, budget_count=2048)
+    k_new, v_new = sess.w.new_kv(sess.lens)
+    H.check_decode(sess, q.cuda(), [3], rep, budget_count=1024, append=(k_new.cuda(), v_new.cuda()))
+    print(sess.ctx.get_cluster_size(), rep)
 
 
 @pytest.mark.parametrize("dtype,bits,group,n,cluster", [("bf16", 128, 4, 9000, 0), ("bf16", 128, 4, 9000, 1), ("bf16", 64, 8, 5000, 2),
